@@ -1,0 +1,433 @@
+#!/usr/bin/env python
+"""Benchmark of the GETT contraction path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--dtype bf16]
+    python bench.py --impl reference ...        # the CPU oracle on the host cores
+
+One step = one gett_contract call (pack A/B tiles, macro-kernel, alpha/beta
+update of C; plus the slice reduction when the plan splits K) over one seeded
+synthetic input set.  The headline line is the 8192^3 GEMM control through the
+tensor path; `--all` appends the other workloads and the equal-GEMM ratios under
+"workloads".  Prints exactly one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import (BF16_F32, DTYPE_NAMES, F32, Contraction, TensorSpec, make_inputs,  # noqa: E402
+                       packed_strides, workload)
+
+METRIC = "TFLOP/s per contraction"
+UNIT = "TFLOP/s"
+DTYPE_BY_NAME = {"f32": F32, "bf16": BF16_F32}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"],
+                "bf16_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+# fp32 FMA peak: 148 SMs x 128 lanes x 2 flop at the sampled SM clock (no measured
+# figure exists for it; the clock is the one seen during the timed region).
+def _fp32_peak_tflops(sm_mhz: float) -> float:
+    return 148 * 128 * 2 * sm_mhz * 1e6 / 1e12
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self._stop = index, [], threading.Event()
+        self._t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.index}",
+                                      f"--query-gpu={self.FIELDS}",
+                                      "--format=csv,noheader,nounits"],
+                                     capture_output=True, text=True, timeout=5).stdout.strip()
+                if out:
+                    self.rows.append([x.strip() for x in out.split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.2)
+
+    def __enter__(self):
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=10)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(np.max(mx)),
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def equal_gemm(con: Contraction) -> Contraction:
+    """The plain GEMM with the same M, N, K (Sec. 7: the equal-sized GEMM line)."""
+    M, N, K = con.mnk()
+    return Contraction("equal-gemm", TensorSpec([0, 2], [M, K], [1, M]),
+                       TensorSpec([2, 1], [K, N], [1, K]), TensorSpec([0, 1], [M, N], [1, M]))
+
+
+def roofline_time_s(con, dtype, beta, peaks, fp32_peak):
+    flops = con.flops()
+    peak = peaks["bf16_burst"] if dtype != F32 else fp32_peak
+    t_c = flops / (peak * 1e12)
+    t_m = con.compulsory_bytes(dtype, beta) / (peaks["hbm_gbs"] * 1e9)
+    return max(t_c, t_m), ("hbm" if t_m >= t_c else ("tensor" if dtype != F32 else "alu"))
+
+
+# --------------------------------------------------------------------------- #
+def run_reference(args):
+    """The CPU oracle as it stands, on the host cores, on a bounded sample."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = workload(args.workload)
+    dtype = DTYPE_BY_NAME[args.dtype]
+    con = w.contraction
+    a, b, c = make_inputs(con, dtype, w.dist, w.seed, w.beta)
+    cores = oracle.default_threads()
+    M, N, K = con.mnk()
+    rng = np.random.default_rng(0)
+    npts = max(cores, int(args.ref_macs // max(K, 1)))
+    pts = np.stack([rng.integers(0, e, npts) for e in con.C.extents], axis=1)
+
+    def step():
+        oracle.points(con, dtype, w.alpha, a, b, w.beta, c, pts, threads=cores)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    tflops = 2.0 * npts * K / dt / 1e12
+    sample = f"{npts} random outputs of {con.C.numel} per step ({npts * K:.3g} multiply-adds)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": f"{w.key} {DTYPE_NAMES[dtype]} {M}x{N}x{K}", "sample": sample},
+        "cpu_baseline": {"value": tflops, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": tflops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def cpu_baseline(w, dtype, a, b, c, budget_macs):
+    import oracle
+    con = w.contraction
+    cores = oracle.default_threads()
+    K = con.mnk()[2]
+    npts = max(cores, int(budget_macs // max(K, 1)))
+    rng = np.random.default_rng(0)
+    pts = np.stack([rng.integers(0, e, npts) for e in con.C.extents], axis=1)
+    t0 = time.perf_counter()
+    oracle.points(con, dtype, w.alpha, a, b, w.beta, c, pts, threads=cores)
+    dt = time.perf_counter() - t0
+    return {"value": 2.0 * npts * K / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{npts} random outputs of {con.C.numel} ({npts * K:.3g} multiply-adds, "
+                      f"{dt:.1f} s)"}
+
+
+def _to_dev(x, torch):
+    if x.dtype == np.uint16:
+        return torch.from_numpy(x.view(np.int16)).cuda()
+    return torch.from_numpy(x).cuda()
+
+
+def time_contraction(torch, g, con, dtype, alpha, beta, dev, steps, warmup, opts=None):
+    """Device-timed launches of one plan on resident inputs.  Returns seconds/launch."""
+    plan = g.Plan(con, dtype, **(opts or {}))
+    a, b, c = dev
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        plan(alpha, a, b, beta, c, stream)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        plan(alpha, a, b, beta, c, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    status = plan.device_status()
+    info = plan.info.as_dict()
+    plan.close()
+    if status != 0:
+        raise RuntimeError(f"device status {status}")
+    return e0.elapsed_time(e1) / 1e3 / steps, info
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_1607_00145_b200 as g
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = _peaks()
+    w = workload(args.workload)
+    dtype = DTYPE_BY_NAME[args.dtype]
+    con = w.contraction
+    M, N, K = con.mnk()
+    a, b, c = make_inputs(con, dtype, w.dist, w.seed, w.beta)
+    dev = (_to_dev(a, torch), _to_dev(b, torch), _to_dev(c, torch))
+    nbytes_in = a.nbytes + b.nbytes + (c.nbytes if w.beta != 0.0 else 0)
+    l2_note = "inputs_larger_than_l2" if nbytes_in + c.nbytes > 2 * 126e6 else "l2_flush_between_steps"
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") \
+        if l2_note == "l2_flush_between_steps" else None
+
+    opts = {}
+    if args.path:
+        opts["path"] = args.path
+    if args.split_k:
+        opts["split_k"] = args.split_k
+    plan = g.Plan(con, dtype, **opts)
+    info = plan.info.as_dict()
+    stream = torch.cuda.current_stream()
+    launches_per_step = 1 + (1 if info["split_k"] > 1 else 0)
+
+    def step():
+        plan(w.alpha, dev[0], dev[1], w.beta, dev[2], stream)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(args.steps)]
+    with ClockSampler(local) as clk:
+        t_wall0 = time.perf_counter()
+        for e0, e1 in evs:
+            if flush is not None:
+                flush.zero_()
+            e0.record(stream)
+            step()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        # keep the sampler alive long enough for at least a few samples
+        while time.perf_counter() - t_wall0 < 0.7:
+            step()
+            torch.cuda.synchronize()
+    if plan.device_status() != 0:
+        raise RuntimeError(f"kernel reported status {plan.device_status()}")
+    per = np.array([e0.elapsed_time(e1) for e0, e1 in evs]) / 1e3   # seconds per launch
+    total = float(per.sum())
+    if world > 1:
+        t = torch.tensor([total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total = float(t.item())
+        dist.barrier()
+    sec_per_step = total / args.steps
+    flops = con.flops()
+    value = world * flops / sec_per_step / 1e12
+    clocks = clk.summary()
+    sm_mhz = clocks["sm_mhz"] or 1965.0
+    fp32_peak = _fp32_peak_tflops(sm_mhz)
+
+    # ---- roofline of the contraction kernel ----
+    avg = float(per.mean())
+    t_roof, bound = roofline_time_s(con, dtype, w.beta, peaks, fp32_peak)
+    if bound == "hbm":
+        achieved = con.compulsory_bytes(dtype, w.beta) / avg / 1e9
+        peak, runit = peaks["hbm_gbs"], "GB/s"
+        peak_note = f"{peaks['source']} HBM copy bandwidth"
+    elif bound == "tensor":
+        achieved = flops / avg / 1e12
+        sustained = total > 1.0
+        peak = peaks["bf16_sustained"] if sustained else peaks["bf16_burst"]
+        runit = "TFLOP/s"
+        peak_note = f"{peaks['source']} cuBLAS bf16 {'sustained' if sustained else 'burst'}"
+    else:
+        achieved = flops / avg / 1e12
+        peak, runit = fp32_peak, "TFLOP/s"
+        peak_note = f"derived: 148 SM x 128 FMA lanes x 2 x {sm_mhz:.0f} MHz sampled"
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get(f"{w.key}:{DTYPE_NAMES[dtype]}:{info['path']}")
+    roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
+                "frac": achieved / peak, "traffic": traffic, "peak_note": peak_note,
+                "kernel_ms_avg": avg * 1e3, "kernel_ms_min": float(per.min()) * 1e3,
+                "roofline_time_ms": t_roof * 1e3}
+
+    out = None
+    if rank == 0:
+        # ---- end to end through the C ABI with host buffers ----
+        pin = [torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
+               for x in (a, b, c)]
+        c_host = torch.empty(c.size, dtype=torch.float32).pin_memory()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+
+        def e2e_step():
+            dev[0].copy_(pin[0], non_blocking=True)
+            dev[1].copy_(pin[1], non_blocking=True)
+            if w.beta != 0.0:
+                dev[2].copy_(pin[2], non_blocking=True)
+            plan(w.alpha, dev[0], dev[1], w.beta, dev[2], stream)
+            c_host.copy_(dev[2], non_blocking=True)
+
+        e2e_step()
+        torch.cuda.synchronize()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        s1.record(stream)
+        torch.cuda.synchronize()
+        e2e_s = s0.elapsed_time(s1) / 1e3 / e2e_steps
+        e2e = {"value": flops / e2e_s / 1e12, "unit": UNIT, "h2d_bytes_per_step": int(nbytes_in),
+               "d2h_bytes_per_step": int(c.nbytes), "steps": e2e_steps,
+               "note": "single-GPU figure; plan reused, pinned host buffers"}
+
+        # ---- equal-sized GEMM through the same kernels (Sec. 7) ----
+        extra = {}
+        if con.A.labels != [0, 2] or len(con.C.labels) != 2:
+            eg = equal_gemm(con)
+            ga, gb, gc = make_inputs(eg, dtype, w.dist, w.seed, w.beta)
+            gdev = (_to_dev(ga, torch), _to_dev(gb, torch), _to_dev(gc, torch))
+            t_eq, _ = time_contraction(torch, g, eg, dtype, w.alpha, w.beta, gdev,
+                                       max(3, args.steps // 2), args.warmup)
+            extra["equal_gemm"] = {"tflops": flops / t_eq / 1e12, "speedup_vs_equal_gemm": t_eq / avg}
+            del gdev
+
+        base = cpu_baseline(w, dtype, a, b, c, 8 * args.ref_macs)
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec_per_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": DTYPE_NAMES[dtype] + "-in/f32-acc"
+            if dtype != F32 else "f32", "data": "synthetic",
+            "config": {"workload": f"{w.key} {DTYPE_NAMES[dtype]} {M}x{N}x{K} alpha={w.alpha} "
+                                   f"beta={w.beta}", "l2": l2_note, "replicas": world,
+                       "path": info["path"], "tile": [info["tile_m"], info["tile_n"], info["tile_k"]],
+                       "stages": info["stages"], "split_k": info["split_k"],
+                       "loaders": [info["loader_a"], info["loader_b"]],
+                       "epilogue": info["epilogue"], "grid": info["grid"]},
+            "roofline": roofline, "cpu_baseline": base, "e2e": e2e,
+            "gpu_launches": args.steps * launches_per_step, "clocks": clocks, **extra,
+        }
+        if args.all:
+            out["workloads"] = run_all(torch, g, peaks, fp32_peak, args)
+    plan.close()
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_all(torch, g, peaks, fp32_peak, args):
+    """Every workload/dtype pair: TFLOP/s, roofline fraction, equal-GEMM ratio."""
+    rows = []
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for key in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "splitk"):
+        w = workload(key)
+        for dtype in w.dtypes:
+            con = w.contraction
+            a, b, c = make_inputs(con, dtype, w.dist, w.seed, w.beta)
+            dev = (_to_dev(a, torch), _to_dev(b, torch), _to_dev(c, torch))
+            variants = [("auto", {})]
+            if key in ("cfg3", "splitk"):
+                variants += [("split_k=1", {"split_k": 1}), ("split_k=2", {"split_k": 2}),
+                             ("split_k=4", {"split_k": 4})]
+            for name, opts in variants:
+                try:
+                    t, info = time_contraction(torch, g, con, dtype, w.alpha, w.beta, dev,
+                                               args.all_steps, 3, opts)
+                except Exception as e:  # an unsupported forced option is reported, not fatal
+                    rows.append({"workload": key, "dtype": DTYPE_NAMES[dtype], "variant": name,
+                                 "error": str(e)})
+                    continue
+                flush.zero_()
+                t_roof, bound = roofline_time_s(con, dtype, w.beta, peaks, fp32_peak)
+                row = {"workload": key, "dtype": DTYPE_NAMES[dtype], "variant": name,
+                       "ms": t * 1e3, "tflops": con.flops() / t / 1e12,
+                       "gbs": con.compulsory_bytes(dtype, w.beta) / t / 1e9, "bound": bound,
+                       "roofline_frac": t_roof / t, "path": info["path"],
+                       "tile": [info["tile_m"], info["tile_n"], info["tile_k"]],
+                       "split_k": info["split_k"]}
+                if name == "auto" and key != "cfg2":
+                    eg = equal_gemm(con)
+                    ga, gb, gc = make_inputs(eg, dtype, w.dist, w.seed, w.beta)
+                    gdev = (_to_dev(ga, torch), _to_dev(gb, torch), _to_dev(gc, torch))
+                    t_eq, _ = time_contraction(torch, g, eg, dtype, w.alpha, w.beta, gdev,
+                                               args.all_steps, 3)
+                    row["speedup_vs_equal_gemm"] = t_eq / t
+                    del gdev
+                rows.append(row)
+            del dev
+    return rows
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--dtype", default="bf16", choices=sorted(DTYPE_BY_NAME))
+    ap.add_argument("--path", type=int, default=0, help="force a gett_path_t")
+    ap.add_argument("--split-k", type=int, default=0)
+    ap.add_argument("--all", action="store_true", help="also time every workload")
+    ap.add_argument("--all-steps", type=int, default=10)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--ref-macs", type=float, default=5.0e8,
+                    help="multiply-adds in the oracle's bounded sample")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,206 @@
+/*
+ * gett.h -- C ABI of the B200 (sm_100a) GEMM-like tensor-tensor multiplication.
+ *
+ * The operation (Sec. 2.2, Eq. 2 / Eq. 3 of "Design of a High-Performance
+ * GEMM-like Tensor-Tensor Multiplication"):
+ *
+ *     C[Pi_C(I_m u I_n)] <- alpha * sum_{I_k} A[Pi_A(I_m u I_k)] * B[Pi_B(I_k u I_n)]
+ *                           + beta * C[Pi_C(I_m u I_n)]
+ *
+ * I_m = labels carried by A and C (free in A), I_n = labels carried by B and C
+ * (free in B), I_k = labels carried by A and B (contracted).  The contraction is
+ * computed GEMM-like (Sec. 3, Listing 4): the three index sets are fused into
+ * logical M, N, K dimensions, sub-tensors of A and B are packed into on-chip
+ * memory tile by tile, multiplied by a macro-kernel, and C is updated in place
+ * through its own mode permutation.  No transposed copy of A, B or C is ever
+ * written to global memory.
+ *
+ * Everything here is plain C: sizes, host/device pointers, no C++ or torch types.
+ * The library never prints, throws or aborts; every call returns a status.
+ */
+#ifndef GETT_H
+#define GETT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GETT_MAX_MODES 12 /* modes per tensor */
+
+#if defined(__GNUC__)
+#define GETT_API __attribute__((visibility("default")))
+#else
+#define GETT_API
+#endif
+
+typedef struct gett_plan gett_plan_t; /* opaque, library-owned */
+
+typedef enum {
+    GETT_OK = 0,
+    GETT_ERR_INVALID_ARG = 1,     /* NULL, mode count, extent < 1, stride < 1, overlapping C */
+    GETT_ERR_BAD_LABELS = 2,      /* label twice in a tensor, in all three, or in one only  */
+    GETT_ERR_EXTENT_MISMATCH = 3, /* the two carriers of a label disagree on its extent     */
+    GETT_ERR_UNSUPPORTED = 4,     /* dtype / size outside what the kernels cover            */
+    GETT_ERR_ALIGNMENT = 5,       /* operand base not aligned to its element size           */
+    GETT_ERR_ALLOC = 6,           /* workspace allocation failed                            */
+    GETT_ERR_CUDA = 7,            /* no device, launch failure                              */
+    GETT_ERR_TIMEOUT = 8          /* a bounded device-side wait gave up (see gett_plan_last_device_status) */
+} gett_status_t;
+
+typedef enum {
+    GETT_F32 = 0,      /* A, B, C fp32; strict fp32 FMA accumulation          */
+    GETT_BF16_F32 = 1, /* A, B bf16; fp32 accumulation; C fp32                */
+    GETT_F16_F32 = 2   /* A, B fp16; fp32 accumulation; C fp32                */
+} gett_dtype_t;
+
+/*
+ * One tensor: mode i has extent[i] >= 1, stride[i] >= 1 (in elements) and an
+ * integer label.  stride == NULL means packed with the FIRST mode stride-1
+ * (the paper's Fortran-order convention, Sec. 2.2).  The arrays are copied by
+ * gett_plan_create; the caller keeps ownership.
+ */
+typedef struct {
+    int32_t nmodes; /* 0 .. GETT_MAX_MODES */
+    const int64_t* extent;
+    const int64_t* stride;
+    const int32_t* label;
+} gett_tensor_desc_t;
+
+typedef enum {
+    GETT_PATH_AUTO = 0,
+    GETT_PATH_SIMT = 1, /* scalar gathers, any layout, any dtype (always available)        */
+    GETT_PATH_FFMA = 2, /* fp32: 16-byte cp.async gathers, register-blocked FFMA           */
+    GETT_PATH_UMMA = 3  /* bf16/fp16: 16-byte gathers into swizzled smem, tcgen05 + TMEM   */
+} gett_path_t;
+
+typedef enum {
+    GETT_LOAD_SCALAR = 0, /* element-wise gather                                           */
+    GETT_LOAD_VEC_FREE = 1, /* 16-byte vectors along the operand's free (M or N) dimension */
+    GETT_LOAD_VEC_K = 2     /* 16-byte vectors along the contracted dimension              */
+} gett_loader_t;
+
+typedef enum {
+    GETT_EPI_AUTO = 0,
+    GETT_EPI_DIRECT = 1, /* each thread stores its accumulators straight to C              */
+    GETT_EPI_STAGED = 2  /* accumulators pass through a shared-memory transpose so that
+                            stores run along C's stride-1 mode (Eq. 11 as a transposition) */
+} gett_epilogue_t;
+
+/* Planner overrides; zero-initialise for "auto".  Unsupported combinations make
+ * gett_plan_create return GETT_ERR_UNSUPPORTED rather than being silently changed. */
+typedef struct {
+    int32_t path;     /* gett_path_t                                     */
+    int32_t tile_m;   /* 0 = auto                                        */
+    int32_t tile_n;   /* 0 = auto                                        */
+    int32_t tile_k;   /* 0 = auto (K elements per pipeline stage)        */
+    int32_t stages;   /* 0 = auto                                        */
+    int32_t split_k;  /* 0 = auto, 1 = never, s > 1 = exactly s slices   */
+    int32_t epilogue; /* gett_epilogue_t                                 */
+    int32_t reserved[9];
+} gett_plan_opts_t;
+
+/* What the planner decided (Sec. 3.2.1: index sets, fused sizes, blocking). */
+typedef struct {
+    int64_t M, N, K;                  /* S_{I_m}, S_{I_n}, S_{I_k}                         */
+    int32_t n_m, n_n, n_k;            /* sizes of I_m, I_n, I_k after dropping extent-1    */
+    int32_t labels_m[GETT_MAX_MODES]; /* canonical order: ascending stride in C            */
+    int32_t labels_n[GETT_MAX_MODES]; /* canonical order: ascending stride in C            */
+    int32_t labels_k[GETT_MAX_MODES]; /* canonical order: ascending stride in A            */
+    int32_t merged_m, merged_n, merged_k; /* super-indices left after merging (Sec. 6)     */
+    int32_t path;                     /* gett_path_t actually chosen                       */
+    int32_t loader_a, loader_b;       /* gett_loader_t                                     */
+    int32_t epilogue;                 /* gett_epilogue_t                                   */
+    int32_t tile_m, tile_n, tile_k, stages, split_k;
+    int32_t grid, block, smem_bytes;
+    int32_t digits_m, digits_n, digits_k; /* digits of the tile-order fused indices        */
+    int64_t workspace_bytes;          /* split-K partial sums owned by the plan            */
+    int64_t tiles;                    /* output tiles (M tiles x N tiles)                  */
+    int32_t device;                   /* CUDA device the plan is bound to, -1 = none       */
+    int32_t reserved[7];
+} gett_plan_info_t;
+
+typedef enum {
+    GETT_TABLE_A_M = 0, /* offset in A of fused free-in-A index m   (length M) */
+    GETT_TABLE_A_K = 1, /* offset in A of fused contracted index k  (length K) */
+    GETT_TABLE_B_N = 2,
+    GETT_TABLE_B_K = 3,
+    GETT_TABLE_C_M = 4,
+    GETT_TABLE_C_N = 5
+} gett_table_t;
+
+/*
+ * gett_plan_create -- classify the labels into I_m, I_n, I_k (Sec. 2.2), drop
+ * extent-1 modes, merge adjacent modes into super-indices (Sec. 6, stage 1),
+ * choose the order in which each set is fused so that the stride-1 modes of A,
+ * B and C stay inside a tile (Sec. 3.2.1), and pick kernel, blocking and split-K.
+ *   out    : receives the plan (host pointer to host pointer).  Untouched on error.
+ *   A,B,C  : host descriptors; copied.  C's modes must not overlap in memory.
+ *   dtype  : gett_dtype_t.
+ *   opts   : host pointer or NULL for automatic choices.
+ * The plan is bound to the CUDA device current at the call; its split-K
+ * workspace (device memory, info.workspace_bytes) is allocated here.  Without
+ * any CUDA device the plan is still created (device = -1) and can be
+ * inspected, but gett_contract returns GETT_ERR_CUDA.
+ * Errors: INVALID_ARG, BAD_LABELS, EXTENT_MISMATCH, UNSUPPORTED (fused M, N or
+ * K >= 2^31, dtype, impossible opts), ALLOC.
+ */
+GETT_API gett_status_t gett_plan_create(gett_plan_t** out, const gett_tensor_desc_t* A,
+                               const gett_tensor_desc_t* B, const gett_tensor_desc_t* C,
+                               gett_dtype_t dtype, const gett_plan_opts_t* opts);
+
+/*
+ * gett_contract -- run C <- alpha * A*B + beta * C (Eq. 2) on `cuda_stream`
+ * (a cudaStream_t passed as void*; NULL = the default stream).
+ *   A, B, C : DEVICE pointers, caller-owned, covering 1 + sum (extent-1)*stride
+ *             elements each; A/B of the plan's input type, C fp32.  Bases must be
+ *             aligned to the element size; 16-byte aligned bases enable the
+ *             vectorised kernels, otherwise the scalar path is used.
+ *   alpha, beta : host scalars.  beta == 0 means C is not read (NaN/Inf in the
+ *             old C do not propagate).  alpha == 0 takes no shortcut.
+ * Asynchronous; allocates nothing; returns launch-time errors only.  C must not
+ * alias A or B.  A plan may be reused; calls that use the same plan concurrently
+ * on different streams race on its workspace when info.split_k > 1.
+ * Every element of C that its descriptor addresses is written exactly once per
+ * call; gaps left by padded strides are not touched.
+ */
+GETT_API gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A, const void* B,
+                            float beta, void* C, void* cuda_stream);
+
+/* gett_plan_destroy -- free the plan and its workspace.  NULL is a no-op. */
+GETT_API gett_status_t gett_plan_destroy(gett_plan_t* plan);
+
+/* gett_plan_get_info -- copy the planner's decisions into *info (host). */
+GETT_API gett_status_t gett_plan_get_info(const gett_plan_t* plan, gett_plan_info_t* info);
+
+/*
+ * gett_plan_get_table -- one of the six offset tables of Sec. 3.2 ("identify
+ * sub-tensor"): entry i is the storage offset (elements) contributed by fused
+ * index i, fused in the canonical order reported by gett_plan_get_info with the
+ * first mode fastest.  The element addressed by (m, n) of C is
+ * C_M[m] + C_N[n]; likewise A_M[m] + A_K[k] and B_N[n] + B_K[k].
+ * The entries are produced by the same index-decomposition routine and digit
+ * data that the kernels use on the device (evaluated here on the host, through
+ * the tile-order digits the kernels receive).
+ *   dst : host array of `capacity` int64; needs capacity >= table length,
+ *         else INVALID_ARG.
+ */
+GETT_API gett_status_t gett_plan_get_table(const gett_plan_t* plan, int which, int64_t* dst,
+                                  size_t capacity);
+
+/*
+ * gett_plan_last_device_status -- 0 if no kernel launched from this plan has
+ * reported a problem, else the gett_status_t a kernel recorded (GETT_ERR_TIMEOUT
+ * when a bounded wait on a barrier ran out).  Synchronises with the device.
+ */
+GETT_API gett_status_t gett_plan_last_device_status(const gett_plan_t* plan);
+
+/* Human-readable name of a status; never NULL. */
+GETT_API const char* gett_status_string(gett_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GETT_H */

@@ -1,0 +1,170 @@
+// C ABI of the library (declared in include/gett.h): plan life cycle, kernel
+// dispatch, introspection.  Device memory is touched only here (split-K
+// workspace and the status word); gett_contract itself allocates nothing.
+#include <cuda_runtime.h>
+
+#include <new>
+
+#include "kernels.h"
+
+namespace {
+
+int current_device_sm_count(int* device_out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        *device_out = -1;
+        return 0;
+    }
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        *device_out = -1;
+        return 0;
+    }
+    *device_out = dev;
+    return sms;
+}
+
+} // namespace
+
+extern "C" {
+
+gett_status_t gett_plan_create(gett_plan_t** out, const gett_tensor_desc_t* A,
+                               const gett_tensor_desc_t* B, const gett_tensor_desc_t* C,
+                               gett_dtype_t dtype, const gett_plan_opts_t* opts)
+{
+    if (!out || !A || !B || !C)
+        return GETT_ERR_INVALID_ARG;
+    gett_plan* p = new (std::nothrow) gett_plan();
+    if (!p)
+        return GETT_ERR_ALLOC;
+    p->ws = nullptr;
+    p->status = nullptr;
+    int device = -1;
+    const int sms = current_device_sm_count(&device);
+    gett_status_t rc = gett_planner_build(p, A, B, C, dtype, opts, sms > 0 ? sms : 148);
+    if (rc != GETT_OK) {
+        delete p;
+        return rc;
+    }
+    p->info.device = device;
+    p->sm_count = sms > 0 ? sms : 148;
+    if (device >= 0) {
+        if (cudaMalloc(&p->status, sizeof(int32_t)) != cudaSuccess ||
+            cudaMemset(p->status, 0, sizeof(int32_t)) != cudaSuccess) {
+            cudaGetLastError();
+            gett_plan_destroy(p);
+            return GETT_ERR_ALLOC;
+        }
+        if (p->info.workspace_bytes > 0 &&
+            cudaMalloc(&p->ws, (size_t)p->info.workspace_bytes) != cudaSuccess) {
+            cudaGetLastError();
+            gett_plan_destroy(p);
+            return GETT_ERR_ALLOC;
+        }
+    }
+    *out = p;
+    return GETT_OK;
+}
+
+gett_status_t gett_plan_destroy(gett_plan_t* plan)
+{
+    if (!plan)
+        return GETT_OK;
+    if (plan->ws)
+        cudaFree(plan->ws);
+    if (plan->status)
+        cudaFree(plan->status);
+    delete plan;
+    return GETT_OK;
+}
+
+gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A, const void* B,
+                            float beta, void* C, void* cuda_stream)
+{
+    if (!plan || !A || !B || !C)
+        return GETT_ERR_INVALID_ARG;
+    if (plan->info.device < 0)
+        return GETT_ERR_CUDA;
+    const uintptr_t es = plan->dtype == GETT_F32 ? 4 : 2;
+    if (((uintptr_t)A % es) || ((uintptr_t)B % es) || ((uintptr_t)C % 4))
+        return GETT_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    GettKernelArgs args;
+    args.M = plan->M;
+    args.N = plan->N;
+    args.K = plan->K;
+    args.A = A;
+    args.B = B;
+    args.C = static_cast<float*>(C);
+    args.ws = plan->ws;
+    args.status = plan->status;
+    args.alpha = alpha;
+    args.beta = beta;
+    args.tiles_m = plan->tiles_m;
+    args.tiles_n = plan->tiles_n;
+    args.split_k = (uint32_t)plan->info.split_k;
+    args.k_per_split = plan->k_per_split;
+    args.dtype = plan->dtype;
+    args.a_kmajor = plan->a_kmajor;
+    args.b_kmajor = plan->b_kmajor;
+
+    cudaError_t err = cudaSuccess;
+    switch (plan->info.path) {
+    case GETT_PATH_SIMT: err = gett_launch_simt(args, plan->info.grid, stream); break;
+    default: return GETT_ERR_UNSUPPORTED;
+    }
+    if (err == cudaSuccess && args.split_k > 1)
+        err = gett_launch_splitk_reduce(args, plan->sm_count, stream);
+    return err == cudaSuccess ? GETT_OK : GETT_ERR_CUDA;
+}
+
+gett_status_t gett_plan_get_info(const gett_plan_t* plan, gett_plan_info_t* info)
+{
+    if (!plan || !info)
+        return GETT_ERR_INVALID_ARG;
+    *info = plan->info;
+    return GETT_OK;
+}
+
+gett_status_t gett_plan_get_table(const gett_plan_t* plan, int which, int64_t* dst, size_t capacity)
+{
+    if (!plan)
+        return GETT_ERR_INVALID_ARG;
+    return gett_planner_table(plan, which, dst, capacity);
+}
+
+gett_status_t gett_plan_last_device_status(const gett_plan_t* plan)
+{
+    if (!plan)
+        return GETT_ERR_INVALID_ARG;
+    if (!plan->status)
+        return GETT_ERR_CUDA;
+    int32_t host = 0;
+    if (cudaMemcpy(&host, plan->status, sizeof host, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return GETT_ERR_CUDA;
+    }
+    return static_cast<gett_status_t>(host);
+}
+
+const char* gett_status_string(gett_status_t status)
+{
+    switch (status) {
+    case GETT_OK: return "ok";
+    case GETT_ERR_INVALID_ARG: return "invalid argument";
+    case GETT_ERR_BAD_LABELS: return "bad labels";
+    case GETT_ERR_EXTENT_MISMATCH: return "extent mismatch";
+    case GETT_ERR_UNSUPPORTED: return "unsupported";
+    case GETT_ERR_ALIGNMENT: return "misaligned operand";
+    case GETT_ERR_ALLOC: return "allocation failed";
+    case GETT_ERR_CUDA: return "cuda error";
+    case GETT_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+} // extern "C"

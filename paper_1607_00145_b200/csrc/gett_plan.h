@@ -1,0 +1,63 @@
+// Internal plan object: what the host planner decides and what every kernel
+// launch receives.  Nothing in this header is part of the public ABI.
+#pragma once
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/gett.h"
+#include "gett_dims.h"
+
+// One mode of the contraction after classification (Sec. 2.2).
+struct GettMode {
+    int32_t label;
+    int64_t ext;
+    int64_t sA, sB, sC; // element strides; 0 where the tensor does not carry the mode
+};
+
+// One digit of a tile-order fused index: indices (i / mult) % ext of mode `mode`
+// (an index into the canonical list of that set).  mult > 1 or ext < mode extent
+// means the mode was split by factors of its extent (Sec. 3.2.1, Examples 1-2).
+struct GettDigit {
+    int32_t mode;
+    int64_t ext;
+    int64_t mult;
+};
+
+// Arguments common to every contraction kernel (passed by value).
+struct GettKernelArgs {
+    GettDim M, N, K; // tile-order digits, merged where contiguous
+    const void* A;
+    const void* B;
+    float* C;
+    float* ws;      // split-K partial sums [split][N][M] (tile-order fused indices), or null
+    int32_t* status; // device status word, written only on failure
+    float alpha, beta;
+    uint32_t tiles_m, tiles_n;
+    uint32_t split_k;     // >= 1
+    uint32_t k_per_split; // K elements per slice, a multiple of tile_k
+    int32_t dtype;        // gett_dtype_t
+    int32_t a_kmajor;     // A's fastest-varying direction in memory is K (else M)
+    int32_t b_kmajor;
+};
+
+struct gett_plan {
+    int32_t dtype;
+    std::vector<GettMode> im, in, ik; // canonical order (what get_info reports)
+    std::vector<GettDigit> tm, tn, tk; // tile order, before merging
+    GettDim M, N, K;                   // tile order, merged: what the kernels get
+    gett_plan_info_t info;
+    // geometry
+    uint32_t tiles_m, tiles_n, k_per_split;
+    int32_t a_kmajor, b_kmajor;
+    // device side
+    float* ws;
+    int32_t* status;
+    int32_t sm_count;
+};
+
+// Host planner (planner.cpp): everything except device allocation.
+gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* A,
+                                 const gett_tensor_desc_t* B, const gett_tensor_desc_t* C,
+                                 gett_dtype_t dtype, const gett_plan_opts_t* opts, int sm_count);
+gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, size_t capacity);

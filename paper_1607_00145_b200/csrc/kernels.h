@@ -1,0 +1,12 @@
+// Launch entry points of the device kernels (internal).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "gett_plan.h"
+
+// Scalar-gather kernel, any layout / dtype.  grid = tiles * split_k.
+cudaError_t gett_launch_simt(const GettKernelArgs& args, int grid, cudaStream_t stream);
+
+// Sum the split-K slices in `ws` and apply C <- alpha * sum + beta * C (Eq. 11).
+cudaError_t gett_launch_splitk_reduce(const GettKernelArgs& args, int sm_count,
+                                      cudaStream_t stream);

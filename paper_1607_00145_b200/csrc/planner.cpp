@@ -1,0 +1,379 @@
+// Host planner: from three tensor descriptors to index sets, fused dimensions,
+// tile order, kernel path and blocking.  Pure host C++ (no CUDA calls), so it can
+// be exercised on a machine without a GPU.
+//
+// Steps and where the paper describes them:
+//   classify labels into I_m / I_n / I_k ............ Sec. 2.2
+//   merge adjacent modes into super-indices .......... Sec. 6 (stage 1)
+//   choose the sub-tensor that forms a tile, keeping
+//   the stride-1 mode of each tensor inside it ....... Sec. 3.2.1
+//   split a mode by factors of its extent ............ Sec. 3.2.1, Examples 1-2
+//   blocking sizes, GEMM variant (here: split-K) ..... Sec. 3.3
+#include <algorithm>
+#include <cstring>
+#include <map>
+
+#include "gett_plan.h"
+
+namespace {
+
+struct RawTensor {
+    int n;
+    int64_t ext[GETT_MAX_MODES], stride[GETT_MAX_MODES];
+    int32_t label[GETT_MAX_MODES];
+    int find(int32_t l) const
+    {
+        for (int i = 0; i < n; ++i)
+            if (label[i] == l)
+                return i;
+        return -1;
+    }
+};
+
+gett_status_t read_desc(const gett_tensor_desc_t* d, RawTensor& t)
+{
+    if (!d || d->nmodes < 0 || d->nmodes > GETT_MAX_MODES)
+        return GETT_ERR_INVALID_ARG;
+    if (d->nmodes > 0 && (!d->extent || !d->label))
+        return GETT_ERR_INVALID_ARG;
+    t.n = d->nmodes;
+    int64_t packed = 1;
+    for (int i = 0; i < t.n; ++i) {
+        t.ext[i] = d->extent[i];
+        t.label[i] = d->label[i];
+        if (t.ext[i] < 1 || t.ext[i] >= (1ll << 31))
+            return GETT_ERR_INVALID_ARG;
+        t.stride[i] = d->stride ? d->stride[i] : packed;
+        if (t.stride[i] < 1 || t.stride[i] >= (1ll << 46))
+            return GETT_ERR_INVALID_ARG;
+        packed *= t.ext[i];
+        if (packed >= (1ll << 46))
+            return GETT_ERR_UNSUPPORTED;
+        for (int j = 0; j < i; ++j)
+            if (t.label[j] == t.label[i])
+                return GETT_ERR_BAD_LABELS;
+    }
+    return GETT_OK;
+}
+
+// C must address every element once: sorted by stride, each mode must step over
+// the whole extent of the previous one.
+bool c_overlaps(const RawTensor& c)
+{
+    std::vector<std::pair<int64_t, int64_t>> v; // (stride, extent)
+    for (int i = 0; i < c.n; ++i)
+        if (c.ext[i] > 1)
+            v.push_back({c.stride[i], c.ext[i]});
+    std::sort(v.begin(), v.end());
+    for (size_t i = 1; i < v.size(); ++i)
+        if (v[i].first < v[i - 1].first * v[i - 1].second)
+            return true;
+    return false;
+}
+
+// Tile order of one set: `lead` (index into modes, or -1) first, the rest in
+// canonical order.  Each mode is one digit (no split).
+std::vector<GettDigit> order_with_lead(const std::vector<GettMode>& modes, int lead)
+{
+    std::vector<GettDigit> out;
+    if (lead >= 0)
+        out.push_back({lead, modes[lead].ext, 1});
+    for (int i = 0; i < (int)modes.size(); ++i)
+        if (i != lead)
+            out.push_back({i, modes[i].ext, 1});
+    return out;
+}
+
+// Build the kernel-side dimension: one entry per digit, merging a digit into its
+// predecessor when it continues it contiguously in both carrier tensors.
+gett_status_t make_dim(const std::vector<GettMode>& modes, const std::vector<GettDigit>& digits,
+                       int carrierX, int carrierY, GettDim& D)
+{
+    auto stride_of = [](const GettMode& m, int which) {
+        return which == 0 ? m.sA : which == 1 ? m.sB : m.sC;
+    };
+    memset(&D, 0, sizeof D);
+    struct E {
+        int64_t ext, sx, sy;
+    };
+    std::vector<E> e;
+    for (const GettDigit& g : digits) {
+        const GettMode& m = modes[g.mode];
+        E cur{g.ext, stride_of(m, carrierX) * g.mult, stride_of(m, carrierY) * g.mult};
+        if (cur.ext == 1)
+            continue;
+        if (!e.empty() && cur.sx == e.back().sx * e.back().ext && cur.sy == e.back().sy * e.back().ext &&
+            e.back().ext * cur.ext < (1ll << 31))
+            e.back().ext *= cur.ext;
+        else
+            e.push_back(cur);
+    }
+    if ((int)e.size() > GETT_MAX_DIGITS)
+        return GETT_ERR_UNSUPPORTED;
+    int64_t size = 1;
+    D.ndig = (int)e.size();
+    for (int d = 0; d < D.ndig; ++d) {
+        D.ext[d] = (uint32_t)e[d].ext;
+        gett_magic(D.ext[d], D.mul[d], D.sh[d]);
+        D.sX[d] = e[d].sx;
+        D.sY[d] = e[d].sy;
+        size *= e[d].ext;
+        if (size >= (1ll << 31))
+            return GETT_ERR_UNSUPPORTED;
+    }
+    D.size = (uint32_t)size;
+    return GETT_OK;
+}
+
+int merged_count(const std::vector<GettMode>& modes, int cx, int cy)
+{
+    std::vector<GettDigit> canon;
+    for (int i = 0; i < (int)modes.size(); ++i)
+        canon.push_back({i, modes[i].ext, 1});
+    GettDim D;
+    if (make_dim(modes, canon, cx, cy, D) != GETT_OK)
+        return (int)modes.size();
+    return D.ndig;
+}
+
+int find_unit(const std::vector<GettMode>& modes, int which)
+{
+    for (int i = 0; i < (int)modes.size(); ++i) {
+        int64_t s = which == 0 ? modes[i].sA : which == 1 ? modes[i].sB : modes[i].sC;
+        if (s == 1)
+            return i;
+    }
+    return -1;
+}
+
+int64_t min_stride(const std::vector<GettMode>& modes, int which)
+{
+    int64_t best = INT64_MAX;
+    for (const GettMode& m : modes) {
+        int64_t s = which == 0 ? m.sA : which == 1 ? m.sB : m.sC;
+        best = std::min(best, s);
+    }
+    return best;
+}
+
+uint32_t ceil_div(uint32_t a, uint32_t b) { return (a + b - 1) / b; }
+
+// 16-byte vectors of `vec` elements along the first digit of `lead` are legal for
+// carrier X when that digit is stride-1, its extent is a multiple of vec, and every
+// other stride of the tensor (remaining digits of `lead`, all digits of `other`)
+// is a multiple of vec, so that every vector starts on a 16-byte boundary.
+bool vec_ok(const GettDim& lead, bool leadIsX, const GettDim& other, bool otherIsX, uint32_t vec)
+{
+    if (lead.ndig < 1)
+        return false;
+    const int64_t* ls = leadIsX ? lead.sX : lead.sY;
+    const int64_t* os = otherIsX ? other.sX : other.sY;
+    if (ls[0] != 1 || lead.ext[0] % vec != 0)
+        return false;
+    for (int d = 1; d < lead.ndig; ++d)
+        if (ls[d] % vec != 0)
+            return false;
+    for (int d = 0; d < other.ndig; ++d)
+        if (os[d] % vec != 0)
+            return false;
+    return true;
+}
+
+} // namespace
+
+gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
+                                 const gett_tensor_desc_t* dB, const gett_tensor_desc_t* dC,
+                                 gett_dtype_t dtype, const gett_plan_opts_t* opts, int sm_count)
+{
+    RawTensor A, B, C;
+    gett_status_t rc;
+    if ((rc = read_desc(dA, A)) || (rc = read_desc(dB, B)) || (rc = read_desc(dC, C)))
+        return rc;
+    if (dtype != GETT_F32 && dtype != GETT_BF16_F32 && dtype != GETT_F16_F32)
+        return GETT_ERR_UNSUPPORTED;
+    gett_plan_opts_t o;
+    memset(&o, 0, sizeof o);
+    if (opts)
+        o = *opts;
+
+    // ---- classification (Sec. 2.2) ----
+    std::vector<GettMode> im, in, ik;
+    for (int i = 0; i < C.n; ++i) {
+        int ia = A.find(C.label[i]), ib = B.find(C.label[i]);
+        if ((ia >= 0) == (ib >= 0))
+            return GETT_ERR_BAD_LABELS; // in all three tensors, or only in C
+        int64_t e = ia >= 0 ? A.ext[ia] : B.ext[ib];
+        if (e != C.ext[i])
+            return GETT_ERR_EXTENT_MISMATCH;
+        GettMode m{C.label[i], e, ia >= 0 ? A.stride[ia] : 0, ib >= 0 ? B.stride[ib] : 0,
+                   C.stride[i]};
+        if (e > 1)
+            (ia >= 0 ? im : in).push_back(m);
+    }
+    for (int i = 0; i < A.n; ++i) {
+        if (C.find(A.label[i]) >= 0)
+            continue;
+        int ib = B.find(A.label[i]);
+        if (ib < 0)
+            return GETT_ERR_BAD_LABELS; // only in A
+        if (A.ext[i] != B.ext[ib])
+            return GETT_ERR_EXTENT_MISMATCH;
+        if (A.ext[i] > 1)
+            ik.push_back({A.label[i], A.ext[i], A.stride[i], B.stride[ib], 0});
+    }
+    for (int i = 0; i < B.n; ++i)
+        if (C.find(B.label[i]) < 0 && A.find(B.label[i]) < 0)
+            return GETT_ERR_BAD_LABELS; // only in B
+    if (c_overlaps(C))
+        return GETT_ERR_INVALID_ARG;
+
+    // ---- canonical order: I_m, I_n by stride in C; I_k by stride in A ----
+    auto byC = [](const GettMode& a, const GettMode& b) { return a.sC < b.sC; };
+    auto byA = [](const GettMode& a, const GettMode& b) { return a.sA < b.sA; };
+    std::stable_sort(im.begin(), im.end(), byC);
+    std::stable_sort(in.begin(), in.end(), byC);
+    std::stable_sort(ik.begin(), ik.end(), byA);
+    p->dtype = dtype;
+    p->im = im;
+    p->in = in;
+    p->ik = ik;
+
+    // ---- tile order: keep each operand's stride-1 mode first in its set (Sec. 3.2.1) ----
+    int leadM = find_unit(im, 0); // A's stride-1 mode, if it is free
+    int leadN = find_unit(in, 1); // B's stride-1 mode, if it is free
+    int leadK = find_unit(ik, 0); // A's stride-1 mode, if it is contracted ...
+    if (leadK < 0)
+        leadK = find_unit(ik, 1); // ... else B's
+    p->tm = order_with_lead(im, leadM);
+    p->tn = order_with_lead(in, leadN);
+    p->tk = order_with_lead(ik, leadK);
+    if ((rc = make_dim(im, p->tm, 0, 2, p->M)) || (rc = make_dim(in, p->tn, 1, 2, p->N)) ||
+        (rc = make_dim(ik, p->tk, 0, 1, p->K)))
+        return rc;
+    p->a_kmajor = (!ik.empty() && (im.empty() || min_stride(ik, 0) < min_stride(im, 0))) ? 1 : 0;
+    p->b_kmajor = (!ik.empty() && (in.empty() || min_stride(ik, 1) < min_stride(in, 1))) ? 1 : 0;
+
+    gett_plan_info_t& info = p->info;
+    memset(&info, 0, sizeof info);
+    info.M = p->M.size;
+    info.N = p->N.size;
+    info.K = p->K.size;
+    info.n_m = (int)im.size();
+    info.n_n = (int)in.size();
+    info.n_k = (int)ik.size();
+    for (int i = 0; i < info.n_m; ++i)
+        info.labels_m[i] = im[i].label;
+    for (int i = 0; i < info.n_n; ++i)
+        info.labels_n[i] = in[i].label;
+    for (int i = 0; i < info.n_k; ++i)
+        info.labels_k[i] = ik[i].label;
+    info.merged_m = merged_count(im, 0, 2);
+    info.merged_n = merged_count(in, 1, 2);
+    info.merged_k = merged_count(ik, 0, 1);
+    info.digits_m = p->M.ndig;
+    info.digits_n = p->N.ndig;
+    info.digits_k = p->K.ndig;
+    info.device = -1;
+
+    // ---- which operands can be gathered in 16-byte vectors ----
+    const uint32_t vec = dtype == GETT_F32 ? 4 : 8;
+    info.loader_a = vec_ok(p->M, true, p->K, true, vec)    ? GETT_LOAD_VEC_FREE
+                    : vec_ok(p->K, true, p->M, true, vec)  ? GETT_LOAD_VEC_K
+                                                           : GETT_LOAD_SCALAR;
+    info.loader_b = vec_ok(p->N, true, p->K, false, vec)   ? GETT_LOAD_VEC_FREE
+                    : vec_ok(p->K, false, p->N, true, vec) ? GETT_LOAD_VEC_K
+                                                           : GETT_LOAD_SCALAR;
+
+    // ---- path ----
+    int path = o.path;
+    if (path < GETT_PATH_AUTO || path > GETT_PATH_UMMA)
+        return GETT_ERR_INVALID_ARG;
+    if (path == GETT_PATH_AUTO)
+        path = GETT_PATH_SIMT;
+    if (path != GETT_PATH_SIMT)
+        return GETT_ERR_UNSUPPORTED;
+    info.path = path;
+
+    // ---- blocking (Sec. 3.3) ----
+    if (o.tile_m < 0 || o.tile_n < 0 || o.tile_k < 0 || o.stages < 0 || o.split_k < 0)
+        return GETT_ERR_INVALID_ARG;
+    if (path == GETT_PATH_SIMT) {
+        if ((o.tile_m && o.tile_m != 64) || (o.tile_n && o.tile_n != 64) ||
+            (o.tile_k && o.tile_k != 16) || (o.stages && o.stages != 1) ||
+            (o.epilogue && o.epilogue != GETT_EPI_DIRECT))
+            return GETT_ERR_UNSUPPORTED;
+        info.tile_m = 64;
+        info.tile_n = 64;
+        info.tile_k = 16;
+        info.stages = 1;
+        info.block = 256;
+        info.smem_bytes = 0;
+        info.epilogue = GETT_EPI_DIRECT;
+        info.loader_a = info.loader_b = GETT_LOAD_SCALAR;
+    }
+    p->tiles_m = ceil_div(p->M.size, (uint32_t)info.tile_m);
+    p->tiles_n = ceil_div(p->N.size, (uint32_t)info.tile_n);
+    uint64_t tiles = (uint64_t)p->tiles_m * p->tiles_n;
+    if (tiles >= (1ull << 31))
+        return GETT_ERR_UNSUPPORTED;
+    info.tiles = (int64_t)tiles;
+
+    // ---- split-K: slice I_k when the output alone cannot fill the machine ----
+    uint32_t kslabs = ceil_div(p->K.size, (uint32_t)info.tile_k);
+    uint32_t split = 1;
+    if (o.split_k > 1) {
+        split = std::min<uint32_t>((uint32_t)o.split_k, kslabs);
+    } else if (o.split_k == 0 && sm_count > 0 && tiles * 2 <= (uint64_t)sm_count && kslabs >= 8) {
+        uint32_t want = (uint32_t)((2 * (uint64_t)sm_count + tiles - 1) / tiles);
+        split = std::max<uint32_t>(1, std::min<uint32_t>(want, kslabs / 4));
+    }
+    uint32_t slabs_per = ceil_div(kslabs, split);
+    split = ceil_div(kslabs, slabs_per); // no empty slice
+    if (tiles * split >= (1ull << 31))
+        return GETT_ERR_UNSUPPORTED;
+    info.split_k = (int32_t)split;
+    p->k_per_split = slabs_per * (uint32_t)info.tile_k;
+    info.workspace_bytes = split > 1 ? (int64_t)split * p->M.size * p->N.size * 4 : 0;
+    info.grid = (int32_t)(tiles * split);
+    return GETT_OK;
+}
+
+// Canonical table `which`: fused canonical index -> per-mode indices -> tile-order
+// fused index -> gett_decompose() on the digits the kernels receive.
+gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, size_t capacity)
+{
+    const std::vector<GettMode>* modes;
+    const std::vector<GettDigit>* digits;
+    const GettDim* D;
+    bool wantX;
+    switch (which) {
+    case GETT_TABLE_A_M: modes = &p->im; digits = &p->tm; D = &p->M; wantX = true; break;
+    case GETT_TABLE_C_M: modes = &p->im; digits = &p->tm; D = &p->M; wantX = false; break;
+    case GETT_TABLE_B_N: modes = &p->in; digits = &p->tn; D = &p->N; wantX = true; break;
+    case GETT_TABLE_C_N: modes = &p->in; digits = &p->tn; D = &p->N; wantX = false; break;
+    case GETT_TABLE_A_K: modes = &p->ik; digits = &p->tk; D = &p->K; wantX = true; break;
+    case GETT_TABLE_B_K: modes = &p->ik; digits = &p->tk; D = &p->K; wantX = false; break;
+    default: return GETT_ERR_INVALID_ARG;
+    }
+    if (!dst || capacity < D->size)
+        return GETT_ERR_INVALID_ARG;
+    const int nm = (int)modes->size();
+    std::vector<int64_t> idx(nm, 0);
+    for (uint32_t c = 0; c < D->size; ++c) {
+        // tile-order fused index of the tuple idx[]
+        uint64_t t = 0, weight = 1;
+        for (const GettDigit& g : *digits) {
+            t += (uint64_t)((idx[g.mode] / g.mult) % g.ext) * weight;
+            weight *= (uint64_t)g.ext;
+        }
+        int64_t ox, oy;
+        gett_decompose(*D, (uint32_t)t, ox, oy);
+        dst[c] = wantX ? ox : oy;
+        for (int j = 0; j < nm; ++j) { // advance the canonical odometer, first mode fastest
+            if (++idx[j] < (*modes)[j].ext)
+                break;
+            idx[j] = 0;
+        }
+    }
+    return GETT_OK;
+}

@@ -1,0 +1,33 @@
+"""The C-ABI library loads without a GPU and exports every symbol gett.h declares."""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in os.listdir(inc):
+        if f.endswith(".h"):
+            txt = open(os.path.join(inc, f)).read()
+            names |= set(re.findall(r"GETT_API\s+[\w\s\*]+?\b(gett_\w+)\s*\(", txt))
+    return names
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_1607_00145_b200 import library_path
+    lib = ctypes.CDLL(library_path())
+    names = _declared()
+    assert {"gett_plan_create", "gett_contract", "gett_plan_destroy", "gett_plan_get_info",
+            "gett_plan_get_table", "gett_status_string"} <= names
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_status_strings():
+    import paper_1607_00145_b200 as g
+    assert g.gett_status_string(0) == "ok"
+    assert len({g.gett_status_string(i) for i in range(9)}) == 9
+    assert g.gett_status_string(99) == "unknown status"

@@ -1,0 +1,108 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle,
+element by element on the same seeded inputs."""
+import numpy as np
+import pytest
+
+import paper_1607_00145_b200 as g
+from gpu_util import TOL, parity_case
+from helpers import random_contraction
+from workloads import BF16_F32, F16_F32, F32, parse_spec, workload
+
+pytestmark = pytest.mark.gpu
+
+DTYPES = [F32, BF16_F32, F16_F32]
+
+
+def test_cfg1_reference_case():
+    w = workload("cfg1")
+    ratio, info = parity_case(w.contraction, F32, w.dist, w.seed, w.alpha, w.beta, repeat=2)
+    assert (info.M, info.N, info.K) == (768, 40, 48)
+
+
+# Reduced copies of the other workloads: several tiles in M and N plus a ragged
+# tail, several K slabs, sized so the oracle finishes in seconds.
+SMALL = {
+    "cfg2": dict(m=200, n=136, k=88),
+    "cfg3": dict(m0=40, m1=33, n0=24, k=24),
+    "cfg4": dict(m0=24, m1=9, n0=7, n1=24, k0=8, k1=11),
+    "cfg5": dict(m0=3, m1=8, m2=6, n0=8, n1=3, n2=8, k=40),
+}
+
+
+@pytest.mark.parametrize("key", sorted(SMALL))
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("path", [g.GETT_PATH_AUTO, g.GETT_PATH_SIMT])
+def test_reduced_workloads(key, dtype, path):
+    w = workload(key, SMALL[key])
+    parity_case(w.contraction, dtype, w.dist, w.seed, w.alpha, w.beta, repeat=2, path=path)
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_fuzz_random_contractions(seed):
+    rng = np.random.default_rng(5000 + seed)
+    con = random_contraction(rng, max_rank=6, max_extent=9, min_each=0 if seed % 6 == 0 else 1)
+    dtype = DTYPES[seed % 3]
+    alpha, beta = [(1.0, 0.0), (1.0, 1.0), (-0.5, 2.0), (2.0, -0.5), (0.0, 1.0), (0.0, 0.0)][seed % 6]
+    parity_case(con, dtype, "uniform", seed, alpha, beta)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_fuzz_vector_friendly_extents(seed):
+    """Extents that are multiples of 8 (and 4), so the vectorised loaders engage."""
+    rng = np.random.default_rng(7000 + seed)
+    con = random_contraction(rng, max_rank=5, pad=False, extent_choices=[8, 16, 24, 40])
+    dtype = DTYPES[seed % 3]
+    alpha, beta = [(1.0, 0.0), (1.5, -1.0)][seed % 2]
+    parity_case(con, dtype, "normal", seed, alpha, beta)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("split", [2, 3, 7])
+def test_forced_split_k(dtype, split):
+    con = workload("splitk", dict(a=72, b=40, c=24, d=40)).contraction
+    ratio, info = parity_case(con, dtype, "uniform", 5, 1.0, 0.5, repeat=2, split_k=split)
+    assert info.split_k > 1 and info.workspace_bytes > 0
+
+
+def test_auto_split_k_engages_on_small_outputs():
+    con = workload("splitk", dict(a=64, b=48, c=64, d=64)).contraction
+    ratio, info = parity_case(con, F32, "uniform", 5, 1.0, 0.0)
+    assert info.split_k > 1
+
+
+def test_degenerate_index_sets():
+    for spec, sizes in [("C[m,n] = A[m] * B[n]", dict(m=70, n=9)),
+                        ("C[m] = A[m,k] * B[k]", dict(m=130, k=77)),
+                        ("C[n] = A[k] * B[k,n]", dict(n=65, k=33)),
+                        ("C[] = A[k] * B[k]", dict(k=1000))]:
+        for dtype in DTYPES:
+            parity_case(parse_spec(spec, sizes), dtype, "uniform", 3, 2.0, 1.0)
+
+
+def test_padded_strides_and_gaps():
+    con = parse_spec("C[m,n,p] = A[k,m,p] * B[n,k]", dict(m=37, n=10, p=5, k=19),
+                     strides={"A": [2, 41, 1600], "B": [1, 13], "C": [1, 40, 420]})
+    for dtype in DTYPES:
+        parity_case(con, dtype, "uniform", 8, 1.0, 1.0)
+        parity_case(con, dtype, "uniform", 8, 1.0, 0.0)
+
+
+def test_unaligned_bases_fall_back_to_scalar_loads():
+    import torch
+    from oracle import contract, c_offsets, tolerance_ratio
+    from workloads import make_inputs
+    con = workload("cfg4", SMALL["cfg4"]).contraction
+    for dtype in DTYPES:
+        a, b, c = make_inputs(con, dtype, "normal", 3, 0.0)
+        conv = (lambda x: torch.from_numpy(x.view(np.int16))) if dtype != F32 else torch.from_numpy
+        ta = torch.empty(a.size + 1, dtype=conv(a).dtype, device="cuda")
+        tb = torch.empty(b.size + 1, dtype=conv(b).dtype, device="cuda")
+        ta[1:].copy_(conv(a))
+        tb[1:].copy_(conv(b))
+        tc = torch.zeros(c.size + 1, dtype=torch.float32, device="cuda")
+        p = g.Plan(con, dtype)
+        p(1.0, ta[1:], tb[1:], 0.0, tc[1:])
+        torch.cuda.synchronize()
+        ref, absacc = contract(con, dtype, 1.0, a, b, 0.0, None, threads=4)
+        got = tc[1:].cpu().numpy()
+        assert tolerance_ratio(got, ref, absacc, 1.0, 0.0, None, c_offsets(con)) <= TOL

@@ -1,0 +1,145 @@
+"""Host planner through the C ABI (no GPU needed): classification, canonical
+order, merging, the offset tables bit-exact against the oracle's div/mod
+tables, and the error codes of the boundary."""
+import numpy as np
+import pytest
+
+import paper_1607_00145_b200 as g
+from helpers import random_contraction
+from oracle import tables as T
+from workloads import Contraction, TensorSpec, parse_spec, workload
+
+
+def _tables_match(con, dtype=g.GETT_F32, **opts):
+    p = g.Plan(con, dtype, **opts)
+    want = T.canonical_tables(con)
+    for name in g.TABLE_NAMES:
+        got = p.table(name)
+        assert got.dtype == np.int64
+        assert np.array_equal(got, want[name]), name
+    return p
+
+
+@pytest.mark.parametrize("key", ["cfg1", "cfg2", "cfg4", "cfg5"])
+@pytest.mark.parametrize("dtype", [g.GETT_F32, g.GETT_BF16_F32])
+def test_workload_tables_bit_exact(key, dtype):
+    con = workload(key).contraction
+    p = _tables_match(con, dtype)
+    assert (p.info.M, p.info.N, p.info.K) == con.mnk()
+    im, in_, ik = T.classify(con)
+    d = p.info.as_dict()
+    assert (d["labels_m"], d["labels_n"], d["labels_k"]) == (im, in_, ik)
+    mm, mn, mk = T.merged_extents(con)
+    assert (p.info.merged_m, p.info.merged_n, p.info.merged_k) == (len(mm), len(mn), len(mk))
+
+
+def test_cfg3_merges_to_one_m_digit_and_tables_match_on_a_scaled_copy():
+    p = g.Plan(workload("cfg3").contraction, g.GETT_F32)
+    assert (p.info.M, p.info.N, p.info.K) == (1048576, 24, 24)
+    assert p.info.merged_m == 1 and p.info.digits_m == 1
+    _tables_match(workload("cfg3", dict(m0=64, m1=48)).contraction)
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_fuzz_tables_bit_exact(seed):
+    rng = np.random.default_rng(1000 + seed)
+    con = random_contraction(rng, max_rank=6, max_extent=9, min_each=0 if seed % 5 == 0 else 1)
+    _tables_match(con, [g.GETT_F32, g.GETT_BF16_F32, g.GETT_F16_F32][seed % 3])
+
+
+def test_listing8_example_merges_like_the_paper():
+    con = parse_spec("C[a,b,c,i,j,k] = A[i,j,m,c] * B[m,k,a,b]",
+                     dict(a=24, b=24, c=24, i=24, j=24, k=24, m=24))
+    p = _tables_match(con)
+    assert (p.info.merged_m, p.info.merged_n, p.info.merged_k) == (2, 2, 1)
+    assert (p.info.M, p.info.N, p.info.K) == (24 * 576, 576 * 24, 24)
+
+
+def test_extent_one_and_empty_sets():
+    con = parse_spec("C[m,u,n] = A[k,m,u] * B[n,k,v]", dict(m=3, u=1, n=2, k=4, v=1))
+    # v is carried by B only but has extent 1: still a label error (it is in one tensor only)
+    with pytest.raises(g.GettError) as e:
+        g.Plan(con, g.GETT_F32)
+    assert e.value.status == 2
+    con = parse_spec("C[m,u,n] = A[k,m,u] * B[n,k]", dict(m=3, u=1, n=2, k=4))
+    p = _tables_match(con)
+    assert p.info.n_m == 1
+    for spec, sizes, mnk in [("C[m,n] = A[m] * B[n]", dict(m=3, n=4), (3, 4, 1)),
+                             ("C[m] = A[m,k] * B[k]", dict(m=3, k=5), (3, 1, 5)),
+                             ("C[] = A[k] * B[k]", dict(k=7), (1, 1, 7))]:
+        p = _tables_match(parse_spec(spec, sizes))
+        assert (p.info.M, p.info.N, p.info.K) == mnk
+
+
+@pytest.mark.parametrize("spec,sizes,status", [
+    ("C[m,n,b] = A[m,k,b] * B[k,n,b]", dict(m=2, n=2, k=2, b=2), 2),
+    ("C[m,n] = A[m,k,x] * B[k,n]", dict(m=2, n=2, k=2, x=2), 2),
+    ("C[m,n,y] = A[m,k] * B[k,n]", dict(m=2, n=2, k=2, y=2), 2),
+])
+def test_bad_labels(spec, sizes, status):
+    with pytest.raises(g.GettError) as e:
+        g.Plan(parse_spec(spec, sizes), g.GETT_F32)
+    assert e.value.status == status
+
+
+def test_other_error_codes():
+    ok = parse_spec("C[m,n] = A[m,k] * B[k,n]", dict(m=2, n=2, k=2))
+    # repeated label
+    bad = Contraction("x", TensorSpec([0, 0], [2, 2], [1, 2]), ok.B, ok.C)
+    with pytest.raises(g.GettError) as e:
+        g.Plan(bad, g.GETT_F32)
+    assert e.value.status == 2
+    # extent mismatch
+    bad = Contraction("x", TensorSpec([0, 2], [2, 3], [1, 2]), ok.B, ok.C)
+    with pytest.raises(g.GettError) as e:
+        g.Plan(bad, g.GETT_F32)
+    assert e.value.status == 3
+    # zero stride, zero extent
+    for t in (TensorSpec([0, 2], [2, 2], [0, 2]), TensorSpec([0, 2], [0, 2], [1, 2])):
+        with pytest.raises(g.GettError) as e:
+            g.Plan(Contraction("x", t, ok.B, ok.C), g.GETT_F32)
+        assert e.value.status == 1
+    # self-overlapping C
+    bad = Contraction("x", ok.A, ok.B, TensorSpec([0, 1], [2, 2], [1, 1]))
+    with pytest.raises(g.GettError) as e:
+        g.Plan(bad, g.GETT_F32)
+    assert e.value.status == 1
+    # unknown dtype, too many modes
+    with pytest.raises(g.GettError) as e:
+        g.Plan(ok, 7)
+    assert e.value.status == 4
+    many = TensorSpec(list(range(13)), [1] * 13, [1] * 13)
+    with pytest.raises(g.GettError) as e:
+        g.Plan(Contraction("x", many, ok.B, ok.C), g.GETT_F32)
+    assert e.value.status == 1
+
+
+def test_null_strides_mean_packed_first_mode_fastest():
+    con = workload("cfg5", dict(m0=2, m1=3, m2=4, n0=5, n1=2, n2=3, k=6)).contraction
+    packed = Contraction("p", *[TensorSpec(t.labels, t.extents, None) for t in (con.A, con.B, con.C)])
+    p = g.Plan(packed, g.GETT_F32)
+    want = T.canonical_tables(con)
+    for name in g.TABLE_NAMES:
+        assert np.array_equal(p.table(name), want[name])
+
+
+def test_contract_without_device_reports_cuda_error_not_a_crash():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("has a device")
+    p = g.Plan(workload("cfg1").contraction, g.GETT_F32)
+    assert p.info.device == -1
+    with pytest.raises(g.GettError) as e:
+        g.gett_contract(p.handle, 1.0, 16, 16, 0.0, 16, stream=0)
+    assert e.value.status == 7
+
+
+def test_split_k_planning():
+    con = workload("splitk").contraction
+    auto = g.Plan(con, g.GETT_F32)
+    assert auto.info.split_k > 1 and auto.info.workspace_bytes == auto.info.split_k * 384 * 376 * 4
+    never = g.Plan(con, g.GETT_F32, split_k=1)
+    assert never.info.split_k == 1 and never.info.workspace_bytes == 0
+    forced = g.Plan(workload("cfg3").contraction, g.GETT_F32, split_k=2)
+    assert forced.info.split_k == 2
+    assert g.Plan(workload("cfg3").contraction, g.GETT_F32).info.split_k == 1
