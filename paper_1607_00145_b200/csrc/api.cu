@@ -111,10 +111,32 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     args.dtype = plan->dtype;
     args.a_kmajor = plan->a_kmajor;
     args.b_kmajor = plan->b_kmajor;
+    args.loader_a = plan->info.loader_a;
+    args.loader_b = plan->info.loader_b;
+    args.tile_n = plan->info.tile_n;
+    args.stages = plan->info.stages;
+    args.epilogue = plan->info.epilogue;
+    args.debug = plan->debug;
+
+    int path = plan->info.path;
+    // the vectorised kernels need 16-byte aligned operand bases; otherwise gather scalars
+    if (path != GETT_PATH_SIMT && (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 15))
+        path = GETT_PATH_SIMT;
 
     cudaError_t err = cudaSuccess;
-    switch (plan->info.path) {
-    case GETT_PATH_SIMT: err = gett_launch_simt(args, plan->info.grid, stream); break;
+    switch (path) {
+    case GETT_PATH_SIMT: {
+        args.tiles_m = (plan->M.size + 63) / 64;
+        args.tiles_n = (plan->N.size + 63) / 64;
+        const uint64_t grid = (uint64_t)args.tiles_m * args.tiles_n * args.split_k;
+        if (grid >= (1ull << 31))
+            return GETT_ERR_UNSUPPORTED;
+        err = gett_launch_simt(args, (int)grid, stream);
+        break;
+    }
+    case GETT_PATH_UMMA:
+        err = gett_launch_umma(args, plan->info.grid, plan->info.smem_bytes, stream);
+        break;
     default: return GETT_ERR_UNSUPPORTED;
     }
     if (err == cudaSuccess && args.split_k > 1)

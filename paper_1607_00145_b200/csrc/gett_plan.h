@@ -39,6 +39,11 @@ struct GettKernelArgs {
     int32_t dtype;        // gett_dtype_t
     int32_t a_kmajor;     // A's fastest-varying direction in memory is K (else M)
     int32_t b_kmajor;
+    int32_t loader_a, loader_b; // gett_loader_t of the vectorised kernels
+    int32_t tile_n;       // tile width of the tensor-core / FFMA kernels
+    int32_t stages;       // depth of the shared-memory ring
+    int32_t epilogue;     // gett_epilogue_t
+    int32_t debug;        // opts.reserved[0]: experiment switches, 0 in normal use
 };
 
 struct gett_plan {
@@ -54,6 +59,7 @@ struct gett_plan {
     float* ws;
     int32_t* status;
     int32_t sm_count;
+    int32_t debug;
 };
 
 // Host planner (planner.cpp): everything except device allocation.
@@ -61,3 +67,8 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* A,
                                  const gett_tensor_desc_t* B, const gett_tensor_desc_t* C,
                                  gett_dtype_t dtype, const gett_plan_opts_t* opts, int sm_count);
 gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, size_t capacity);
+
+// Geometry of the tensor-core kernel (kernel_umma.cu), needed by the planner.
+int gett_umma_smem_bytes(int tile_n, int stages);
+int gett_umma_max_stages(int tile_n, int smem_limit);
+int gett_umma_block();

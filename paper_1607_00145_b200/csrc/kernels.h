@@ -10,3 +10,6 @@ cudaError_t gett_launch_simt(const GettKernelArgs& args, int grid, cudaStream_t 
 // Sum the split-K slices in `ws` and apply C <- alpha * sum + beta * C (Eq. 11).
 cudaError_t gett_launch_splitk_reduce(const GettKernelArgs& args, int sm_count,
                                       cudaStream_t stream);
+
+// Tensor-core kernel (16-bit inputs, tcgen05 + tensor memory), persistent grid.
+cudaError_t gett_launch_umma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream);

@@ -288,15 +288,21 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     int path = o.path;
     if (path < GETT_PATH_AUTO || path > GETT_PATH_UMMA)
         return GETT_ERR_INVALID_ARG;
+    const bool both_vec = info.loader_a != GETT_LOAD_SCALAR && info.loader_b != GETT_LOAD_SCALAR;
+    const bool umma_ok = dtype != GETT_F32 && both_vec;
     if (path == GETT_PATH_AUTO)
-        path = GETT_PATH_SIMT;
-    if (path != GETT_PATH_SIMT)
+        path = umma_ok ? GETT_PATH_UMMA : GETT_PATH_SIMT;
+    if (path == GETT_PATH_UMMA && !umma_ok)
+        return GETT_ERR_UNSUPPORTED;
+    if (path == GETT_PATH_FFMA)
         return GETT_ERR_UNSUPPORTED;
     info.path = path;
+    p->debug = o.reserved[0];
 
     // ---- blocking (Sec. 3.3) ----
     if (o.tile_m < 0 || o.tile_n < 0 || o.tile_k < 0 || o.stages < 0 || o.split_k < 0)
         return GETT_ERR_INVALID_ARG;
+    const int sms = sm_count > 0 ? sm_count : 148;
     if (path == GETT_PATH_SIMT) {
         if ((o.tile_m && o.tile_m != 64) || (o.tile_n && o.tile_n != 64) ||
             (o.tile_k && o.tile_k != 16) || (o.stages && o.stages != 1) ||
@@ -310,6 +316,39 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.smem_bytes = 0;
         info.epilogue = GETT_EPI_DIRECT;
         info.loader_a = info.loader_b = GETT_LOAD_SCALAR;
+    } else { // GETT_PATH_UMMA
+        if ((o.tile_m && o.tile_m != 128) || (o.tile_k && o.tile_k != 64) ||
+            (o.epilogue && o.epilogue != GETT_EPI_DIRECT))
+            return GETT_ERR_UNSUPPORTED;
+        int tn = o.tile_n;
+        if (tn == 0) {
+            // fewest (waves x tile width); ties go to the wider tile
+            const uint32_t tm_count = ceil_div(p->M.size, 128);
+            uint64_t best = UINT64_MAX;
+            for (int cand : {256, 192, 128, 64}) {
+                if (cand > 64 && (uint32_t)cand >= p->N.size + 64)
+                    continue; // a narrower tile already covers N
+                uint64_t t = (uint64_t)tm_count * ceil_div(p->N.size, (uint32_t)cand);
+                uint64_t cost = ((t + sms - 1) / sms) * (uint64_t)cand;
+                if (cost < best) {
+                    best = cost;
+                    tn = cand;
+                }
+            }
+        }
+        if (tn != 64 && tn != 128 && tn != 192 && tn != 256)
+            return GETT_ERR_UNSUPPORTED;
+        const int smem_limit = 227 * 1024;
+        int st = o.stages ? o.stages : gett_umma_max_stages(tn, smem_limit);
+        if (st < 3 || st > gett_umma_max_stages(tn, smem_limit))
+            return GETT_ERR_UNSUPPORTED;
+        info.tile_m = 128;
+        info.tile_n = tn;
+        info.tile_k = 64;
+        info.stages = st;
+        info.block = gett_umma_block();
+        info.smem_bytes = gett_umma_smem_bytes(tn, st);
+        info.epilogue = GETT_EPI_DIRECT;
     }
     p->tiles_m = ceil_div(p->M.size, (uint32_t)info.tile_m);
     p->tiles_n = ceil_div(p->N.size, (uint32_t)info.tile_n);
@@ -335,6 +374,8 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     p->k_per_split = slabs_per * (uint32_t)info.tile_k;
     info.workspace_bytes = split > 1 ? (int64_t)split * p->M.size * p->N.size * 4 : 0;
     info.grid = (int32_t)(tiles * split);
+    if (path == GETT_PATH_UMMA) // persistent: one CTA per SM walks the work list
+        info.grid = (int32_t)std::min<uint64_t>(tiles * split, (uint64_t)sms);
     return GETT_OK;
 }
 
