@@ -210,7 +210,8 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = _peaks()
-    w = workload(args.workload)
+    scale = {kv.split("=")[0]: int(kv.split("=")[1]) for kv in args.scale.split(",") if kv}
+    w = workload(args.workload, scale or None)
     dtype = DTYPE_BY_NAME[args.dtype]
     con = w.contraction
     M, N, K = con.mnk()
@@ -252,7 +253,7 @@ def run_ours(args):
             e1.record(stream)
         torch.cuda.synchronize()
         # keep the sampler alive long enough for at least a few samples
-        while time.perf_counter() - t_wall0 < 0.7:
+        while not args.kernel_only and time.perf_counter() - t_wall0 < 1.5:
             step()
             torch.cuda.synchronize()
     if plan.device_status() != 0:
@@ -299,7 +300,11 @@ def run_ours(args):
                 "roofline_time_ms": t_roof * 1e3}
 
     out = None
-    if rank == 0:
+    if rank == 0 and args.kernel_only:
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": sec_per_step * 1e3,
+               "config": {"workload": f"{w.key} {DTYPE_NAMES[dtype]} {M}x{N}x{K}", "info": info},
+               "roofline": roofline, "clocks": clocks}
+    elif rank == 0:
         # ---- end to end through the C ABI with host buffers ----
         pin = [torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
                for x in (a, b, c)]
@@ -415,6 +420,9 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=sorted(DTYPE_BY_NAME))
     ap.add_argument("--path", type=int, default=0, help="force a gett_path_t")
     ap.add_argument("--split-k", type=int, default=0)
+    ap.add_argument("--scale", default="", help="override extents, e.g. m=4096,n=4096 (profiling)")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="skip the end-to-end, equal-GEMM and CPU legs (profiling runs)")
     ap.add_argument("--all", action="store_true", help="also time every workload")
     ap.add_argument("--all-steps", type=int, default=10)
     ap.add_argument("--e2e-steps", type=int, default=5)

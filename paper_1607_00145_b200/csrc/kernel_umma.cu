@@ -44,16 +44,14 @@ constexpr uint32_t ATOM_BYTES = 1024;      // 8 rows x 128 B
 constexpr uint32_t MN_BLOCK_BYTES = 8192;  // one 64-wide block of an MN-major operand: 64 k rows
 
 struct SmemTables {
-    int64_t rowA[TILE_M];                   // A offset of each tile row (-1: beyond M)
-    int64_t rowB[256];                      // B offset of each tile column (-1: beyond N)
     int64_t colC[256];                      // C offset of each tile column (epilogue)
-    int64_t kTab[NUM_PROD_WARPS][2][TILE_K]; // per producer warp: A and B offsets of the slab's k
+    int64_t kTab[NUM_PROD_WARPS][2][TILE_K]; // per producer warp: A and B byte offsets of the slab's k
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort_flag;
 };
 
-__host__ __device__ inline uint32_t stage_bytes(uint32_t tile_n) { return A_STAGE_BYTES + tile_n * TILE_K * 2; }
+__host__ __device__ constexpr uint32_t stage_bytes(uint32_t tile_n) { return A_STAGE_BYTES + tile_n * TILE_K * 2; }
 
 struct WorkItem {
     uint32_t m0, n0, z, kbeg, kend, nslab;
@@ -67,53 +65,101 @@ __device__ __forceinline__ WorkItem decode_work(const GettKernelArgs& g, uint32_
     const uint32_t t = w - it.z * tiles;
     const uint32_t tn = t / g.tiles_m;
     it.m0 = (t - tn * g.tiles_m) * TILE_M;
-    it.n0 = tn * g.tile_n;
+    it.n0 = tn * (uint32_t)g.tile_n;
     it.kbeg = it.z * g.k_per_split;
     it.kend = min(g.K.size, it.kbeg + g.k_per_split);
     it.nslab = (it.kend - it.kbeg + TILE_K - 1) / TILE_K;
     return it;
 }
 
-// Gather one operand tile of `rows` free indices x 64 k into a stage buffer.
-//   VEC_FREE: pieces run along the free dimension (8 consecutive free indices).
-//   VEC_K   : pieces run along k (8 consecutive k).
-template <bool VEC_K>
-__device__ __forceinline__ void load_operand(const char* __restrict__ base, uint32_t smem_dst,
-                                             const int64_t* rowTab, const int64_t* kTab,
-                                             uint32_t rows, uint32_t pt)
-{
-    const uint32_t pieces = rows * (TILE_K / 8);
-    if (VEC_K) {
-        // piece q: kc = q % 8 (which 8 k of the slab), r = q / 8
-        const uint32_t kc = pt & 7;
-        const int64_t ko = kTab[kc * 8];
-#pragma unroll 4
-        for (uint32_t q = pt; q < pieces; q += PROD_THREADS) {
-            const uint32_t r = q >> 3;
-            const int64_t ro = rowTab[r];
-            const bool ok = (ro >= 0) && (ko >= 0);
-            const char* src = base + (ok ? (ro + ko) * 2 : 0);
-            const uint32_t dst = smem_dst + r * 128 + ((kc ^ (r & 7)) << 4);
-            ptx::cp_async_16(dst, src, ok ? 16u : 0u);
-        }
-    } else {
-        // piece q: fc = q % (rows / 8) (which 8 free indices), k = q / (rows / 8)
-        const uint32_t fpr = rows >> 3;
-#pragma unroll 4
-        for (uint32_t q = pt; q < pieces; q += PROD_THREADS) {
-            const uint32_t k = q / fpr;
-            const uint32_t fc = q - k * fpr;
-            const int64_t ro = rowTab[fc * 8];
-            const int64_t ko = kTab[k];
-            const bool ok = (ro >= 0) && (ko >= 0);
-            const char* src = base + (ok ? (ro + ko) * 2 : 0);
-            const uint32_t dst = smem_dst + (fc >> 3) * MN_BLOCK_BYTES + k * 128 + (((fc & 7) ^ (k & 7)) << 4);
-            ptx::cp_async_16(dst, src, ok ? 16u : 0u);
+// Producer-side state for one operand tile of R free indices x 64 k.
+//
+// VEC_K   : 16-byte pieces run along k.  Thread pt owns k-piece kc = pt % 8 of rows
+//           pt/8 + 16 p (p = 0 .. R/16-1); the byte offsets of its rows live in
+//           registers for the whole tile, so a piece costs one 64-bit add.
+// VEC_FREE: pieces run along the free dimension.  Thread pt owns free-piece
+//           fc = pt % (R/8) of the k rows kgroup + kstep * p; its single row offset
+//           lives in a register and the k offsets come from the warp's slab table.
+template <bool VEC_K, int R>
+struct OperandLoader {
+    static constexpr int FPR = R / 8;                       // pieces per k row (VEC_FREE)
+    // k rows covered per pass (VEC_FREE): the largest power of two that fits the producers
+    static constexpr int KSTEP = PROD_THREADS / FPR >= 16 ? 16 : PROD_THREADS / FPR >= 8 ? 8 : 4;
+    static constexpr int ACTIVE = VEC_K ? PROD_THREADS : KSTEP * FPR;
+    static constexpr int NP = VEC_K ? R / 16 : TILE_K / KSTEP;
+    static_assert(VEC_K || TILE_K % KSTEP == 0, "k rows must divide evenly over the passes");
+
+    int64_t rowb[VEC_K ? R / 16 : 1]; // byte offsets of this thread's rows
+    uint32_t rowmask;                 // bit p: row p is inside the tensor
+    uint32_t dst_thread;              // byte offset of piece 0 inside the operand's stage buffer
+
+    __device__ __forceinline__ void setup_tile(const GettDim& D, uint32_t origin, uint32_t pt)
+    {
+        rowmask = 0;
+        if (VEC_K) {
+#pragma unroll
+            for (int p = 0; p < NP; ++p) {
+                const uint32_t r = (pt >> 3) + 16 * p;
+                int64_t x = 0, y;
+                if (origin + r < D.size) {
+                    gett_decompose(D, origin + r, x, y);
+                    rowmask |= 1u << p;
+                }
+                rowb[p] = x * 2;
+            }
+            dst_thread = (pt >> 3) * 128 + (((pt & 7) ^ ((pt >> 3) & 7)) << 4);
+        } else {
+            const uint32_t fc = pt % FPR, kgroup = pt / FPR;
+            int64_t x = 0, y;
+            if (pt < ACTIVE && origin + fc * 8 < D.size) {
+                gett_decompose(D, origin + fc * 8, x, y);
+                rowmask = 1;
+            }
+            rowb[0] = x * 2;
+            dst_thread = (fc >> 3) * MN_BLOCK_BYTES + kgroup * 128;
         }
     }
-}
 
-template <bool A_VEC_K, bool B_VEC_K>
+    // kTab: the warp's table of byte offsets of the slab's 64 k (-1 beyond the K range).
+    template <bool FAST>
+    __device__ __forceinline__ void load_slab(const char* __restrict__ base, uint32_t stage_dst,
+                                              const int64_t* kTab, uint32_t pt) const
+    {
+        if (VEC_K) {
+            const int64_t kb = kTab[(pt & 7) * 8];
+            const uint32_t dst = stage_dst + dst_thread;
+#pragma unroll
+            for (int p = 0; p < NP; ++p) {
+                if (FAST) {
+                    ptx::cp_async_16(dst + p * 2048, base + rowb[p] + kb, 16u);
+                } else {
+                    const bool ok = kb >= 0 && ((rowmask >> p) & 1u);
+                    ptx::cp_async_16(dst + p * 2048, base + (ok ? rowb[p] + kb : 0), ok ? 16u : 0u);
+                }
+            }
+        } else {
+            if (ACTIVE < PROD_THREADS && pt >= ACTIVE)
+                return;
+            const uint32_t fc = pt % FPR, kgroup = pt / FPR;
+            const uint32_t dst = stage_dst + dst_thread;
+            const char* rowp = base + rowb[0];
+#pragma unroll
+            for (int p = 0; p < NP; ++p) {
+                const uint32_t k = kgroup + KSTEP * p;
+                const int64_t kb = kTab[k];
+                const uint32_t d = dst + p * (KSTEP * 128) + (((fc & 7) ^ (k & 7)) << 4);
+                if (FAST) {
+                    ptx::cp_async_16(d, rowp + kb, 16u);
+                } else {
+                    const bool ok = kb >= 0 && rowmask;
+                    ptx::cp_async_16(d, ok ? rowp + kb : base, ok ? 16u : 0u);
+                }
+            }
+        }
+    }
+};
+
+template <bool A_VEC_K, bool B_VEC_K, int TILE_N>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
 {
@@ -123,7 +169,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
     const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
     uint8_t* smem = smem_raw + pad;
     const uint32_t stages = (uint32_t)g.stages;
-    const uint32_t sbytes = stage_bytes(g.tile_n);
+    constexpr uint32_t sbytes = stage_bytes(TILE_N);
     SmemTables* T = reinterpret_cast<SmemTables*>(smem + stages * sbytes);
     const uint32_t stage0 = ptx::smem_u32(smem);
 
@@ -158,33 +204,29 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
         const uint32_t pw = warp - PROD_WARP0;
         int64_t* kA = T->kTab[pw][0];
         int64_t* kB = T->kTab[pw][1];
+        OperandLoader<A_VEC_K, TILE_M> la;
+        OperandLoader<B_VEC_K, TILE_N> lb;
+        const char* baseA = static_cast<const char*>(g.A);
+        const char* baseB = static_cast<const char*>(g.B);
         uint32_t it = 0, signalled = 0;
         bool alive = true;
         for (uint32_t w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
             const WorkItem wi = decode_work(g, w);
-            ptx::named_barrier(1, PROD_THREADS); // previous tile's row tables no longer read
-            for (uint32_t r = pt; r < TILE_M; r += PROD_THREADS) {
-                int64_t x = -1, y;
-                if (wi.m0 + r < g.M.size)
-                    gett_decompose(g.M, wi.m0 + r, x, y);
-                T->rowA[r] = x;
-            }
-            for (uint32_t c = pt; c < g.tile_n; c += PROD_THREADS) {
-                int64_t x = -1, y;
-                if (wi.n0 + c < g.N.size)
-                    gett_decompose(g.N, wi.n0 + c, x, y);
-                T->rowB[c] = x;
-            }
-            ptx::named_barrier(1, PROD_THREADS);
+            la.setup_tile(g.M, wi.m0, pt);
+            lb.setup_tile(g.N, wi.n0, pt);
+            const bool tile_full = wi.m0 + TILE_M <= g.M.size && wi.n0 + TILE_N <= g.N.size;
             for (uint32_t j = 0; j < wi.nslab; ++j, ++it) {
                 const uint32_t k0 = wi.kbeg + j * TILE_K;
-                __syncwarp();
+                __syncwarp(); // the warp is done reading the previous slab's table
 #pragma unroll
                 for (uint32_t h = 0; h < TILE_K / 32; ++h) {
                     const uint32_t k = k0 + h * 32 + lane;
                     int64_t x = -1, y = -1;
-                    if (k < wi.kend)
+                    if (k < wi.kend) {
                         gett_decompose(g.K, k, x, y);
+                        x *= 2;
+                        y *= 2;
+                    }
                     kA[h * 32 + lane] = x;
                     kB[h * 32 + lane] = y;
                 }
@@ -195,9 +237,13 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
                     break;
                 }
                 const uint32_t sa = stage0 + s * sbytes;
-                load_operand<A_VEC_K>(static_cast<const char*>(g.A), sa, T->rowA, kA, TILE_M, pt);
-                load_operand<B_VEC_K>(static_cast<const char*>(g.B), sa + A_STAGE_BYTES, T->rowB, kB,
-                                      g.tile_n, pt);
+                if (tile_full && k0 + TILE_K <= wi.kend) {
+                    la.template load_slab<true>(baseA, sa, kA, pt);
+                    lb.template load_slab<true>(baseB, sa + A_STAGE_BYTES, kB, pt);
+                } else {
+                    la.template load_slab<false>(baseA, sa, kA, pt);
+                    lb.template load_slab<false>(baseB, sa + A_STAGE_BYTES, kB, pt);
+                }
                 ptx::cp_async_commit();
                 if (it >= LAG) {
                     ptx::cp_async_wait<LAG>();
@@ -217,7 +263,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
         // ------------------------------ MMA issuer -----------------------------
         if (lane == 0) {
             const uint32_t fmt = g.dtype == GETT_BF16_F32 ? 1u : 0u;
-            const uint32_t idesc = ptx::idesc_f16(fmt, A_VEC_K ? 0u : 1u, B_VEC_K ? 0u : 1u, TILE_M, g.tile_n);
+            const uint32_t idesc = ptx::idesc_f16(fmt, A_VEC_K ? 0u : 1u, B_VEC_K ? 0u : 1u, TILE_M, TILE_N);
             // bytes the descriptor start address advances per 16-wide k step
             const uint32_t a_step = A_VEC_K ? 32u : 2u * ATOM_BYTES;
             const uint32_t b_step = B_VEC_K ? 32u : 2u * ATOM_BYTES;
@@ -267,7 +313,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
             if (wi.m0 + et < g.M.size)
                 gett_decompose(g.M, wi.m0 + et, dummy, rowC);
             ptx::named_barrier(2, NUM_EPI_WARPS * 32); // previous tile's column table no longer read
-            for (uint32_t c = et; c < g.tile_n; c += NUM_EPI_WARPS * 32) {
+            for (uint32_t c = et; c < TILE_N; c += NUM_EPI_WARPS * 32) {
                 int64_t x, y = -1;
                 if (wi.n0 + c < g.N.size)
                     gett_decompose(g.N, wi.n0 + c, x, y);
@@ -280,7 +326,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
             const uint32_t taddr = tmem_base + ((warp * 32u) << 16) + buf * 256;
             const bool row_ok = rowC >= 0;
             const float alpha = g.alpha, beta = g.beta;
-            for (uint32_t c0 = 0; c0 < g.tile_n; c0 += 32) {
+            for (uint32_t c0 = 0; c0 < TILE_N; c0 += 32) {
                 uint32_t v[32];
                 ptx::tmem_ld_32x32(taddr + c0, v);
                 ptx::tmem_wait_ld();
@@ -336,21 +382,32 @@ int gett_umma_max_stages(int tile_n, int smem_limit)
 
 int gett_umma_block() { return NUM_THREADS; }
 
-cudaError_t gett_launch_umma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
+template <bool AK, bool BK>
+static cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
 {
     void (*k)(GettKernelArgs);
-    const bool ak = args.loader_a == GETT_LOAD_VEC_K, bk = args.loader_b == GETT_LOAD_VEC_K;
-    if (ak && bk)
-        k = gett_umma_kernel<true, true>;
-    else if (ak)
-        k = gett_umma_kernel<true, false>;
-    else if (bk)
-        k = gett_umma_kernel<false, true>;
-    else
-        k = gett_umma_kernel<false, false>;
+    switch (args.tile_n) {
+    case 64: k = gett_umma_kernel<AK, BK, 64>; break;
+    case 128: k = gett_umma_kernel<AK, BK, 128>; break;
+    case 192: k = gett_umma_kernel<AK, BK, 192>; break;
+    case 256: k = gett_umma_kernel<AK, BK, 256>; break;
+    default: return cudaErrorInvalidValue;
+    }
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess)
         return e;
     k<<<grid, NUM_THREADS, smem, stream>>>(args);
     return cudaGetLastError();
+}
+
+cudaError_t gett_launch_umma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
+{
+    const bool ak = args.loader_a == GETT_LOAD_VEC_K, bk = args.loader_b == GETT_LOAD_VEC_K;
+    if (ak && bk)
+        return launch_tn<true, true>(args, grid, smem, stream);
+    if (ak)
+        return launch_tn<true, false>(args, grid, smem, stream);
+    if (bk)
+        return launch_tn<false, true>(args, grid, smem, stream);
+    return launch_tn<false, false>(args, grid, smem, stream);
 }
