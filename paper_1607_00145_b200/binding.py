@@ -18,7 +18,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 
 
 def library_path() -> str:
-    return os.path.join(_HERE, "libgett_b200.so")
+    """The in-tree shared library; GETT_LIBRARY names another build of it."""
+    return os.environ.get("GETT_LIBRARY") or os.path.join(_HERE, "libgett_b200.so")
 
 
 class _Desc(ctypes.Structure):

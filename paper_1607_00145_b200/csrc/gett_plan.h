@@ -72,3 +72,4 @@ gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, si
 int gett_umma_smem_bytes(int tile_n, int stages);
 int gett_umma_max_stages(int tile_n, int smem_limit);
 int gett_umma_block();
+int gett_umma_stage_multiple(); // the ring depth must be a multiple of this

@@ -32,20 +32,33 @@ constexpr int TILE_M = 128;
 constexpr int TILE_K = 64;           // 16-bit elements per slab = one 128-byte swizzle row
 constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;
 constexpr int NUM_EPI_WARPS = 4;
-constexpr int NUM_PROD_WARPS = 4;
+#ifndef GETT_PROD_GROUPS
+#define GETT_PROD_GROUPS 4
+#endif
+#ifndef GETT_WARPS_PER_GROUP
+#define GETT_WARPS_PER_GROUP 2
+#endif
+constexpr int PROD_GROUPS = GETT_PROD_GROUPS; // slab number it belongs to producer group it % PROD_GROUPS
+constexpr int WARPS_PER_GROUP = GETT_WARPS_PER_GROUP;
+constexpr int GROUP_LANES = WARPS_PER_GROUP * 32;
+constexpr int NUM_PROD_WARPS = PROD_GROUPS * WARPS_PER_GROUP;
 constexpr int MMA_WARP = NUM_EPI_WARPS;
 constexpr int PROD_WARP0 = NUM_EPI_WARPS + 1;
 constexpr int NUM_THREADS = (NUM_EPI_WARPS + 1 + NUM_PROD_WARPS) * 32;
 constexpr int PROD_THREADS = NUM_PROD_WARPS * 32;
-constexpr int LAG = 2;               // slabs a producer keeps in flight before it signals
 constexpr int MAX_STAGES = 8;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t ATOM_BYTES = 1024;      // 8 rows x 128 B
 constexpr uint32_t MN_BLOCK_BYTES = 8192;  // one 64-wide block of an MN-major operand: 64 k rows
 
+constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-byte-unit offset tables
+
+// Offsets in the producer tables are in units of 16 bytes (every vector a producer
+// copies starts on a 16-byte boundary), which keeps them in 32 bits.
 struct SmemTables {
-    int64_t colC[256];                      // C offset of each tile column (epilogue)
-    int64_t kTab[NUM_PROD_WARPS][2][TILE_K]; // per producer warp: A and B byte offsets of the slab's k
+    int64_t colC[256];                        // C offset of each tile column (epilogue)
+    uint32_t kTab[PROD_GROUPS][2][TILE_K];    // per producer group: A / B offsets of the slab's k
+    uint32_t rowTab[PROD_GROUPS][TILE_M + 256]; // per producer group: row offsets (K-major operands)
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -72,87 +85,95 @@ __device__ __forceinline__ WorkItem decode_work(const GettKernelArgs& g, uint32_
     return it;
 }
 
-// Producer-side state for one operand tile of R free indices x 64 k.
+// One producer group (GROUP_LANES threads) gathers a whole operand slab of R free
+// indices x 64 k.  gl = the thread's index inside its group.
 //
-// VEC_K   : 16-byte pieces run along k.  Thread pt owns k-piece kc = pt % 8 of rows
-//           pt/8 + 16 p (p = 0 .. R/16-1); the byte offsets of its rows live in
-//           registers for the whole tile, so a piece costs one 64-bit add.
-// VEC_FREE: pieces run along the free dimension.  Thread pt owns free-piece
-//           fc = pt % (R/8) of the k rows kgroup + kstep * p; its single row offset
-//           lives in a register and the k offsets come from the warp's slab table.
+// VEC_K   : 16-byte pieces run along k (K-major staging).  Thread gl owns k-piece
+//           kc = gl % 8 of rows gl/8 + RP p; the rows' offsets come from the group's row
+//           table (filled once per tile), the k offset is one register per slab.
+// VEC_FREE: pieces run along the free dimension (MN-major staging).  Thread gl owns
+//           free-piece fc = gl % FPR of the k rows gl/FPR + KSTEP p; its row offset is
+//           one register per tile, the k offsets come from the group's slab table.
 template <bool VEC_K, int R>
 struct OperandLoader {
-    static constexpr int FPR = R / 8;                       // pieces per k row (VEC_FREE)
-    // k rows covered per pass (VEC_FREE): the largest power of two that fits the producers
-    static constexpr int KSTEP = PROD_THREADS / FPR >= 16 ? 16 : PROD_THREADS / FPR >= 8 ? 8 : 4;
-    static constexpr int ACTIVE = VEC_K ? PROD_THREADS : KSTEP * FPR;
-    static constexpr int NP = VEC_K ? R / 16 : TILE_K / KSTEP;
-    static_assert(VEC_K || TILE_K % KSTEP == 0, "k rows must divide evenly over the passes");
+    static constexpr int FPR = R / 8;                 // pieces per k row (VEC_FREE)
+    static constexpr int pow2_floor(int x) { return x >= 64 ? 64 : x >= 32 ? 32 : x >= 16 ? 16 : x >= 8 ? 8 : x >= 4 ? 4 : x >= 2 ? 2 : 1; }
+    static constexpr int KSTEP = pow2_floor(GROUP_LANES / FPR); // k rows per pass (VEC_FREE)
+    static constexpr int RP = GROUP_LANES / 8;                  // rows per pass (VEC_K)
+    static constexpr int ACTIVE = VEC_K ? GROUP_LANES : KSTEP * FPR;
+    static constexpr int NP = VEC_K ? (R + RP - 1) / RP : TILE_K / KSTEP;
+    static_assert(ACTIVE <= GROUP_LANES, "tile too wide for one producer group");
 
-    int64_t rowb[VEC_K ? R / 16 : 1]; // byte offsets of this thread's rows
-    uint32_t rowmask;                 // bit p: row p is inside the tensor
-    uint32_t dst_thread;              // byte offset of piece 0 inside the operand's stage buffer
+    uint32_t row16;    // VEC_FREE: this thread's row offset (16-byte units), INVALID16 if outside
+    uint32_t dst_lane; // byte offset of this thread's piece 0 inside the operand's stage buffer
 
-    __device__ __forceinline__ void setup_tile(const GettDim& D, uint32_t origin, uint32_t pt)
+    // rowTab: the group's table for this operand (used by VEC_K only; the caller
+    // synchronises the group before and after).
+    __device__ __forceinline__ void setup_tile(const GettDim& D, uint32_t origin, uint32_t gl,
+                                               uint32_t* rowTab)
     {
-        rowmask = 0;
         if (VEC_K) {
-#pragma unroll
-            for (int p = 0; p < NP; ++p) {
-                const uint32_t r = (pt >> 3) + 16 * p;
-                int64_t x = 0, y;
+            for (uint32_t r = gl; r < (uint32_t)R; r += GROUP_LANES) {
+                uint32_t v = INVALID16;
                 if (origin + r < D.size) {
+                    int64_t x, y;
                     gett_decompose(D, origin + r, x, y);
-                    rowmask |= 1u << p;
+                    v = (uint32_t)(x >> 3);
                 }
-                rowb[p] = x * 2;
+                rowTab[r] = v;
             }
-            dst_thread = (pt >> 3) * 128 + (((pt & 7) ^ ((pt >> 3) & 7)) << 4);
+            // rows gl/8 + RP p all share r % 8, so the swizzle term is a per-thread constant
+            dst_lane = (gl >> 3) * 128 + (((gl & 7) ^ ((gl >> 3) & 7)) << 4);
+            row16 = 0;
         } else {
-            const uint32_t fc = pt % FPR, kgroup = pt / FPR;
-            int64_t x = 0, y;
-            if (pt < ACTIVE && origin + fc * 8 < D.size) {
+            const uint32_t fc = gl % FPR, kgroup = gl / FPR;
+            row16 = INVALID16;
+            if (gl < ACTIVE && origin + fc * 8 < D.size) {
+                int64_t x, y;
                 gett_decompose(D, origin + fc * 8, x, y);
-                rowmask = 1;
+                row16 = (uint32_t)(x >> 3);
             }
-            rowb[0] = x * 2;
-            dst_thread = (fc >> 3) * MN_BLOCK_BYTES + kgroup * 128;
+            dst_lane = (fc >> 3) * MN_BLOCK_BYTES + kgroup * 128;
         }
     }
 
-    // kTab: the warp's table of byte offsets of the slab's 64 k (-1 beyond the K range).
     template <bool FAST>
     __device__ __forceinline__ void load_slab(const char* __restrict__ base, uint32_t stage_dst,
-                                              const int64_t* kTab, uint32_t pt) const
+                                              const uint32_t* kTab, const uint32_t* rowTab,
+                                              uint32_t gl) const
     {
         if (VEC_K) {
-            const int64_t kb = kTab[(pt & 7) * 8];
-            const uint32_t dst = stage_dst + dst_thread;
-#pragma unroll
+            const uint32_t k16 = kTab[(gl & 7) * 8];
+            const uint32_t dst = stage_dst + dst_lane;
+            const uint32_t* rows = rowTab + (gl >> 3);
+#pragma unroll 8
             for (int p = 0; p < NP; ++p) {
+                if (R % RP != 0 && (gl >> 3) + RP * p >= (uint32_t)R)
+                    break;
+                const uint32_t r16 = rows[RP * p];
                 if (FAST) {
-                    ptx::cp_async_16(dst + p * 2048, base + rowb[p] + kb, 16u);
+                    ptx::cp_async_16(dst + p * (RP * 128), base + ((uint64_t)(r16 + k16) << 4), 16u);
                 } else {
-                    const bool ok = kb >= 0 && ((rowmask >> p) & 1u);
-                    ptx::cp_async_16(dst + p * 2048, base + (ok ? rowb[p] + kb : 0), ok ? 16u : 0u);
+                    const bool ok = r16 != INVALID16 && k16 != INVALID16;
+                    ptx::cp_async_16(dst + p * (RP * 128), base + (ok ? ((uint64_t)(r16 + k16) << 4) : 0),
+                                     ok ? 16u : 0u);
                 }
             }
         } else {
-            if (ACTIVE < PROD_THREADS && pt >= ACTIVE)
+            if (ACTIVE < GROUP_LANES && gl >= ACTIVE)
                 return;
-            const uint32_t fc = pt % FPR, kgroup = pt / FPR;
-            const uint32_t dst = stage_dst + dst_thread;
-            const char* rowp = base + rowb[0];
-#pragma unroll
+            const uint32_t fc = gl % FPR, kgroup = gl / FPR;
+            const uint32_t dst = stage_dst + dst_lane;
+#pragma unroll 8
             for (int p = 0; p < NP; ++p) {
                 const uint32_t k = kgroup + KSTEP * p;
-                const int64_t kb = kTab[k];
+                const uint32_t k16 = kTab[k];
                 const uint32_t d = dst + p * (KSTEP * 128) + (((fc & 7) ^ (k & 7)) << 4);
                 if (FAST) {
-                    ptx::cp_async_16(d, rowp + kb, 16u);
+                    ptx::cp_async_16(d, base + ((uint64_t)(row16 + k16) << 4), 16u);
                 } else {
-                    const bool ok = kb >= 0 && rowmask;
-                    ptx::cp_async_16(d, ok ? rowp + kb : base, ok ? 16u : 0u);
+                    const bool ok = row16 != INVALID16 && k16 != INVALID16;
+                    ptx::cp_async_16(d, base + (ok ? ((uint64_t)(row16 + k16) << 4) : 0), ok ? 16u : 0u);
                 }
             }
         }
@@ -179,7 +200,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < stages; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&T->full[s]), PROD_THREADS);
+            ptx::mbar_init(ptx::smem_u32(&T->full[s]), GROUP_LANES); // the slab's producer group
             ptx::mbar_init(ptx::smem_u32(&T->empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -200,65 +221,73 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
 
     if (warp >= PROD_WARP0) {
         // ------------------------------ producers ------------------------------
-        const uint32_t pt = threadIdx.x - PROD_WARP0 * 32;
-        const uint32_t pw = warp - PROD_WARP0;
-        int64_t* kA = T->kTab[pw][0];
-        int64_t* kB = T->kTab[pw][1];
+        // Slab number `it` (counted over the CTA's whole work list) belongs to producer
+        // group it % PROD_GROUPS, so PROD_GROUPS slabs are gathered concurrently.  The
+        // ring depth is a multiple of PROD_GROUPS, hence a stage's barriers are always
+        // used by the same group, which therefore observes every one of their phases.
+        const uint32_t pg = (warp - PROD_WARP0) / WARPS_PER_GROUP;
+        const uint32_t gl = threadIdx.x - (PROD_WARP0 + pg * WARPS_PER_GROUP) * 32;
+        const uint32_t gbar = 3 + pg; // named barrier of this group
+        uint32_t* kA = T->kTab[pg][0];
+        uint32_t* kB = T->kTab[pg][1];
+        uint32_t* rowA = T->rowTab[pg];
+        uint32_t* rowB = T->rowTab[pg] + TILE_M;
         OperandLoader<A_VEC_K, TILE_M> la;
         OperandLoader<B_VEC_K, TILE_N> lb;
         const char* baseA = static_cast<const char*>(g.A);
         const char* baseB = static_cast<const char*>(g.B);
-        uint32_t it = 0, signalled = 0;
+        uint32_t first = 0; // slab number of the current work item's first slab
         bool alive = true;
-        for (uint32_t w = blockIdx.x; w < total_work && alive; w += gridDim.x) {
+        for (uint32_t w = blockIdx.x; w < total_work; w += gridDim.x) {
             const WorkItem wi = decode_work(g, w);
-            la.setup_tile(g.M, wi.m0, pt);
-            lb.setup_tile(g.N, wi.n0, pt);
-            const bool tile_full = wi.m0 + TILE_M <= g.M.size && wi.n0 + TILE_N <= g.N.size;
-            for (uint32_t j = 0; j < wi.nslab; ++j, ++it) {
-                const uint32_t k0 = wi.kbeg + j * TILE_K;
-                __syncwarp(); // the warp is done reading the previous slab's table
-#pragma unroll
-                for (uint32_t h = 0; h < TILE_K / 32; ++h) {
-                    const uint32_t k = k0 + h * 32 + lane;
-                    int64_t x = -1, y = -1;
-                    if (k < wi.kend) {
-                        gett_decompose(g.K, k, x, y);
-                        x *= 2;
-                        y *= 2;
-                    }
-                    kA[h * 32 + lane] = x;
-                    kB[h * 32 + lane] = y;
-                }
-                __syncwarp();
-                const uint32_t s = it % stages;
-                if (!ptx::mbar_wait(ptx::smem_u32(&T->empty[s]), ((it / stages) & 1) ^ 1, abort_flag)) {
-                    alive = false;
-                    break;
-                }
-                const uint32_t sa = stage0 + s * sbytes;
-                if (tile_full && k0 + TILE_K <= wi.kend) {
-                    la.template load_slab<true>(baseA, sa, kA, pt);
-                    lb.template load_slab<true>(baseB, sa + A_STAGE_BYTES, kB, pt);
-                } else {
-                    la.template load_slab<false>(baseA, sa, kA, pt);
-                    lb.template load_slab<false>(baseB, sa + A_STAGE_BYTES, kB, pt);
-                }
-                ptx::cp_async_commit();
-                if (it >= LAG) {
-                    ptx::cp_async_wait<LAG>();
-                    ptx::fence_proxy_async_smem();
-                    ptx::mbar_arrive(ptx::smem_u32(&T->full[signalled % stages]));
-                    ++signalled;
-                }
+            // my group's first slab in this item: smallest j with (first + j) % PROD_GROUPS == pg
+            uint32_t j = (pg + PROD_GROUPS - first % PROD_GROUPS) % PROD_GROUPS;
+            if (j < wi.nslab) {
+                ptx::named_barrier(gbar, GROUP_LANES); // the group is done with the previous tables
+                la.setup_tile(g.M, wi.m0, gl, rowA);
+                lb.setup_tile(g.N, wi.n0, gl, rowB);
             }
+            const bool tile_full = wi.m0 + TILE_M <= g.M.size && wi.n0 + TILE_N <= g.N.size;
+            for (; j < wi.nslab; j += PROD_GROUPS) {
+                const uint32_t it = first + j;
+                const uint32_t k0 = wi.kbeg + j * TILE_K;
+                ptx::named_barrier(gbar, GROUP_LANES); // previous slab's k table no longer read
+                if (!(g.debug & 16) && gl < TILE_K) {
+                    const uint32_t k = k0 + gl;
+                    uint32_t xa = INVALID16, xb = INVALID16;
+                    if (k < wi.kend) {
+                        int64_t x, y;
+                        gett_decompose(g.K, k, x, y);
+                        xa = (uint32_t)(x >> 3);
+                        xb = (uint32_t)(y >> 3);
+                    }
+                    kA[gl] = xa;
+                    kB[gl] = xb;
+                }
+                ptx::named_barrier(gbar, GROUP_LANES); // tables (rows and k) complete
+                const uint32_t s = it % stages;
+                // After a timeout a thread keeps walking the loop (so its group's named
+                // barriers stay matched) but neither waits nor copies any more.
+                if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->empty[s]), ((it / stages) & 1) ^ 1, abort_flag))
+                    alive = false;
+                if (!alive)
+                    continue;
+                const uint32_t sa = stage0 + s * sbytes;
+                if (g.debug & 4) {
+                    // experiment switch: no copies at all (measures the rest of the pipeline)
+                } else if (tile_full && k0 + TILE_K <= wi.kend) {
+                    la.template load_slab<true>(baseA, sa, kA, rowA, gl);
+                    lb.template load_slab<true>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+                } else {
+                    la.template load_slab<false>(baseA, sa, kA, rowA, gl);
+                    lb.template load_slab<false>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+                }
+                // full[s] hears from this thread when its copies for the slab have landed
+                ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&T->full[s]));
+            }
+            first += wi.nslab;
         }
-        // drain: everything this thread issued has landed; signal the remaining slabs
-        ptx::cp_async_wait<0>();
-        ptx::fence_proxy_async_smem();
-        if (alive)
-            for (; signalled < it; ++signalled)
-                ptx::mbar_arrive(ptx::smem_u32(&T->full[signalled % stages]));
+        ptx::cp_async_wait_all();
     } else if (warp == MMA_WARP) {
         // ------------------------------ MMA issuer -----------------------------
         if (lane == 0) {
@@ -284,6 +313,10 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
                         alive = false;
                         break;
                     }
+                    // the copies were generic-proxy writes; the tensor core reads through the
+                    // async proxy, so order the two before issuing
+                    if (!(g.debug & 8))
+                        ptx::fence_proxy_async_smem();
                     ptx::tc_fence_after();
                     const uint32_t sa = stage0 + s * sbytes, sb = sa + A_STAGE_BYTES;
 #pragma unroll
@@ -305,6 +338,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
         // ------------------------------- epilogue ------------------------------
         const uint32_t et = threadIdx.x; // 0..127: tile row, = tensor-memory lane
         uint32_t local = 0;
+        bool alive = true;
         for (uint32_t w = blockIdx.x; w < total_work; w += gridDim.x, ++local) {
             const WorkItem wi = decode_work(g, w);
             const uint32_t buf = local & 1;
@@ -320,35 +354,47 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
                 T->colC[c] = y;
             }
             ptx::named_barrier(2, NUM_EPI_WARPS * 32);
-            if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), (local >> 1) & 1, abort_flag))
-                break;
+            if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), (local >> 1) & 1, abort_flag))
+                alive = false;
+            if (!alive)
+                continue; // keep the named barriers above matched, do nothing else
             ptx::tc_fence_after();
             const uint32_t taddr = tmem_base + ((warp * 32u) << 16) + buf * 256;
             const bool row_ok = rowC >= 0;
             const float alpha = g.alpha, beta = g.beta;
-            for (uint32_t c0 = 0; c0 < TILE_N; c0 += 32) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(taddr + c0, v);
+            for (uint32_t c0 = 0; c0 < TILE_N; c0 += 16) {
+                uint32_t v[16];
+                ptx::tmem_ld_32x16(taddr + c0, v);
                 ptx::tmem_wait_ld();
-                if (!row_ok)
+                if (!row_ok || (g.debug & 2)) // (debug & 2: experiment switch, no stores)
                     continue;
                 if (g.split_k > 1) {
                     float* dst = g.ws + ((size_t)wi.z * g.N.size + wi.n0 + c0) * g.M.size + wi.m0 + et;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
+                    for (int i = 0; i < 16; ++i)
                         if (wi.n0 + c0 + i < g.N.size)
                             dst[(size_t)i * g.M.size] = __uint_as_float(v[i]);
                 } else {
                     float* crow = g.C + rowC;
+                    int64_t co[16];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int64_t co = T->colC[c0 + i];
-                        if (co >= 0) {
-                            float r = alpha * __uint_as_float(v[i]);
-                            if (beta != 0.f)
-                                r = fmaf(beta, crow[co], r);
-                            crow[co] = r;
-                        }
+                    for (int i = 0; i < 16; ++i)
+                        co[i] = T->colC[c0 + i];
+                    if (beta != 0.f) {
+                        // all reads of the old C first, so their latencies overlap
+                        float old[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            old[i] = co[i] >= 0 ? __ldcg(crow + co[i]) : 0.f;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (co[i] >= 0)
+                                crow[co[i]] = fmaf(beta, old[i], alpha * __uint_as_float(v[i]));
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (co[i] >= 0)
+                                crow[co[i]] = alpha * __uint_as_float(v[i]);
                     }
                 }
             }
@@ -377,10 +423,13 @@ int gett_umma_smem_bytes(int tile_n, int stages)
 int gett_umma_max_stages(int tile_n, int smem_limit)
 {
     int s = (smem_limit - 1024 - (int)sizeof(SmemTables)) / (int)stage_bytes((uint32_t)tile_n);
-    return s > MAX_STAGES ? MAX_STAGES : s;
+    s = s > MAX_STAGES ? MAX_STAGES : s;
+    return s - s % PROD_GROUPS; // a stage must always be served by the same producer group
 }
 
 int gett_umma_block() { return NUM_THREADS; }
+
+int gett_umma_stage_multiple() { return PROD_GROUPS; }
 
 template <bool AK, bool BK>
 static cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)

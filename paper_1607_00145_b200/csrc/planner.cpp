@@ -322,14 +322,14 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
             return GETT_ERR_UNSUPPORTED;
         int tn = o.tile_n;
         if (tn == 0) {
-            // fewest (waves x tile width); ties go to the wider tile
+            // fewest waves x per-tile cost; ties go to the wider tile
             const uint32_t tm_count = ceil_div(p->M.size, 128);
             uint64_t best = UINT64_MAX;
             for (int cand : {256, 192, 128, 64}) {
                 if (cand > 64 && (uint32_t)cand >= p->N.size + 64)
                     continue; // a narrower tile already covers N
                 uint64_t t = (uint64_t)tm_count * ceil_div(p->N.size, (uint32_t)cand);
-                uint64_t cost = ((t + sms - 1) / sms) * (uint64_t)cand;
+                uint64_t cost = ((t + sms - 1) / sms) * (uint64_t)(cand + 64); // MMA width + A reload
                 if (cost < best) {
                     best = cost;
                     tn = cand;
@@ -340,7 +340,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
             return GETT_ERR_UNSUPPORTED;
         const int smem_limit = 227 * 1024;
         int st = o.stages ? o.stages : gett_umma_max_stages(tn, smem_limit);
-        if (st < 3 || st > gett_umma_max_stages(tn, smem_limit))
+        if (st < 3 || st > gett_umma_max_stages(tn, smem_limit) || st % gett_umma_stage_multiple())
             return GETT_ERR_UNSUPPORTED;
         info.tile_m = 128;
         info.tile_n = tn;
