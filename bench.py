@@ -304,6 +304,8 @@ def run_ours(args):
         out = {"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": sec_per_step * 1e3,
                "config": {"workload": f"{w.key} {DTYPE_NAMES[dtype]} {M}x{N}x{K}", "info": info},
                "roofline": roofline, "clocks": clocks}
+        if args.all:
+            out["workloads"] = run_all(torch, g, peaks, fp32_peak, args)
     elif rank == 0:
         # ---- end to end through the C ABI with host buffers ----
         pin = [torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
@@ -397,7 +399,7 @@ def run_all(torch, g, peaks, fp32_peak, args):
                        "roofline_frac": t_roof / t, "path": info["path"],
                        "tile": [info["tile_m"], info["tile_n"], info["tile_k"]],
                        "split_k": info["split_k"]}
-                if name == "auto" and key != "cfg2":
+                if name == "auto" and key != "cfg2" and not args.kernel_only:
                     eg = equal_gemm(con)
                     ga, gb, gc = make_inputs(eg, dtype, w.dist, w.seed, w.beta)
                     gdev = (_to_dev(ga, torch), _to_dev(gb, torch), _to_dev(gc, torch))

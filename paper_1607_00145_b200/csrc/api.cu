@@ -117,6 +117,7 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     args.stages = plan->info.stages;
     args.epilogue = plan->info.epilogue;
     args.debug = plan->debug;
+    args.c_vec = plan->c_vec;
 
     int path = plan->info.path;
     // the vectorised kernels need 16-byte aligned operand bases; otherwise gather scalars
@@ -134,6 +135,9 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
         err = gett_launch_simt(args, (int)grid, stream);
         break;
     }
+    case GETT_PATH_FFMA:
+        err = gett_launch_ffma(args, plan->info.grid, plan->info.smem_bytes, stream);
+        break;
     case GETT_PATH_UMMA:
         err = gett_launch_umma(args, plan->info.grid, plan->info.smem_bytes, stream);
         break;

@@ -43,6 +43,8 @@ struct GettKernelArgs {
     int32_t tile_n;       // tile width of the tensor-core / FFMA kernels
     int32_t stages;       // depth of the shared-memory ring
     int32_t epilogue;     // gett_epilogue_t
+    int32_t c_vec;        // direct epilogue: 1 = four consecutive tile rows are one aligned 16-byte
+                          // vector of C; staged epilogue: column-to-slot pattern (1 or 8)
     int32_t debug;        // opts.reserved[0]: experiment switches, 0 in normal use
 };
 
@@ -55,6 +57,7 @@ struct gett_plan {
     // geometry
     uint32_t tiles_m, tiles_n, k_per_split;
     int32_t a_kmajor, b_kmajor;
+    int32_t c_vec;
     // device side
     float* ws;
     int32_t* status;
@@ -69,7 +72,10 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* A,
 gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, size_t capacity);
 
 // Geometry of the tensor-core kernel (kernel_umma.cu), needed by the planner.
-int gett_umma_smem_bytes(int tile_n, int stages);
-int gett_umma_max_stages(int tile_n, int smem_limit);
+int gett_umma_smem_bytes(int tile_n, int stages, int staged);
+int gett_umma_max_stages(int tile_n, int smem_limit, int staged);
 int gett_umma_block();
 int gett_umma_stage_multiple(); // the ring depth must be a multiple of this
+
+// Geometry of the fp32 kernel (kernel_ffma.cu).
+int gett_ffma_smem_bytes(int tile_n, int stages);

@@ -1,0 +1,317 @@
+// Strict-fp32 contraction kernel: 16-byte cp.async gathers, register-blocked FFMA.
+//
+// One CTA of 256 threads owns a 128 x TN tile of the fused (M, N) output and walks its
+// K range in slabs of 32 through a ring of shared-memory stages (Listing 4 with the
+// m-/n-loops spread over the grid).  Packing (Eq. 9 / Eq. 10) is the gather of
+// 16-byte pieces of the A and B sub-tensors into one of two shared layouts:
+//   stride-1 mode free  ("VEC_FREE") -> [k][row]  rows contiguous, as the FMA loop reads it
+//   stride-1 mode in K  ("VEC_K")    -> [row][k]  32 k = 128 B per row, 16-byte pieces
+//                                       XOR-swizzled by (row / 4) % 8 so that both the
+//                                       copy and the 128-bit fragment reads are
+//                                       bank-conflict free
+// The macro-kernel is an 8 x (TN/16) register tile per thread fed by 128-bit shared
+// loads (Sec. 3.1: outer products into a register-resident tile); unpacking
+// (Eq. 11) writes alpha*acc + beta*C through C's permutation, as 128-bit stores
+// along M when C's stride-1 mode leads the M order.
+#include "kernels.h"
+#include "ptx_sm100.cuh"
+
+namespace {
+
+constexpr int TM = 128, TK = 32, NT = 256;
+constexpr uint32_t INVALID16 = 0xFFFFFFFFu;
+
+template <int TN>
+struct FfmaSmem {
+    int64_t offCM[TM];
+    int64_t offCN[TN];
+    uint32_t rowA[TM];       // A row offsets, 16-byte units (INVALID16 beyond M)
+    uint32_t rowB[TN];
+    uint32_t kTab[2][2][TK]; // [parity][A/B][k] offsets of a slab's k, 16-byte units
+};
+
+template <int TN>
+__host__ __device__ constexpr int ffma_stage_bytes() { return (TM + TN) * TK * 4; }
+
+// Gather one operand slab: R rows x 32 k.
+template <bool VEC_K, int R>
+__device__ __forceinline__ void load_operand(const char* __restrict__ base, uint32_t dst,
+                                             const uint32_t* rowTab, const uint32_t* kTab, int tid)
+{
+    constexpr int PIECES = R * TK / 4;
+    constexpr int NP = (PIECES + NT - 1) / NT;
+    if (VEC_K) {
+        const uint32_t kc = tid & 7;
+        const uint32_t k16 = kTab[kc * 4];
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            const uint32_t m = (tid >> 3) + 32 * p;
+            if (PIECES % NT != 0 && m >= (uint32_t)R)
+                break;
+            const uint32_t r16 = rowTab[m];
+            const bool ok = r16 != INVALID16 && k16 != INVALID16;
+            ptx::cp_async_16(dst + m * 128 + ((kc ^ ((m >> 2) & 7)) << 4),
+                             base + (ok ? ((uint64_t)(r16 + k16) << 4) : 0), ok ? 16u : 0u);
+        }
+    } else {
+        constexpr int PPR = R / 4; // pieces per k row
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            const uint32_t q = tid + NT * p;
+            if (PIECES % NT != 0 && q >= (uint32_t)PIECES)
+                break;
+            const uint32_t k = q / PPR, mc = q % PPR;
+            const uint32_t r16 = rowTab[mc * 4], k16 = kTab[k];
+            const bool ok = r16 != INVALID16 && k16 != INVALID16;
+            ptx::cp_async_16(dst + (k * R + mc * 4) * 4, base + (ok ? ((uint64_t)(r16 + k16) << 4) : 0),
+                             ok ? 16u : 0u);
+        }
+    }
+}
+
+// Fragment of F (4 or 8, or 2) rows for 4 consecutive k from a [row][k] swizzled tile.
+template <int F>
+__device__ __forceinline__ void frag_kmajor(const char* tile, const uint32_t (&rows)[F], uint32_t sw,
+                                            int k4, float (&out)[F][4])
+{
+#pragma unroll
+    for (int i = 0; i < F; ++i) {
+        const float4 v = *reinterpret_cast<const float4*>(tile + rows[i] * 128 + (((uint32_t)k4 ^ sw) << 4));
+        out[i][0] = v.x;
+        out[i][1] = v.y;
+        out[i][2] = v.z;
+        out[i][3] = v.w;
+    }
+}
+
+template <bool A_K, bool B_K, int TN>
+__global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant__ GettKernelArgs g)
+{
+    constexpr int FN = TN / 16;                 // columns per thread (8 or 2)
+    constexpr int STAGE = ffma_stage_bytes<TN>();
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int stages = g.stages;
+    FfmaSmem<TN>* T = reinterpret_cast<FfmaSmem<TN>*>(smem + stages * STAGE);
+    const uint32_t smem0 = ptx::smem_u32(smem);
+
+    const uint32_t tiles = g.tiles_m * g.tiles_n;
+    const uint32_t z = blockIdx.x / tiles;
+    const uint32_t tile = blockIdx.x - z * tiles;
+    const uint32_t tn = tile / g.tiles_m, tm = tile - tn * g.tiles_m;
+    const uint32_t m0 = tm * TM, n0 = tn * TN;
+    const uint32_t Msz = g.M.size, Nsz = g.N.size;
+    const uint32_t kbeg = z * g.k_per_split;
+    const uint32_t kend = min(g.K.size, kbeg + g.k_per_split);
+    const int nslab = (int)((kend - kbeg + TK - 1) / TK);
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+
+    // ---- per-tile tables ----
+    for (int r = tid; r < TM + TN; r += NT) {
+        const bool isA = r < TM;
+        const uint32_t idx = isA ? m0 + r : n0 + (r - TM);
+        int64_t x = 0, y = 0;
+        const bool ok = idx < (isA ? Msz : Nsz);
+        if (ok)
+            gett_decompose(isA ? g.M : g.N, idx, x, y);
+        if (isA) {
+            T->rowA[r] = ok ? (uint32_t)(x >> 2) : INVALID16;
+            T->offCM[r] = ok ? y : -1;
+        } else {
+            T->rowB[r - TM] = ok ? (uint32_t)(x >> 2) : INVALID16;
+            T->offCN[r - TM] = ok ? y : -1;
+        }
+    }
+    auto fill_ktab = [&](int slab) {
+        if (tid < TK) {
+            const uint32_t k = kbeg + slab * TK + tid;
+            uint32_t xa = INVALID16, xb = INVALID16;
+            if (slab < nslab && k < kend) {
+                int64_t x, y;
+                gett_decompose(g.K, k, x, y);
+                xa = (uint32_t)(x >> 2);
+                xb = (uint32_t)(y >> 2);
+            }
+            T->kTab[slab & 1][0][tid] = xa;
+            T->kTab[slab & 1][1][tid] = xb;
+        }
+    };
+    auto issue = [&](int slab) {
+        if (slab < nslab) {
+            const uint32_t dst = smem0 + (slab % stages) * STAGE;
+            load_operand<A_K, TM>(static_cast<const char*>(g.A), dst, T->rowA, T->kTab[slab & 1][0], tid);
+            load_operand<B_K, TN>(static_cast<const char*>(g.B), dst + TM * TK * 4, T->rowB,
+                                  T->kTab[slab & 1][1], tid);
+        }
+        ptx::cp_async_commit();
+    };
+
+    // ---- prologue: fill stages - 1 slabs ----
+    for (int s = 0; s < stages - 1; ++s) {
+        fill_ktab(s);
+        __syncthreads();
+        issue(s);
+    }
+    fill_ktab(stages - 1);
+
+    // rows / columns this thread accumulates
+    uint32_t rows[8], cols[FN];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        rows[i] = (i < 4 ? 0 : 64) + tx * 4 + (i & 3);
+#pragma unroll
+    for (int j = 0; j < FN; ++j)
+        cols[j] = FN == 8 ? (j < 4 ? 0 : 64) + ty * 4 + (j & 3) : ty * FN + j;
+    const uint32_t swA = tx & 7;
+    const uint32_t swB = FN == 8 ? (ty & 7) : ((ty * FN) >> 2) & 7;
+
+    float acc[8][FN];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < FN; ++j)
+            acc[i][j] = 0.f;
+
+    for (int slab = 0; slab < nslab; ++slab) {
+        // all but the newest (stages - 2) copy groups have landed => this slab is complete
+        if (stages == 2)
+            ptx::cp_async_wait<0>();
+        else if (stages == 3)
+            ptx::cp_async_wait<1>();
+        else
+            ptx::cp_async_wait<2>();
+        __syncthreads(); // slab's data visible; previous slab's stage free; kTab ready
+        issue(slab + stages - 1);
+        fill_ktab(slab + stages); // for the issue of the next iteration
+        const char* As = reinterpret_cast<const char*>(smem) + (slab % stages) * STAGE;
+        const char* Bs = As + TM * TK * 4;
+#pragma unroll
+        for (int k4 = 0; k4 < TK / 4; ++k4) {
+            float a[8][4], b[FN][4];
+            if (A_K) {
+                frag_kmajor<8>(As, rows, swA, k4, a);
+            } else {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const float* row = reinterpret_cast<const float*>(As) + (k4 * 4 + kk) * TM;
+                    const float4 lo = *reinterpret_cast<const float4*>(row + tx * 4);
+                    const float4 hi = *reinterpret_cast<const float4*>(row + 64 + tx * 4);
+                    a[0][kk] = lo.x; a[1][kk] = lo.y; a[2][kk] = lo.z; a[3][kk] = lo.w;
+                    a[4][kk] = hi.x; a[5][kk] = hi.y; a[6][kk] = hi.z; a[7][kk] = hi.w;
+                }
+            }
+            if (B_K) {
+                frag_kmajor<FN>(Bs, cols, swB, k4, b);
+            } else {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const float* row = reinterpret_cast<const float*>(Bs) + (k4 * 4 + kk) * TN;
+                    if constexpr (FN == 8) {
+                        const float4 lo = *reinterpret_cast<const float4*>(row + ty * 4);
+                        const float4 hi = *reinterpret_cast<const float4*>(row + 64 + ty * 4);
+                        b[0][kk] = lo.x; b[1][kk] = lo.y; b[2][kk] = lo.z; b[3][kk] = lo.w;
+                        b[4][kk] = hi.x; b[5][kk] = hi.y; b[6][kk] = hi.z; b[7][kk] = hi.w;
+                    } else {
+                        const float2 v = *reinterpret_cast<const float2*>(row + ty * 2);
+                        b[0][kk] = v.x;
+                        b[1][kk] = v.y;
+                    }
+                }
+            }
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+#pragma unroll
+                    for (int j = 0; j < FN; ++j)
+                        acc[i][j] = fmaf(a[i][kk], b[j][kk], acc[i][j]);
+        }
+    }
+    ptx::cp_async_wait_all();
+    __syncthreads();
+
+    // ---- unpack: C <- alpha * acc + beta * C (or the raw slice sums under split-K) ----
+    const float alpha = g.alpha, beta = g.beta;
+    const bool vec_m = g.c_vec == 1;
+#pragma unroll
+    for (int j = 0; j < FN; ++j) {
+        const int64_t cn = T->offCN[cols[j]];
+        if (cn < 0)
+            continue;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t r0 = rows[4 * h];
+            if (g.split_k > 1) {
+                float* dst = g.ws + ((size_t)z * Nsz + n0 + cols[j]) * Msz + m0 + r0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (m0 + r0 + i < Msz)
+                        dst[i] = acc[4 * h + i][j];
+            } else if (vec_m) {
+                const int64_t cm = T->offCM[r0];
+                if (cm < 0)
+                    continue;
+                float4* dst = reinterpret_cast<float4*>(g.C + cm + cn);
+                float4 v = make_float4(alpha * acc[4 * h][j], alpha * acc[4 * h + 1][j],
+                                       alpha * acc[4 * h + 2][j], alpha * acc[4 * h + 3][j]);
+                if (beta != 0.f) {
+                    const float4 o = *dst;
+                    v.x = fmaf(beta, o.x, v.x);
+                    v.y = fmaf(beta, o.y, v.y);
+                    v.z = fmaf(beta, o.z, v.z);
+                    v.w = fmaf(beta, o.w, v.w);
+                }
+                *dst = v;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int64_t cm = T->offCM[r0 + i];
+                    if (cm < 0)
+                        continue;
+                    float* dst = g.C + cm + cn;
+                    float v = alpha * acc[4 * h + i][j];
+                    if (beta != 0.f)
+                        v = fmaf(beta, *dst, v);
+                    *dst = v;
+                }
+            }
+        }
+    }
+}
+
+template <bool AK, bool BK>
+cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
+{
+    void (*k)(GettKernelArgs);
+    if (args.tile_n == 128)
+        k = gett_ffma_kernel<AK, BK, 128>;
+    else if (args.tile_n == 32)
+        k = gett_ffma_kernel<AK, BK, 32>;
+    else
+        return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess)
+        return e;
+    k<<<grid, NT, smem, stream>>>(args);
+    return cudaGetLastError();
+}
+
+} // namespace
+
+int gett_ffma_smem_bytes(int tile_n, int stages)
+{
+    return tile_n == 128 ? stages * ffma_stage_bytes<128>() + (int)sizeof(FfmaSmem<128>)
+                         : stages * ffma_stage_bytes<32>() + (int)sizeof(FfmaSmem<32>);
+}
+
+cudaError_t gett_launch_ffma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
+{
+    const bool ak = args.loader_a == GETT_LOAD_VEC_K, bk = args.loader_b == GETT_LOAD_VEC_K;
+    if (ak && bk)
+        return launch_tn<true, true>(args, grid, smem, stream);
+    if (ak)
+        return launch_tn<true, false>(args, grid, smem, stream);
+    if (bk)
+        return launch_tn<false, true>(args, grid, smem, stream);
+    return launch_tn<false, false>(args, grid, smem, stream);
+}

@@ -50,19 +50,24 @@ constexpr int MAX_STAGES = 8;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t ATOM_BYTES = 1024;      // 8 rows x 128 B
 constexpr uint32_t MN_BLOCK_BYTES = 8192;  // one 64-wide block of an MN-major operand: 64 k rows
+constexpr int EPI_PITCH = 68;              // floats per staged row: 64 + 4 keeps 128-bit accesses conflict-free
+constexpr int EPI_STAGE_BYTES = NUM_EPI_WARPS * 32 * EPI_PITCH * 4;
 
 constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-byte-unit offset tables
 
 // Offsets in the producer tables are in units of 16 bytes (every vector a producer
 // copies starts on a 16-byte boundary), which keeps them in 32 bits.
-struct SmemTables {
+struct alignas(16) SmemTables { // the staging rows that follow it hold 128-bit vectors
     int64_t colC[256];                        // C offset of each tile column (epilogue)
+    int64_t rowCs[TILE_M];                    // C offset of each tile row (staged epilogue)
     uint32_t kTab[PROD_GROUPS][2][TILE_K];    // per producer group: A / B offsets of the slab's k
     uint32_t rowTab[PROD_GROUPS][TILE_M + 256]; // per producer group: row offsets (K-major operands)
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort_flag;
 };
+
+static_assert(sizeof(SmemTables) % 16 == 0, "staging area must stay 16-byte aligned");
 
 __host__ __device__ constexpr uint32_t stage_bytes(uint32_t tile_n) { return A_STAGE_BYTES + tile_n * TILE_K * 2; }
 
@@ -179,6 +184,78 @@ struct OperandLoader {
         }
     }
 };
+
+// ---- staged epilogue (Eq. 11 as a transposition through shared memory) ----
+// Within a 64-column chunk of the accumulator the columns are re-ordered into "slots"
+// so that four consecutive slots are four consecutive floats of C:
+//   CV == 1: the tile's columns already run along C's stride-1 mode (slot = column)
+//   CV == 8: the first N digit is the 8-wide piece of B's stride-1 mode and the second
+//            digit is C's stride-1 mode, i.e. column = a + 8 n'  ->  slot = 8 a + n'
+template <int CV>
+__device__ __forceinline__ uint32_t col_of_slot(uint32_t slot)
+{
+    return CV == 1 ? slot : (slot >> 3) + ((slot & 7) << 3);
+}
+
+// Thread `lane` of an epilogue warp writes its 32 accumulator columns (half h of the
+// chunk) into its staging row as eight 128-bit stores.
+template <int CV>
+__device__ __forceinline__ void stage_half(float* Srow, uint32_t h, const uint32_t (&v)[32])
+{
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+        float4 q;
+        if (CV == 1) {
+            q = make_float4(__uint_as_float(v[4 * a]), __uint_as_float(v[4 * a + 1]),
+                            __uint_as_float(v[4 * a + 2]), __uint_as_float(v[4 * a + 3]));
+            *reinterpret_cast<float4*>(Srow + h * 32 + 4 * a) = q;
+        } else {
+            q = make_float4(__uint_as_float(v[a]), __uint_as_float(v[a + 8]), __uint_as_float(v[a + 16]),
+                            __uint_as_float(v[a + 24]));
+            *reinterpret_cast<float4*>(Srow + a * 8 + h * 4) = q;
+        }
+    }
+}
+
+// One 64-column chunk: 32 rows x 16 float4 per warp, lanes running along C.
+template <int CV>
+__device__ __forceinline__ void store_chunk(const float* Sw, float* __restrict__ C, const int64_t* rowCs,
+                                            const int64_t* colC, uint32_t chunk, uint32_t lane,
+                                            float alpha, float beta)
+{
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        float4 val[8];
+        float* ptr[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const uint32_t q = lane + 32 * (half * 8 + t);
+            const uint32_t row = q >> 4, s4 = q & 15;
+            val[t] = *reinterpret_cast<const float4*>(Sw + row * EPI_PITCH + 4 * s4);
+            const int64_t rc = rowCs[row];
+            const int64_t cn = colC[chunk * 64 + col_of_slot<CV>(4 * s4)];
+            ptr[t] = (rc >= 0 && cn >= 0) ? C + rc + cn : nullptr;
+        }
+        if (beta != 0.f) {
+            float4 old[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+                old[t] = ptr[t] ? __ldcg(reinterpret_cast<const float4*>(ptr[t])) : make_float4(0, 0, 0, 0);
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+                if (ptr[t])
+                    *reinterpret_cast<float4*>(ptr[t]) =
+                        make_float4(fmaf(beta, old[t].x, alpha * val[t].x), fmaf(beta, old[t].y, alpha * val[t].y),
+                                    fmaf(beta, old[t].z, alpha * val[t].z), fmaf(beta, old[t].w, alpha * val[t].w));
+        } else {
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+                if (ptr[t])
+                    *reinterpret_cast<float4*>(ptr[t]) =
+                        make_float4(alpha * val[t].x, alpha * val[t].y, alpha * val[t].z, alpha * val[t].w);
+        }
+    }
+}
 
 template <bool A_VEC_K, bool B_VEC_K, int TILE_N>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -347,6 +424,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
             if (wi.m0 + et < g.M.size)
                 gett_decompose(g.M, wi.m0 + et, dummy, rowC);
             ptx::named_barrier(2, NUM_EPI_WARPS * 32); // previous tile's column table no longer read
+            T->rowCs[et] = rowC;
             for (uint32_t c = et; c < TILE_N; c += NUM_EPI_WARPS * 32) {
                 int64_t x, y = -1;
                 if (wi.n0 + c < g.N.size)
@@ -362,6 +440,31 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
             const uint32_t taddr = tmem_base + ((warp * 32u) << 16) + buf * 256;
             const bool row_ok = rowC >= 0;
             const float alpha = g.alpha, beta = g.beta;
+            if (g.epilogue == GETT_EPI_STAGED && g.split_k == 1 && !(g.debug & 2)) {
+                float* Sw = reinterpret_cast<float*>(smem + stages * sbytes + sizeof(SmemTables)) +
+                            warp * 32 * EPI_PITCH;
+                for (uint32_t chunk = 0; chunk < TILE_N / 64; ++chunk) {
+#pragma unroll
+                    for (uint32_t h = 0; h < 2; ++h) {
+                        uint32_t v[32];
+                        ptx::tmem_ld_32x32(taddr + chunk * 64 + h * 32, v);
+                        ptx::tmem_wait_ld();
+                        if (g.c_vec == 8)
+                            stage_half<8>(Sw + lane * EPI_PITCH, h, v);
+                        else
+                            stage_half<1>(Sw + lane * EPI_PITCH, h, v);
+                    }
+                    __syncwarp();
+                    if (g.c_vec == 8)
+                        store_chunk<8>(Sw, g.C, T->rowCs + warp * 32, T->colC, chunk, lane, alpha, beta);
+                    else
+                        store_chunk<1>(Sw, g.C, T->rowCs + warp * 32, T->colC, chunk, lane, alpha, beta);
+                    __syncwarp(); // the staging rows are free again
+                }
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(ptx::smem_u32(&T->acc_empty[buf]));
+                continue;
+            }
             for (uint32_t c0 = 0; c0 < TILE_N; c0 += 16) {
                 uint32_t v[16];
                 ptx::tmem_ld_32x16(taddr + c0, v);
@@ -415,14 +518,16 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
 
 } // namespace
 
-int gett_umma_smem_bytes(int tile_n, int stages)
+int gett_umma_smem_bytes(int tile_n, int stages, int staged)
 {
-    return 1024 + stages * (int)stage_bytes((uint32_t)tile_n) + (int)sizeof(SmemTables);
+    return 1024 + stages * (int)stage_bytes((uint32_t)tile_n) + (int)sizeof(SmemTables) +
+           (staged ? EPI_STAGE_BYTES : 0);
 }
 
-int gett_umma_max_stages(int tile_n, int smem_limit)
+int gett_umma_max_stages(int tile_n, int smem_limit, int staged)
 {
-    int s = (smem_limit - 1024 - (int)sizeof(SmemTables)) / (int)stage_bytes((uint32_t)tile_n);
+    int s = (smem_limit - 1024 - (int)sizeof(SmemTables) - (staged ? EPI_STAGE_BYTES : 0)) /
+            (int)stage_bytes((uint32_t)tile_n);
     s = s > MAX_STAGES ? MAX_STAGES : s;
     return s - s % PROD_GROUPS; // a stage must always be served by the same producer group
 }

@@ -246,6 +246,24 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         leadK = find_unit(ik, 1); // ... else B's
     p->tm = order_with_lead(im, leadM);
     p->tn = order_with_lead(in, leadN);
+    {
+        // Sec. 3.2.1: when B's stride-1 mode and C's stride-1 mode are two different
+        // modes of I_n, split B's mode by the width of one 16-byte vector and put C's
+        // mode right after that piece, so that a tile holds vectors of B and runs of C.
+        const int unitCn = find_unit(in, 2);
+        const int64_t vecB = dtype == GETT_F32 ? 4 : 8;
+        if (leadN >= 0 && unitCn >= 0 && unitCn != leadN && in[leadN].ext % vecB == 0 &&
+            in[leadN].ext > vecB && o.epilogue != GETT_EPI_DIRECT && dtype != GETT_F32) {
+            std::vector<GettDigit> t;
+            t.push_back({leadN, vecB, 1});
+            t.push_back({unitCn, in[unitCn].ext, 1});
+            t.push_back({leadN, in[leadN].ext / vecB, vecB});
+            for (int i = 0; i < (int)in.size(); ++i)
+                if (i != leadN && i != unitCn)
+                    t.push_back({i, in[i].ext, 1});
+            p->tn = t;
+        }
+    }
     p->tk = order_with_lead(ik, leadK);
     if ((rc = make_dim(im, p->tm, 0, 2, p->M)) || (rc = make_dim(in, p->tn, 1, 2, p->N)) ||
         (rc = make_dim(ik, p->tk, 0, 1, p->K)))
@@ -290,12 +308,13 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         return GETT_ERR_INVALID_ARG;
     const bool both_vec = info.loader_a != GETT_LOAD_SCALAR && info.loader_b != GETT_LOAD_SCALAR;
     const bool umma_ok = dtype != GETT_F32 && both_vec;
+    const bool ffma_ok = dtype == GETT_F32 && both_vec;
     if (path == GETT_PATH_AUTO)
-        path = umma_ok ? GETT_PATH_UMMA : GETT_PATH_SIMT;
-    if (path == GETT_PATH_UMMA && !umma_ok)
+        path = umma_ok ? GETT_PATH_UMMA : ffma_ok ? GETT_PATH_FFMA : GETT_PATH_SIMT;
+    if ((path == GETT_PATH_UMMA && !umma_ok) || (path == GETT_PATH_FFMA && !ffma_ok))
         return GETT_ERR_UNSUPPORTED;
-    if (path == GETT_PATH_FFMA)
-        return GETT_ERR_UNSUPPORTED;
+    // four consecutive tile rows of C form one aligned 16-byte vector
+    p->c_vec = vec_ok(p->M, false, p->N, false, 4) ? 1 : 0;
     info.path = path;
     p->debug = o.reserved[0];
 
@@ -316,11 +335,61 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.smem_bytes = 0;
         info.epilogue = GETT_EPI_DIRECT;
         info.loader_a = info.loader_b = GETT_LOAD_SCALAR;
-    } else { // GETT_PATH_UMMA
-        if ((o.tile_m && o.tile_m != 128) || (o.tile_k && o.tile_k != 64) ||
+    } else if (path == GETT_PATH_FFMA) {
+        if ((o.tile_m && o.tile_m != 128) || (o.tile_k && o.tile_k != 32) ||
             (o.epilogue && o.epilogue != GETT_EPI_DIRECT))
             return GETT_ERR_UNSUPPORTED;
+        int tn = o.tile_n ? o.tile_n : (p->N.size <= 32 ? 32 : 128);
+        if (tn != 32 && tn != 128)
+            return GETT_ERR_UNSUPPORTED;
+        int st = o.stages ? o.stages : (tn == 128 ? 3 : 4);
+        if (st < 2 || st > 4)
+            return GETT_ERR_UNSUPPORTED;
+        info.tile_m = 128;
+        info.tile_n = tn;
+        info.tile_k = 32;
+        info.stages = st;
+        info.block = 256;
+        info.smem_bytes = gett_ffma_smem_bytes(tn, st);
+        info.epilogue = GETT_EPI_DIRECT;
+    } else { // GETT_PATH_UMMA
+        if ((o.tile_m && o.tile_m != 128) || (o.tile_k && o.tile_k != 64))
+            return GETT_ERR_UNSUPPORTED;
+        // Unpacking (Eq. 11).  Direct stores are already coalesced when C's stride-1
+        // mode leads the M order (a warp's 32 rows are 32 consecutive floats).  When it
+        // is a mode of I_n instead, the accumulator goes through a shared-memory
+        // transpose if four consecutive "slots" are one aligned 16-byte vector of C.
+        auto others_mult4 = [&](int skip_n_digit) {
+            for (int d = 0; d < p->M.ndig; ++d)
+                if (p->M.sY[d] % 4)
+                    return false;
+            for (int d = 0; d < p->N.ndig; ++d)
+                if (d != skip_n_digit && p->N.sY[d] % 4)
+                    return false;
+            return true;
+        };
+        int staged_cv = 0;
+        if (!(p->M.ndig >= 1 && p->M.sY[0] == 1)) {
+            if (p->N.ndig >= 2 && p->N.ext[0] == 8 && p->N.sY[1] == 1 && p->N.ext[1] % 4 == 0 &&
+                others_mult4(1))
+                staged_cv = 8;
+            else if (p->N.ndig >= 1 && p->N.sY[0] == 1 && p->N.ext[0] % 4 == 0 && others_mult4(0))
+                staged_cv = 1;
+        }
+        if (o.epilogue == GETT_EPI_DIRECT)
+            staged_cv = 0;
+        if (o.epilogue == GETT_EPI_STAGED && !staged_cv)
+            return GETT_ERR_UNSUPPORTED;
+        info.epilogue = staged_cv ? GETT_EPI_STAGED : GETT_EPI_DIRECT;
+        if (staged_cv)
+            p->c_vec = staged_cv;
         int tn = o.tile_n;
+        if (tn == 0 && staged_cv == 8) {
+            // one tile = all 8-wide pieces x the whole of C's stride-1 mode, if that is a legal width
+            const uint32_t want = 8 * p->N.ext[1];
+            if (want == 64 || want == 128 || want == 192 || want == 256)
+                tn = (int)want;
+        }
         if (tn == 0) {
             // fewest waves x per-tile cost; ties go to the wider tile
             const uint32_t tm_count = ceil_div(p->M.size, 128);
@@ -339,16 +408,16 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         if (tn != 64 && tn != 128 && tn != 192 && tn != 256)
             return GETT_ERR_UNSUPPORTED;
         const int smem_limit = 227 * 1024;
-        int st = o.stages ? o.stages : gett_umma_max_stages(tn, smem_limit);
-        if (st < 3 || st > gett_umma_max_stages(tn, smem_limit) || st % gett_umma_stage_multiple())
+        const int staged = info.epilogue == GETT_EPI_STAGED;
+        int st = o.stages ? o.stages : gett_umma_max_stages(tn, smem_limit, staged);
+        if (st < 3 || st > gett_umma_max_stages(tn, smem_limit, staged) || st % gett_umma_stage_multiple())
             return GETT_ERR_UNSUPPORTED;
         info.tile_m = 128;
         info.tile_n = tn;
         info.tile_k = 64;
         info.stages = st;
         info.block = gett_umma_block();
-        info.smem_bytes = gett_umma_smem_bytes(tn, st);
-        info.epilogue = GETT_EPI_DIRECT;
+        info.smem_bytes = gett_umma_smem_bytes(tn, st, staged);
     }
     p->tiles_m = ceil_div(p->M.size, (uint32_t)info.tile_m);
     p->tiles_n = ceil_div(p->N.size, (uint32_t)info.tile_n);

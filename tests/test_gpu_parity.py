@@ -37,6 +37,27 @@ def test_reduced_workloads(key, dtype, path):
     parity_case(w.contraction, dtype, w.dist, w.seed, w.alpha, w.beta, repeat=2, path=path)
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("epilogue", [g.GETT_EPI_AUTO, g.GETT_EPI_DIRECT])
+def test_cfg5_shape_with_split_stride_one_mode(dtype, epilogue):
+    """B's stride-1 mode (16) is split into 8-wide pieces around C's stride-1 mode (12):
+    exercises the staged epilogue (16-bit inputs) against the direct one."""
+    w = workload("cfg5", dict(m0=2, m1=16, m2=5, n0=12, n1=3, n2=16, k=72))
+    ratio, info = parity_case(w.contraction, dtype, w.dist, w.seed, w.alpha, w.beta, repeat=2,
+                              epilogue=epilogue)
+    if dtype != F32 and epilogue == g.GETT_EPI_AUTO:
+        assert info.epilogue == g.GETT_EPI_STAGED
+    parity_case(w.contraction, dtype, w.dist, w.seed, -0.5, 0.0, epilogue=epilogue)
+
+
+def test_staged_epilogue_when_columns_already_run_along_c():
+    # B is K-major, C's stride-1 mode is a mode of I_n: slots are the columns themselves
+    con = parse_spec("C[n0,m,n1] = A[m,k] * B[k,n1,n0]", dict(m=136, n0=24, n1=7, k=80))
+    for dtype in (BF16_F32, F16_F32):
+        ratio, info = parity_case(con, dtype, "uniform", 11, 1.0, 1.0, repeat=2)
+        assert info.epilogue == g.GETT_EPI_STAGED and info.path == g.GETT_PATH_UMMA
+
+
 @pytest.mark.parametrize("seed", range(48))
 def test_fuzz_random_contractions(seed):
     rng = np.random.default_rng(5000 + seed)

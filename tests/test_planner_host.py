@@ -140,6 +140,32 @@ def test_split_k_planning():
     assert auto.info.split_k > 1 and auto.info.workspace_bytes == auto.info.split_k * 384 * 376 * 4
     never = g.Plan(con, g.GETT_F32, split_k=1)
     assert never.info.split_k == 1 and never.info.workspace_bytes == 0
-    forced = g.Plan(workload("cfg3").contraction, g.GETT_F32, split_k=2)
-    assert forced.info.split_k == 2
+    forced = g.Plan(workload("cfg4").contraction, g.GETT_F32, split_k=2)
+    assert forced.info.split_k == 2 and forced.info.workspace_bytes == 2 * 5184 * 5184 * 4
+    # cfg3's whole contracted range (24) is a single K slab: it cannot be sliced
+    assert g.Plan(workload("cfg3").contraction, g.GETT_F32, split_k=2).info.split_k == 1
+    assert g.Plan(workload("cfg3").contraction, g.GETT_F32, path=g.GETT_PATH_SIMT,
+                  split_k=2).info.split_k == 2
     assert g.Plan(workload("cfg3").contraction, g.GETT_F32).info.split_k == 1
+
+
+def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
+    want = {  # key, dtype -> (path, loader_a, loader_b, epilogue)
+        ("cfg1", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_K, g.GETT_EPI_DIRECT),
+        ("cfg2", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_K, g.GETT_EPI_DIRECT),
+        ("cfg3", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_K, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_DIRECT),
+        ("cfg4", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_DIRECT),
+        ("cfg5", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_STAGED),
+    }
+    for (key, dtype), exp in want.items():
+        i = g.Plan(workload(key).contraction, dtype).info
+        assert (i.path, i.loader_a, i.loader_b, i.epilogue) == exp, key
+    # cfg5: the tile is all 8-wide pieces of B's stride-1 mode x the whole of C's stride-1 mode
+    i = g.Plan(workload("cfg5").contraction, g.GETT_BF16_F32).info
+    assert (i.tile_m, i.tile_n, i.tile_k) == (128, 192, 64) and i.digits_n == 4
+    # odd extents cannot be gathered in 16-byte vectors: scalar path
+    odd = parse_spec("C[m,n] = A[m,k] * B[k,n]", dict(m=7, n=5, k=3))
+    assert g.Plan(odd, g.GETT_BF16_F32).info.path == g.GETT_PATH_SIMT
+    with pytest.raises(g.GettError) as e:
+        g.Plan(odd, g.GETT_BF16_F32, path=g.GETT_PATH_UMMA)
+    assert e.value.status == 4
