@@ -118,6 +118,7 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     args.epilogue = plan->info.epilogue;
     args.debug = plan->debug;
     args.c_vec = plan->c_vec;
+    args.prod_groups = plan->info.path == GETT_PATH_UMMA ? gett_umma_prod_groups(plan->info.stages) : 0;
 
     int path = plan->info.path;
     // the vectorised kernels need 16-byte aligned operand bases; otherwise gather scalars

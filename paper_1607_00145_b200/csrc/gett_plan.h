@@ -46,6 +46,7 @@ struct GettKernelArgs {
     int32_t c_vec;        // direct epilogue: 1 = four consecutive tile rows are one aligned 16-byte
                           // vector of C; staged epilogue: column-to-slot pattern (1 or 8)
     int32_t debug;        // opts.reserved[0]: experiment switches, 0 in normal use
+    int32_t prod_groups;  // producer groups the tensor-core kernel uses (divides stages)
 };
 
 struct gett_plan {
@@ -75,7 +76,7 @@ gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, si
 int gett_umma_smem_bytes(int tile_n, int stages, int staged);
 int gett_umma_max_stages(int tile_n, int smem_limit, int staged);
 int gett_umma_block();
-int gett_umma_stage_multiple(); // the ring depth must be a multiple of this
+int gett_umma_prod_groups(int stages); // producer groups in use; must divide the ring depth
 
 // Geometry of the fp32 kernel (kernel_ffma.cu).
 int gett_ffma_smem_bytes(int tile_n, int stages);

@@ -51,7 +51,9 @@ constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t ATOM_BYTES = 1024;      // 8 rows x 128 B
 constexpr uint32_t MN_BLOCK_BYTES = 8192;  // one 64-wide block of an MN-major operand: 64 k rows
 constexpr int EPI_PITCH = 68;              // floats per staged row: 64 + 4 keeps 128-bit accesses conflict-free
-constexpr int EPI_STAGE_BYTES = NUM_EPI_WARPS * 32 * EPI_PITCH * 4;
+constexpr int EPI_GROUPS = 256 / 4;          // 16-byte groups per tile row, at most
+constexpr int EPI_WARP_BYTES = 2 * 32 * EPI_PITCH * 4 + 2 * EPI_GROUPS * 8; // two chunk buffers + two group tables
+constexpr int EPI_STAGE_BYTES = NUM_EPI_WARPS * EPI_WARP_BYTES;
 
 constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-byte-unit offset tables
 
@@ -59,7 +61,6 @@ constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-by
 // copies starts on a 16-byte boundary), which keeps them in 32 bits.
 struct alignas(16) SmemTables { // the staging rows that follow it hold 128-bit vectors
     int64_t colC[256];                        // C offset of each tile column (epilogue)
-    int64_t rowCs[TILE_M];                    // C offset of each tile row (staged epilogue)
     uint32_t kTab[PROD_GROUPS][2][TILE_K];    // per producer group: A / B offsets of the slab's k
     uint32_t rowTab[PROD_GROUPS][TILE_M + 256]; // per producer group: row offsets (K-major operands)
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
@@ -197,64 +198,133 @@ __device__ __forceinline__ uint32_t col_of_slot(uint32_t slot)
     return CV == 1 ? slot : (slot >> 3) + ((slot & 7) << 3);
 }
 
-// Thread `lane` of an epilogue warp writes its 32 accumulator columns (half h of the
-// chunk) into its staging row as eight 128-bit stores.
-template <int CV>
-__device__ __forceinline__ void stage_half(float* Srow, uint32_t h, const uint32_t (&v)[32])
+// Staged epilogue, run by each epilogue warp on its own 32 tile rows, one 64-column
+// chunk at a time, software-pipelined one chunk ahead (across tile boundaries):
+//   prepare(c+1): (first chunk of a tile) C offsets of my row and of the tile's 16-byte
+//                 groups; if beta != 0, cp.async the old C values of chunk c+1 into the
+//                 other staging buffer -- the reads of C never wait for the accumulator
+//   process(c)  : accumulator -> registers, alpha*acc + beta*old (old read from staging,
+//                 one row per lane), result written back to staging with 128-bit stores;
+//                 then the warp re-reads staging with lanes running along C and issues
+//                 128-bit global stores
+template <int TILE_N, int CV>
+__device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTables* T, uint8_t* epi_smem,
+                                                uint32_t tmem_base, uint32_t warp, uint32_t lane,
+                                                uint32_t total_work, volatile int* abort_flag)
 {
-#pragma unroll
-    for (int a = 0; a < 8; ++a) {
-        float4 q;
-        if (CV == 1) {
-            q = make_float4(__uint_as_float(v[4 * a]), __uint_as_float(v[4 * a + 1]),
-                            __uint_as_float(v[4 * a + 2]), __uint_as_float(v[4 * a + 3]));
-            *reinterpret_cast<float4*>(Srow + h * 32 + 4 * a) = q;
-        } else {
-            q = make_float4(__uint_as_float(v[a]), __uint_as_float(v[a + 8]), __uint_as_float(v[a + 16]),
-                            __uint_as_float(v[a + 24]));
-            *reinterpret_cast<float4*>(Srow + a * 8 + h * 4) = q;
-        }
-    }
-}
+    constexpr uint32_t NCH = TILE_N / 64;
+    constexpr uint32_t FULL = 0xFFFFFFFFu;
+    float* S = reinterpret_cast<float*>(epi_smem + warp * EPI_WARP_BYTES);
+    int64_t* grp = reinterpret_cast<int64_t*>(S + 2 * 32 * EPI_PITCH);
+    const uint32_t s_u32 = ptx::smem_u32(S);
+    const float alpha = g.alpha, beta = g.beta;
+    const bool rmw = beta != 0.f;
+    const uint32_t ntile = total_work > blockIdx.x ? (total_work - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const uint32_t nchunk = ntile * NCH;
+    long long rowC0 = -1, rowC1 = -1; // C offset of my row in the tiles of even / odd local number
 
-// One 64-column chunk: 32 rows x 16 float4 per warp, lanes running along C.
-template <int CV>
-__device__ __forceinline__ void store_chunk(const float* Sw, float* __restrict__ C, const int64_t* rowCs,
-                                            const int64_t* colC, uint32_t chunk, uint32_t lane,
-                                            float alpha, float beta)
-{
+    auto prepare = [&](uint32_t cj) {
+        if (cj < nchunk) {
+            const uint32_t tl = cj / NCH, ch = cj - tl * NCH;
+            if (ch == 0) {
+                const WorkItem wi = decode_work(g, blockIdx.x + tl * gridDim.x);
+                int64_t rc = -1, dummy;
+                const uint32_t m = wi.m0 + warp * 32 + lane;
+                if (m < g.M.size)
+                    gett_decompose(g.M, m, dummy, rc);
+                if (tl & 1)
+                    rowC1 = rc;
+                else
+                    rowC0 = rc;
+                for (uint32_t e = lane; e < TILE_N / 4; e += 32) {
+                    const uint32_t col = (e >> 4) * 64 + col_of_slot<CV>(4 * (e & 15));
+                    int64_t x, y = -1;
+                    if (wi.n0 + col < g.N.size)
+                        gett_decompose(g.N, wi.n0 + col, x, y);
+                    grp[(tl & 1) * EPI_GROUPS + e] = y;
+                }
+                __syncwarp();
+            }
+            if (rmw) {
+                const long long myrow = (tl & 1) ? rowC1 : rowC0;
+                const uint32_t dst = s_u32 + (cj & 1) * (32 * EPI_PITCH * 4);
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        float4 val[8];
-        float* ptr[8];
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const uint32_t q = lane + 32 * (half * 8 + t);
-            const uint32_t row = q >> 4, s4 = q & 15;
-            val[t] = *reinterpret_cast<const float4*>(Sw + row * EPI_PITCH + 4 * s4);
-            const int64_t rc = rowCs[row];
-            const int64_t cn = colC[chunk * 64 + col_of_slot<CV>(4 * s4)];
-            ptr[t] = (rc >= 0 && cn >= 0) ? C + rc + cn : nullptr;
+                for (int t = 0; t < 16; ++t) {
+                    const uint32_t q = lane + 32 * t, row = q >> 4, s4 = q & 15;
+                    const long long rc = __shfl_sync(FULL, myrow, row);
+                    const int64_t cn = grp[(tl & 1) * EPI_GROUPS + ch * 16 + s4];
+                    const bool ok = rc >= 0 && cn >= 0;
+                    ptx::cp_async_16(dst + (row * EPI_PITCH + 4 * s4) * 4, ok ? g.C + rc + cn : g.C, ok ? 16u : 0u);
+                }
+            }
         }
-        if (beta != 0.f) {
-            float4 old[8];
-#pragma unroll
-            for (int t = 0; t < 8; ++t)
-                old[t] = ptr[t] ? __ldcg(reinterpret_cast<const float4*>(ptr[t])) : make_float4(0, 0, 0, 0);
-#pragma unroll
-            for (int t = 0; t < 8; ++t)
-                if (ptr[t])
-                    *reinterpret_cast<float4*>(ptr[t]) =
-                        make_float4(fmaf(beta, old[t].x, alpha * val[t].x), fmaf(beta, old[t].y, alpha * val[t].y),
-                                    fmaf(beta, old[t].z, alpha * val[t].z), fmaf(beta, old[t].w, alpha * val[t].w));
-        } else {
-#pragma unroll
-            for (int t = 0; t < 8; ++t)
-                if (ptr[t])
-                    *reinterpret_cast<float4*>(ptr[t]) =
-                        make_float4(alpha * val[t].x, alpha * val[t].y, alpha * val[t].z, alpha * val[t].w);
+        ptx::cp_async_commit();
+    };
+
+    prepare(0);
+    for (uint32_t ci = 0; ci < nchunk; ++ci) {
+        prepare(ci + 1);
+        ptx::cp_async_wait<1>(); // chunk ci's old C has landed (my copies) ...
+        __syncwarp();            // ... and everybody else's
+        const uint32_t tl = ci / NCH, ch = ci - tl * NCH, buf = tl & 1;
+        if (ch == 0) {
+            if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), (tl >> 1) & 1, abort_flag))
+                break;
+            ptx::tc_fence_after();
         }
+        float* Sb = S + (ci & 1) * (32 * EPI_PITCH);
+        float* Srow = Sb + lane * EPI_PITCH;
+        const uint32_t taddr = tmem_base + ((warp * 32u) << 16) + buf * 256 + ch * 64;
+#pragma unroll
+        for (uint32_t h = 0; h < 2; ++h) {
+            uint32_t v[32];
+            ptx::tmem_ld_32x32(taddr + h * 32, v);
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int a = 0; a < 8; ++a) {
+                float4 q;
+                float* p;
+                if (CV == 1) {
+                    q = make_float4(__uint_as_float(v[4 * a]), __uint_as_float(v[4 * a + 1]),
+                                    __uint_as_float(v[4 * a + 2]), __uint_as_float(v[4 * a + 3]));
+                    p = Srow + h * 32 + 4 * a;
+                } else {
+                    q = make_float4(__uint_as_float(v[a]), __uint_as_float(v[a + 8]),
+                                    __uint_as_float(v[a + 16]), __uint_as_float(v[a + 24]));
+                    p = Srow + a * 8 + h * 4;
+                }
+                q.x *= alpha;
+                q.y *= alpha;
+                q.z *= alpha;
+                q.w *= alpha;
+                if (rmw) {
+                    const float4 o = *reinterpret_cast<const float4*>(p);
+                    q.x = fmaf(beta, o.x, q.x);
+                    q.y = fmaf(beta, o.y, q.y);
+                    q.z = fmaf(beta, o.z, q.z);
+                    q.w = fmaf(beta, o.w, q.w);
+                }
+                *reinterpret_cast<float4*>(p) = q;
+            }
+        }
+        if (ch == NCH - 1) { // the accumulator buffer can be overwritten by the next-but-one tile
+            ptx::tc_fence_before();
+            ptx::mbar_arrive(ptx::smem_u32(&T->acc_empty[buf]));
+        }
+        __syncwarp();
+        const long long myrow = (tl & 1) ? rowC1 : rowC0;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+            const uint32_t q = lane + 32 * t, row = q >> 4, s4 = q & 15;
+            const long long rc = __shfl_sync(FULL, myrow, row);
+            const int64_t cn = grp[(tl & 1) * EPI_GROUPS + ch * 16 + s4];
+            if (rc >= 0 && cn >= 0)
+                *reinterpret_cast<float4*>(g.C + rc + cn) =
+                    *reinterpret_cast<const float4*>(Sb + row * EPI_PITCH + 4 * s4);
+        }
+        __syncwarp(); // this staging buffer is free for the prefetch two chunks ahead
     }
+    ptx::cp_async_wait_all();
 }
 
 template <bool A_VEC_K, bool B_VEC_K, int TILE_N>
@@ -303,6 +373,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
         // ring depth is a multiple of PROD_GROUPS, hence a stage's barriers are always
         // used by the same group, which therefore observes every one of their phases.
         const uint32_t pg = (warp - PROD_WARP0) / WARPS_PER_GROUP;
+        const uint32_t ng = (uint32_t)g.prod_groups; // groups in use: divides the ring depth
         const uint32_t gl = threadIdx.x - (PROD_WARP0 + pg * WARPS_PER_GROUP) * 32;
         const uint32_t gbar = 3 + pg; // named barrier of this group
         uint32_t* kA = T->kTab[pg][0];
@@ -315,17 +386,17 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
         const char* baseB = static_cast<const char*>(g.B);
         uint32_t first = 0; // slab number of the current work item's first slab
         bool alive = true;
-        for (uint32_t w = blockIdx.x; w < total_work; w += gridDim.x) {
+        for (uint32_t w = blockIdx.x; w < total_work && pg < ng; w += gridDim.x) {
             const WorkItem wi = decode_work(g, w);
-            // my group's first slab in this item: smallest j with (first + j) % PROD_GROUPS == pg
-            uint32_t j = (pg + PROD_GROUPS - first % PROD_GROUPS) % PROD_GROUPS;
+            // my group's first slab in this item: smallest j with (first + j) % ng == pg
+            uint32_t j = (pg + ng - first % ng) % ng;
             if (j < wi.nslab) {
                 ptx::named_barrier(gbar, GROUP_LANES); // the group is done with the previous tables
                 la.setup_tile(g.M, wi.m0, gl, rowA);
                 lb.setup_tile(g.N, wi.n0, gl, rowB);
             }
             const bool tile_full = wi.m0 + TILE_M <= g.M.size && wi.n0 + TILE_N <= g.N.size;
-            for (; j < wi.nslab; j += PROD_GROUPS) {
+            for (; j < wi.nslab; j += ng) {
                 const uint32_t it = first + j;
                 const uint32_t k0 = wi.kbeg + j * TILE_K;
                 ptx::named_barrier(gbar, GROUP_LANES); // previous slab's k table no longer read
@@ -416,7 +487,15 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
         const uint32_t et = threadIdx.x; // 0..127: tile row, = tensor-memory lane
         uint32_t local = 0;
         bool alive = true;
-        for (uint32_t w = blockIdx.x; w < total_work; w += gridDim.x, ++local) {
+        const bool staged = g.epilogue == GETT_EPI_STAGED && g.split_k == 1;
+        if (staged) {
+            uint8_t* epi_smem = smem + stages * sbytes + sizeof(SmemTables);
+            if (g.c_vec == 8)
+                epilogue_staged<TILE_N, 8>(g, T, epi_smem, tmem_base, warp, lane, total_work, abort_flag);
+            else
+                epilogue_staged<TILE_N, 1>(g, T, epi_smem, tmem_base, warp, lane, total_work, abort_flag);
+        }
+        for (uint32_t w = blockIdx.x; w < total_work && !staged; w += gridDim.x, ++local) {
             const WorkItem wi = decode_work(g, w);
             const uint32_t buf = local & 1;
             // C offsets of this tile: my row in a register, the columns in shared memory
@@ -424,7 +503,6 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
             if (wi.m0 + et < g.M.size)
                 gett_decompose(g.M, wi.m0 + et, dummy, rowC);
             ptx::named_barrier(2, NUM_EPI_WARPS * 32); // previous tile's column table no longer read
-            T->rowCs[et] = rowC;
             for (uint32_t c = et; c < TILE_N; c += NUM_EPI_WARPS * 32) {
                 int64_t x, y = -1;
                 if (wi.n0 + c < g.N.size)
@@ -440,31 +518,6 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
             const uint32_t taddr = tmem_base + ((warp * 32u) << 16) + buf * 256;
             const bool row_ok = rowC >= 0;
             const float alpha = g.alpha, beta = g.beta;
-            if (g.epilogue == GETT_EPI_STAGED && g.split_k == 1 && !(g.debug & 2)) {
-                float* Sw = reinterpret_cast<float*>(smem + stages * sbytes + sizeof(SmemTables)) +
-                            warp * 32 * EPI_PITCH;
-                for (uint32_t chunk = 0; chunk < TILE_N / 64; ++chunk) {
-#pragma unroll
-                    for (uint32_t h = 0; h < 2; ++h) {
-                        uint32_t v[32];
-                        ptx::tmem_ld_32x32(taddr + chunk * 64 + h * 32, v);
-                        ptx::tmem_wait_ld();
-                        if (g.c_vec == 8)
-                            stage_half<8>(Sw + lane * EPI_PITCH, h, v);
-                        else
-                            stage_half<1>(Sw + lane * EPI_PITCH, h, v);
-                    }
-                    __syncwarp();
-                    if (g.c_vec == 8)
-                        store_chunk<8>(Sw, g.C, T->rowCs + warp * 32, T->colC, chunk, lane, alpha, beta);
-                    else
-                        store_chunk<1>(Sw, g.C, T->rowCs + warp * 32, T->colC, chunk, lane, alpha, beta);
-                    __syncwarp(); // the staging rows are free again
-                }
-                ptx::tc_fence_before();
-                ptx::mbar_arrive(ptx::smem_u32(&T->acc_empty[buf]));
-                continue;
-            }
             for (uint32_t c0 = 0; c0 < TILE_N; c0 += 16) {
                 uint32_t v[16];
                 ptx::tmem_ld_32x16(taddr + c0, v);
@@ -529,12 +582,12 @@ int gett_umma_max_stages(int tile_n, int smem_limit, int staged)
     int s = (smem_limit - 1024 - (int)sizeof(SmemTables) - (staged ? EPI_STAGE_BYTES : 0)) /
             (int)stage_bytes((uint32_t)tile_n);
     s = s > MAX_STAGES ? MAX_STAGES : s;
-    return s - s % PROD_GROUPS; // a stage must always be served by the same producer group
+    return s >= PROD_GROUPS ? s - s % PROD_GROUPS : s; // a stage is always served by the same group
 }
 
 int gett_umma_block() { return NUM_THREADS; }
 
-int gett_umma_stage_multiple() { return PROD_GROUPS; }
+int gett_umma_prod_groups(int stages) { return stages >= PROD_GROUPS ? PROD_GROUPS : stages; }
 
 template <bool AK, bool BK>
 static cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
