@@ -31,7 +31,8 @@ namespace {
 constexpr int TILE_M = 128;
 constexpr int TILE_K = 64;           // 16-bit elements per slab = one 128-byte swizzle row
 constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;
-constexpr int NUM_EPI_WARPS = 4;
+constexpr int NUM_EPI_WARPS = 8;           // two sets of four: set s takes the CTA's tiles number s, s+2, ...
+constexpr int EPI_SET_THREADS = 128;
 #ifndef GETT_PROD_GROUPS
 #define GETT_PROD_GROUPS 4
 #endif
@@ -52,7 +53,8 @@ constexpr uint32_t ATOM_BYTES = 1024;      // 8 rows x 128 B
 constexpr uint32_t MN_BLOCK_BYTES = 8192;  // one 64-wide block of an MN-major operand: 64 k rows
 constexpr int EPI_PITCH = 68;              // floats per staged row: 64 + 4 keeps 128-bit accesses conflict-free
 constexpr int EPI_GROUPS = 256 / 4;          // 16-byte groups per tile row, at most
-constexpr int EPI_WARP_BYTES = 2 * 32 * EPI_PITCH * 4 + 2 * EPI_GROUPS * 8; // two chunk buffers + two group tables
+constexpr int EPI_DEPTH = 2;                 // staging buffers per warp: old C is fetched EPI_DEPTH-1 chunks ahead
+constexpr int EPI_WARP_BYTES = EPI_DEPTH * (32 * EPI_PITCH * 4 + EPI_GROUPS * 8); // chunk buffers + group tables
 constexpr int EPI_STAGE_BYTES = NUM_EPI_WARPS * EPI_WARP_BYTES;
 
 constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-byte-unit offset tables
@@ -60,7 +62,7 @@ constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-by
 // Offsets in the producer tables are in units of 16 bytes (every vector a producer
 // copies starts on a 16-byte boundary), which keeps them in 32 bits.
 struct alignas(16) SmemTables { // the staging rows that follow it hold 128-bit vectors
-    int64_t colC[256];                        // C offset of each tile column (epilogue)
+    int64_t colC[2][256];                     // per epilogue set: C offset of each tile column
     uint32_t kTab[PROD_GROUPS][2][TILE_K];    // per producer group: A / B offsets of the slab's k
     uint32_t rowTab[PROD_GROUPS][TILE_M + 256]; // per producer group: row offsets (K-major operands)
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
@@ -215,44 +217,47 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
     constexpr uint32_t NCH = TILE_N / 64;
     constexpr uint32_t FULL = 0xFFFFFFFFu;
     float* S = reinterpret_cast<float*>(epi_smem + warp * EPI_WARP_BYTES);
-    int64_t* grp = reinterpret_cast<int64_t*>(S + 2 * 32 * EPI_PITCH);
+    int64_t* grp = reinterpret_cast<int64_t*>(S + EPI_DEPTH * 32 * EPI_PITCH);
     const uint32_t s_u32 = ptx::smem_u32(S);
     const float alpha = g.alpha, beta = g.beta;
     const bool rmw = beta != 0.f;
-    const uint32_t ntile = total_work > blockIdx.x ? (total_work - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    // this warp's set handles the CTA's tiles with local number es, es + 2, ...; `j` counts them
+    const uint32_t es = warp >> 2, eq = warp & 3;
+    const uint32_t ncta = total_work > blockIdx.x ? (total_work - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const uint32_t ntile = ncta > es ? (ncta - es + 1) / 2 : 0;
     const uint32_t nchunk = ntile * NCH;
-    long long rowC0 = -1, rowC1 = -1; // C offset of my row in the tiles of even / odd local number
+    static_assert(EPI_DEPTH == 2, "row offsets are kept in two scalars");
+    long long rowC_0 = -1, rowC_1 = -1; // C offset of my row, for j even / odd
+    auto my_row = [&](uint32_t j) { return (j & 1) ? rowC_1 : rowC_0; };
 
     auto prepare = [&](uint32_t cj) {
         if (cj < nchunk) {
-            const uint32_t tl = cj / NCH, ch = cj - tl * NCH;
+            const uint32_t j = cj / NCH, ch = cj - j * NCH;
             if (ch == 0) {
-                const WorkItem wi = decode_work(g, blockIdx.x + tl * gridDim.x);
+                const WorkItem wi = decode_work(g, blockIdx.x + (es + 2 * j) * gridDim.x);
                 int64_t rc = -1, dummy;
-                const uint32_t m = wi.m0 + warp * 32 + lane;
+                const uint32_t m = wi.m0 + eq * 32 + lane;
                 if (m < g.M.size)
                     gett_decompose(g.M, m, dummy, rc);
-                if (tl & 1)
-                    rowC1 = rc;
-                else
-                    rowC0 = rc;
+                rowC_0 = (j & 1) ? rowC_0 : rc;
+                rowC_1 = (j & 1) ? rc : rowC_1;
                 for (uint32_t e = lane; e < TILE_N / 4; e += 32) {
                     const uint32_t col = (e >> 4) * 64 + col_of_slot<CV>(4 * (e & 15));
                     int64_t x, y = -1;
                     if (wi.n0 + col < g.N.size)
                         gett_decompose(g.N, wi.n0 + col, x, y);
-                    grp[(tl & 1) * EPI_GROUPS + e] = y;
+                    grp[(j & 1) * EPI_GROUPS + e] = y;
                 }
                 __syncwarp();
             }
             if (rmw) {
-                const long long myrow = (tl & 1) ? rowC1 : rowC0;
+                const long long myrow = my_row(j);
                 const uint32_t dst = s_u32 + (cj & 1) * (32 * EPI_PITCH * 4);
 #pragma unroll
                 for (int t = 0; t < 16; ++t) {
                     const uint32_t q = lane + 32 * t, row = q >> 4, s4 = q & 15;
                     const long long rc = __shfl_sync(FULL, myrow, row);
-                    const int64_t cn = grp[(tl & 1) * EPI_GROUPS + ch * 16 + s4];
+                    const int64_t cn = grp[(j & 1) * EPI_GROUPS + ch * 16 + s4];
                     const bool ok = rc >= 0 && cn >= 0;
                     ptx::cp_async_16(dst + (row * EPI_PITCH + 4 * s4) * 4, ok ? g.C + rc + cn : g.C, ok ? 16u : 0u);
                 }
@@ -266,15 +271,15 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
         prepare(ci + 1);
         ptx::cp_async_wait<1>(); // chunk ci's old C has landed (my copies) ...
         __syncwarp();            // ... and everybody else's
-        const uint32_t tl = ci / NCH, ch = ci - tl * NCH, buf = tl & 1;
+        const uint32_t j = ci / NCH, ch = ci - j * NCH, buf = es; // tile es + 2j uses accumulator es
         if (ch == 0) {
-            if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), (tl >> 1) & 1, abort_flag))
+            if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag))
                 break;
             ptx::tc_fence_after();
         }
         float* Sb = S + (ci & 1) * (32 * EPI_PITCH);
         float* Srow = Sb + lane * EPI_PITCH;
-        const uint32_t taddr = tmem_base + ((warp * 32u) << 16) + buf * 256 + ch * 64;
+        const uint32_t taddr = tmem_base + ((eq * 32u) << 16) + buf * 256 + ch * 64;
 #pragma unroll
         for (uint32_t h = 0; h < 2; ++h) {
             uint32_t v[32];
@@ -307,22 +312,22 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
                 *reinterpret_cast<float4*>(p) = q;
             }
         }
-        if (ch == NCH - 1) { // the accumulator buffer can be overwritten by the next-but-one tile
+        if (ch == NCH - 1) { // the accumulator buffer can be overwritten by the set's next tile
             ptx::tc_fence_before();
             ptx::mbar_arrive(ptx::smem_u32(&T->acc_empty[buf]));
         }
         __syncwarp();
-        const long long myrow = (tl & 1) ? rowC1 : rowC0;
+        const long long myrow = my_row(j);
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
             const uint32_t q = lane + 32 * t, row = q >> 4, s4 = q & 15;
             const long long rc = __shfl_sync(FULL, myrow, row);
-            const int64_t cn = grp[(tl & 1) * EPI_GROUPS + ch * 16 + s4];
+            const int64_t cn = grp[(j & 1) * EPI_GROUPS + ch * 16 + s4];
             if (rc >= 0 && cn >= 0)
                 *reinterpret_cast<float4*>(g.C + rc + cn) =
                     *reinterpret_cast<const float4*>(Sb + row * EPI_PITCH + 4 * s4);
         }
-        __syncwarp(); // this staging buffer is free for the prefetch two chunks ahead
+        __syncwarp(); // this staging buffer is free for the next prefetch into it
     }
     ptx::cp_async_wait_all();
 }
@@ -352,7 +357,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(ptx::smem_u32(&T->acc_full[b]), 1);
-            ptx::mbar_init(ptx::smem_u32(&T->acc_empty[b]), NUM_EPI_WARPS * 32);
+            ptx::mbar_init(ptx::smem_u32(&T->acc_empty[b]), EPI_SET_THREADS);
         }
         T->abort_flag = 0;
         ptx::fence_mbar_init();
@@ -484,8 +489,11 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
         __syncwarp();
     } else {
         // ------------------------------- epilogue ------------------------------
-        const uint32_t et = threadIdx.x; // 0..127: tile row, = tensor-memory lane
-        uint32_t local = 0;
+        // Epilogue set es = warp / 4 takes the CTA's tiles number es, es + 2, ... (exactly
+        // the tiles whose accumulator lives in buffer es); warp % 4 selects the 32
+        // tensor-memory lanes (= tile rows) a warp may read.
+        const uint32_t es = warp >> 2, eq = warp & 3;
+        const uint32_t et = eq * 32 + lane; // tile row
         bool alive = true;
         const bool staged = g.epilogue == GETT_EPI_STAGED && g.split_k == 1;
         if (staged) {
@@ -495,27 +503,29 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
             else
                 epilogue_staged<TILE_N, 1>(g, T, epi_smem, tmem_base, warp, lane, total_work, abort_flag);
         }
-        for (uint32_t w = blockIdx.x; w < total_work && !staged; w += gridDim.x, ++local) {
+        int64_t* colC = T->colC[es];
+        uint32_t j = 0; // counts this set's tiles
+        for (uint32_t w = blockIdx.x + es * gridDim.x; w < total_work && !staged; w += 2 * gridDim.x, ++j) {
             const WorkItem wi = decode_work(g, w);
-            const uint32_t buf = local & 1;
+            const uint32_t buf = es;
             // C offsets of this tile: my row in a register, the columns in shared memory
             int64_t rowC = -1, dummy;
             if (wi.m0 + et < g.M.size)
                 gett_decompose(g.M, wi.m0 + et, dummy, rowC);
-            ptx::named_barrier(2, NUM_EPI_WARPS * 32); // previous tile's column table no longer read
-            for (uint32_t c = et; c < TILE_N; c += NUM_EPI_WARPS * 32) {
+            ptx::named_barrier(1 + es, EPI_SET_THREADS); // previous tile's column table no longer read
+            for (uint32_t c = et; c < TILE_N; c += EPI_SET_THREADS) {
                 int64_t x, y = -1;
                 if (wi.n0 + c < g.N.size)
                     gett_decompose(g.N, wi.n0 + c, x, y);
-                T->colC[c] = y;
+                colC[c] = y;
             }
-            ptx::named_barrier(2, NUM_EPI_WARPS * 32);
-            if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), (local >> 1) & 1, abort_flag))
+            ptx::named_barrier(1 + es, EPI_SET_THREADS);
+            if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag))
                 alive = false;
             if (!alive)
                 continue; // keep the named barriers above matched, do nothing else
             ptx::tc_fence_after();
-            const uint32_t taddr = tmem_base + ((warp * 32u) << 16) + buf * 256;
+            const uint32_t taddr = tmem_base + ((eq * 32u) << 16) + buf * 256;
             const bool row_ok = rowC >= 0;
             const float alpha = g.alpha, beta = g.beta;
             for (uint32_t c0 = 0; c0 < TILE_N; c0 += 16) {
@@ -535,7 +545,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
                     int64_t co[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
-                        co[i] = T->colC[c0 + i];
+                        co[i] = colC[c0 + i];
                     if (beta != 0.f) {
                         // all reads of the old C first, so their latencies overlap
                         float old[16];

@@ -410,7 +410,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         const int smem_limit = 227 * 1024;
         const int staged = info.epilogue == GETT_EPI_STAGED;
         int st = o.stages ? o.stages : gett_umma_max_stages(tn, smem_limit, staged);
-        if (st < 2 || st > gett_umma_max_stages(tn, smem_limit, staged) || st % gett_umma_prod_groups(st))
+        if (st < 1 || st > gett_umma_max_stages(tn, smem_limit, staged) || st % gett_umma_prod_groups(st))
             return GETT_ERR_UNSUPPORTED;
         info.tile_m = 128;
         info.tile_n = tn;
