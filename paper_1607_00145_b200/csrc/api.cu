@@ -137,7 +137,8 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
         break;
     }
     case GETT_PATH_FFMA:
-        err = gett_launch_ffma(args, plan->info.grid, plan->info.smem_bytes, stream);
+        err = plan->skinny ? gett_launch_ffma_skinny(args, plan->info.grid, plan->info.smem_bytes, stream)
+                           : gett_launch_ffma(args, plan->info.grid, plan->info.smem_bytes, stream);
         break;
     case GETT_PATH_UMMA:
         err = gett_launch_umma(args, plan->info.grid, plan->info.smem_bytes, stream);

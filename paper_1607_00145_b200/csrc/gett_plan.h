@@ -59,6 +59,7 @@ struct gett_plan {
     uint32_t tiles_m, tiles_n, k_per_split;
     int32_t a_kmajor, b_kmajor;
     int32_t c_vec;
+    int32_t skinny; // fp32: B resident in shared memory, A streamed (small N and K)
     // device side
     float* ws;
     int32_t* status;
@@ -80,3 +81,8 @@ int gett_umma_prod_groups(int stages); // producer groups in use; must divide th
 
 // Geometry of the fp32 kernel (kernel_ffma.cu).
 int gett_ffma_smem_bytes(int tile_n, int stages);
+
+// fp32 kernel for N <= 32, K <= gett_ffma_skinny_max_k(), A K-major (kernel_ffma_skinny.cu).
+int gett_ffma_skinny_smem_bytes(int N, int K);
+int gett_ffma_skinny_rows();
+int gett_ffma_skinny_max_k();

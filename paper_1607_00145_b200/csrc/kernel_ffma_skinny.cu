@@ -1,0 +1,196 @@
+// Strict-fp32 kernel for the bandwidth-bound "tensor times small matrix" regime:
+// N <= 32, K <= 64, A staged K-major (its stride-1 mode is contracted).
+//
+// The whole of B (K x N) stays in shared memory for the life of the CTA, so the
+// loop nest of Listing 4 degenerates to the m-loop alone: persistent CTAs stream
+// 256-row tiles of A through a cp.async ring (packing, Eq. 9), every thread holds a
+// 4-row x CPT-column register tile (micro-kernel, Sec. 3.1), and C is written once
+// with 32 consecutive rows per warp store (Eq. 11).  Nothing but A is read from HBM
+// and nothing but C is written, which is the compulsory traffic.
+#include "kernels.h"
+#include "ptx_sm100.cuh"
+
+namespace {
+
+constexpr int ROWS = 256, NT = 256, KMAX = 64, STAGES = 3;
+// Row tables are alive from the moment they are filled (one iteration before the tile's
+// copy is issued) until the tile's epilogue: STAGES + 1 tiles at any time.
+constexpr int TSLOTS = STAGES + 1;
+constexpr uint32_t INVALID16 = 0xFFFFFFFFu;
+
+struct SkinnyTables {
+    int64_t offCM[TSLOTS][ROWS]; // C offset of each tile row (-1 beyond M)
+    uint32_t rowA[TSLOTS][ROWS]; // A offset of each tile row, 16-byte units
+    int64_t offCN[32];
+    uint32_t kA[KMAX / 4];       // A offset of each 4-wide k piece, 16-byte units
+};
+
+// Row pitch (floats) of an A tile: a multiple of 4 whose quarter is odd, so that the
+// 128-bit reads of eight consecutive rows fall into eight different bank groups.
+__host__ __device__ constexpr uint32_t skinny_pitch(uint32_t K) { return K + (K % 8 == 0 ? 4 : 8); }
+
+template <int CPT>
+__global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_constant__ GettKernelArgs g)
+{
+    constexpr int NP = 4 * CPT; // padded row of B in shared memory
+    extern __shared__ __align__(16) uint8_t smem[];
+    const uint32_t K = g.K.size, N = g.N.size, Msz = g.M.size;
+    const uint32_t KC = K / 4;
+    const uint32_t pitch = skinny_pitch(K);
+    const uint32_t tile_bytes = ROWS * pitch * 4;
+    float* Bs = reinterpret_cast<float*>(smem);                       // [K][NP]
+    uint8_t* ring = smem + K * NP * 4;
+    SkinnyTables* T = reinterpret_cast<SkinnyTables*>(ring + STAGES * tile_bytes);
+    const uint32_t ring_u32 = ptx::smem_u32(ring);
+    const int tid = threadIdx.x;
+    const uint32_t ntiles = g.tiles_m;
+
+    // ---- B and the tile-independent tables, once ----
+    for (uint32_t i = tid; i < K * NP; i += NT) {
+        const uint32_t k = i / NP, n = i - k * NP;
+        float v = 0.f;
+        if (n < N) {
+            int64_t bn, cn, ak, bk;
+            gett_decompose(g.N, n, bn, cn);
+            gett_decompose(g.K, k, ak, bk);
+            v = __ldg(static_cast<const float*>(g.B) + bn + bk);
+        }
+        Bs[i] = v;
+    }
+    if (tid < 32) {
+        int64_t bn, cn = -1;
+        if ((uint32_t)tid < N)
+            gett_decompose(g.N, tid, bn, cn);
+        T->offCN[tid] = cn;
+    }
+    if ((uint32_t)tid < KC) {
+        int64_t ak, bk;
+        gett_decompose(g.K, tid * 4, ak, bk);
+        T->kA[tid] = (uint32_t)(ak >> 2);
+    }
+    auto fill_rows = [&](uint32_t it) { // tables of the `it`-th tile of this CTA
+        const uint32_t t = blockIdx.x + it * gridDim.x;
+        const uint32_t m = t * ROWS + tid;
+        int64_t x = 0, y = -1;
+        const bool ok = t < ntiles && m < Msz;
+        if (ok)
+            gett_decompose(g.M, m, x, y);
+        T->rowA[it % TSLOTS][tid] = ok ? (uint32_t)(x >> 2) : INVALID16;
+        T->offCM[it % TSLOTS][tid] = y;
+    };
+    auto issue = [&](uint32_t it) {
+        const uint32_t t = blockIdx.x + it * gridDim.x;
+        if (t < ntiles) {
+            const uint32_t dst = ring_u32 + (it % STAGES) * tile_bytes;
+            const uint32_t* rowA = T->rowA[it % TSLOTS];
+            for (uint32_t q = tid; q < ROWS * KC; q += NT) {
+                const uint32_t row = q / KC, kc = q - row * KC;
+                const uint32_t r16 = rowA[row];
+                const bool ok = r16 != INVALID16;
+                ptx::cp_async_16(dst + (row * pitch + kc * 4) * 4,
+                                 static_cast<const char*>(g.A) + (ok ? ((uint64_t)(r16 + T->kA[kc]) << 4) : 0),
+                                 ok ? 16u : 0u);
+            }
+        }
+        ptx::cp_async_commit();
+    };
+
+    for (uint32_t s = 0; s < STAGES - 1; ++s) {
+        fill_rows(s);
+        __syncthreads();
+        issue(s);
+    }
+    fill_rows(STAGES - 1);
+
+    const uint32_t q = tid & 63, cg = tid >> 6;
+    const float alpha = g.alpha, beta = g.beta;
+    for (uint32_t it = 0; blockIdx.x + it * gridDim.x < ntiles; ++it) {
+        ptx::cp_async_wait<STAGES - 2>();
+        __syncthreads(); // tile `it` visible; stage of tile it-1 free; tables for it+STAGES-1 ready
+        issue(it + STAGES - 1);
+        fill_rows(it + STAGES); // read by the issue of the next iteration
+        const float* As = reinterpret_cast<const float*>(ring + (it % STAGES) * tile_bytes);
+        float acc[4][CPT];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < CPT; ++j)
+                acc[i][j] = 0.f;
+#pragma unroll 2
+        for (uint32_t kc = 0; kc < KC; ++kc) {
+            float4 a[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                a[i] = *reinterpret_cast<const float4*>(As + (q + 64 * i) * pitch + kc * 4);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                float b[CPT];
+                const float* brow = Bs + (kc * 4 + kk) * NP + cg * CPT;
+#pragma unroll
+                for (int j = 0; j < CPT; j += 2) {
+                    const float2 v = *reinterpret_cast<const float2*>(brow + j);
+                    b[j] = v.x;
+                    b[j + 1] = v.y;
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float av = kk == 0 ? a[i].x : kk == 1 ? a[i].y : kk == 2 ? a[i].z : a[i].w;
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j)
+                        acc[i][j] = fmaf(av, b[j], acc[i][j]);
+                }
+            }
+        }
+        const int64_t* offCM = T->offCM[it % TSLOTS];
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) {
+            const int64_t cn = T->offCN[cg * CPT + j];
+            if (cn < 0)
+                continue;
+            float old[4];
+            int64_t cm[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                cm[i] = offCM[q + 64 * i];
+                old[i] = (beta != 0.f && cm[i] >= 0) ? __ldcg(g.C + cm[i] + cn) : 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (cm[i] >= 0)
+                    g.C[cm[i] + cn] = fmaf(beta, old[i], alpha * acc[i][j]);
+        }
+    }
+    ptx::cp_async_wait_all();
+}
+
+} // namespace
+
+static int skinny_cpt(uint32_t N) { return (int)((N + 3) / 4 + 1) & ~1; } // even, 4 * cpt >= N
+
+int gett_ffma_skinny_smem_bytes(int N, int K)
+{
+    return K * 4 * skinny_cpt((uint32_t)N) * 4 + STAGES * ROWS * (int)skinny_pitch((uint32_t)K) * 4 +
+           (int)sizeof(SkinnyTables);
+}
+
+int gett_ffma_skinny_max_k() { return KMAX; }
+
+int gett_ffma_skinny_rows() { return ROWS; }
+
+cudaError_t gett_launch_ffma_skinny(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
+{
+    const int cpt = skinny_cpt(args.N.size);
+    void (*k)(GettKernelArgs);
+    switch (cpt) {
+    case 2: k = gett_ffma_skinny_kernel<2>; break;
+    case 4: k = gett_ffma_skinny_kernel<4>; break;
+    case 6: k = gett_ffma_skinny_kernel<6>; break;
+    case 8: k = gett_ffma_skinny_kernel<8>; break;
+    default: return cudaErrorInvalidValue;
+    }
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess)
+        return e;
+    k<<<grid, NT, smem, stream>>>(args);
+    return cudaGetLastError();
+}

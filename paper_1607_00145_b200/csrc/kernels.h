@@ -16,3 +16,6 @@ cudaError_t gett_launch_umma(const GettKernelArgs& args, int grid, int smem, cud
 
 // Strict-fp32 kernel: 16-byte gathers, register-blocked FFMA.  grid = tiles * split_k.
 cudaError_t gett_launch_ffma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream);
+
+// fp32, small N and K: B resident in shared memory, persistent CTAs stream A.
+cudaError_t gett_launch_ffma_skinny(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream);

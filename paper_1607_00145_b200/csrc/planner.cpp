@@ -308,7 +308,13 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         return GETT_ERR_INVALID_ARG;
     const bool both_vec = info.loader_a != GETT_LOAD_SCALAR && info.loader_b != GETT_LOAD_SCALAR;
     const bool umma_ok = dtype != GETT_F32 && both_vec;
-    const bool ffma_ok = dtype == GETT_F32 && both_vec;
+    // fp32 with small N and K and a K-major A: B is read once element by element, so
+    // only A has to be gatherable in 16-byte vectors
+    const bool skinny_ok = dtype == GETT_F32 && info.loader_a == GETT_LOAD_VEC_K && p->N.size <= 32 &&
+                           p->K.size <= (uint32_t)gett_ffma_skinny_max_k() && o.split_k <= 1 &&
+                           (o.tile_m == 0 || o.tile_m == gett_ffma_skinny_rows()) && o.tile_n == 0 &&
+                           o.tile_k == 0 && o.stages == 0 && o.epilogue != GETT_EPI_STAGED;
+    const bool ffma_ok = dtype == GETT_F32 && (both_vec || skinny_ok);
     if (path == GETT_PATH_AUTO)
         path = umma_ok ? GETT_PATH_UMMA : ffma_ok ? GETT_PATH_FFMA : GETT_PATH_SIMT;
     if ((path == GETT_PATH_UMMA && !umma_ok) || (path == GETT_PATH_FFMA && !ffma_ok))
@@ -317,6 +323,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     p->c_vec = vec_ok(p->M, false, p->N, false, 4) ? 1 : 0;
     info.path = path;
     p->debug = o.reserved[0];
+    p->skinny = 0;
 
     // ---- blocking (Sec. 3.3) ----
     if (o.tile_m < 0 || o.tile_n < 0 || o.tile_k < 0 || o.stages < 0 || o.split_k < 0)
@@ -335,6 +342,17 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.smem_bytes = 0;
         info.epilogue = GETT_EPI_DIRECT;
         info.loader_a = info.loader_b = GETT_LOAD_SCALAR;
+    } else if (path == GETT_PATH_FFMA && skinny_ok) {
+        // tensor times small matrix: B stays in shared memory, A is streamed once
+        p->skinny = 1;
+        info.tile_m = gett_ffma_skinny_rows();
+        info.tile_n = 32;
+        info.tile_k = (int)p->K.size;
+        info.stages = 3;
+        info.block = 256;
+        info.smem_bytes = gett_ffma_skinny_smem_bytes((int)p->N.size, (int)p->K.size);
+        info.epilogue = GETT_EPI_DIRECT;
+        info.loader_b = GETT_LOAD_SCALAR; // B is read once, element by element
     } else if (path == GETT_PATH_FFMA) {
         if ((o.tile_m && o.tile_m != 128) || (o.tile_k && o.tile_k != 32) ||
             (o.epilogue && o.epilogue != GETT_EPI_DIRECT))
@@ -445,6 +463,8 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     info.grid = (int32_t)(tiles * split);
     if (path == GETT_PATH_UMMA) // persistent: one CTA per SM walks the work list
         info.grid = (int32_t)std::min<uint64_t>(tiles * split, (uint64_t)sms);
+    if (p->skinny) // persistent: two CTAs per SM stream the row tiles
+        info.grid = (int32_t)std::min<uint64_t>(p->tiles_m, 2ull * sms);
     return GETT_OK;
 }
 

@@ -58,6 +58,20 @@ def test_staged_epilogue_when_columns_already_run_along_c():
         assert info.epilogue == g.GETT_EPI_STAGED and info.path == g.GETT_PATH_UMMA
 
 
+@pytest.mark.parametrize("sizes", [dict(m0=40, m1=33, n0=24, k=24), dict(m0=300, m1=7, n0=5, k=12),
+                                   dict(m0=64, m1=9, n0=32, k=64), dict(m0=17, m1=3, n0=1, k=4)])
+def test_tensor_times_small_matrix_kernel(sizes):
+    """cfg3's shape family: B resident in shared memory, A streamed (fp32 only)."""
+    w = workload("cfg3", sizes)
+    for alpha, beta in [(1.0, 0.0), (0.5, 2.0)]:
+        ratio, info = parity_case(w.contraction, F32, w.dist, w.seed, alpha, beta, repeat=2)
+        assert info.path == g.GETT_PATH_FFMA and info.tile_m == 256
+    # the same contraction through the general fp32 kernel, where B can be vector-gathered too
+    if sizes["n0"] % 4 == 0:
+        ratio, info = parity_case(w.contraction, F32, w.dist, w.seed, 1.0, 1.0, tile_m=128)
+        assert info.tile_m == 128
+
+
 @pytest.mark.parametrize("seed", range(48))
 def test_fuzz_random_contractions(seed):
     rng = np.random.default_rng(5000 + seed)

@@ -153,7 +153,8 @@ def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
     want = {  # key, dtype -> (path, loader_a, loader_b, epilogue)
         ("cfg1", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_K, g.GETT_EPI_DIRECT),
         ("cfg2", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_K, g.GETT_EPI_DIRECT),
-        ("cfg3", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_K, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_DIRECT),
+        # cfg3: small N and K -> B is read once into shared memory, element by element
+        ("cfg3", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_K, g.GETT_LOAD_SCALAR, g.GETT_EPI_DIRECT),
         ("cfg4", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_DIRECT),
         ("cfg5", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_STAGED),
     }
