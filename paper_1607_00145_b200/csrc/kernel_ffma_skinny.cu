@@ -13,14 +13,14 @@
 namespace {
 
 constexpr int ROWS = 256, NT = 256, KMAX = 64, STAGES = 3;
+constexpr int QL = NT / 4;      // threads per column group
+constexpr int RPT = ROWS / QL;  // rows per thread: q, q + QL, ...
 // Row tables are alive from the moment they are filled (one iteration before the tile's
 // copy is issued) until the tile's epilogue: STAGES + 1 tiles at any time.
 constexpr int TSLOTS = STAGES + 1;
-constexpr uint32_t INVALID16 = 0xFFFFFFFFu;
 
 struct SkinnyTables {
     int64_t offCM[TSLOTS][ROWS]; // C offset of each tile row (-1 beyond M)
-    uint32_t rowA[TSLOTS][ROWS]; // A offset of each tile row, 16-byte units
     int64_t offCN[32];
     uint32_t kA[KMAX / 4];       // A offset of each 4-wide k piece, 16-byte units
 };
@@ -68,72 +68,78 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
         gett_decompose(g.K, tid * 4, ak, bk);
         T->kA[tid] = (uint32_t)(ak >> 2);
     }
-    auto fill_rows = [&](uint32_t it) { // tables of the `it`-th tile of this CTA
-        const uint32_t t = blockIdx.x + it * gridDim.x;
-        const uint32_t m = t * ROWS + tid;
-        int64_t x = 0, y = -1;
-        const bool ok = t < ntiles && m < Msz;
-        if (ok)
-            gett_decompose(g.M, m, x, y);
-        T->rowA[it % TSLOTS][tid] = ok ? (uint32_t)(x >> 2) : INVALID16;
-        T->offCM[it % TSLOTS][tid] = y;
-    };
+    // Thread `tid` owns rows tid and tid + NT of every tile: it computes their offsets,
+    // copies their K/4 pieces, and publishes their C offsets for whoever accumulates them.
     auto issue = [&](uint32_t it) {
         const uint32_t t = blockIdx.x + it * gridDim.x;
         if (t < ntiles) {
-            const uint32_t dst = ring_u32 + (it % STAGES) * tile_bytes;
-            const uint32_t* rowA = T->rowA[it % TSLOTS];
-            for (uint32_t q = tid; q < ROWS * KC; q += NT) {
-                const uint32_t row = q / KC, kc = q - row * KC;
-                const uint32_t r16 = rowA[row];
-                const bool ok = r16 != INVALID16;
-                ptx::cp_async_16(dst + (row * pitch + kc * 4) * 4,
-                                 static_cast<const char*>(g.A) + (ok ? ((uint64_t)(r16 + T->kA[kc]) << 4) : 0),
-                                 ok ? 16u : 0u);
+#pragma unroll
+            for (int h = 0; h < ROWS / NT; ++h) {
+                const uint32_t row = tid + h * NT;
+                const uint32_t m = t * ROWS + row;
+                int64_t x = 0, y = -1;
+                const bool ok = m < Msz;
+                if (ok)
+                    gett_decompose(g.M, m, x, y);
+                T->offCM[it % TSLOTS][row] = y;
+                const char* src = static_cast<const char*>(g.A) + (ok ? x * 4 : 0);
+                const uint32_t dst = ring_u32 + (it % STAGES) * tile_bytes + row * pitch * 4;
+#pragma unroll 2
+                for (uint32_t kc = 0; kc < KC; ++kc)
+                    ptx::cp_async_16(dst + kc * 16, src + (ok ? ((uint64_t)T->kA[kc] << 4) : 0), ok ? 16u : 0u);
             }
         }
         ptx::cp_async_commit();
     };
 
-    for (uint32_t s = 0; s < STAGES - 1; ++s) {
-        fill_rows(s);
-        __syncthreads();
+    __syncthreads(); // kA ready
+    for (uint32_t s = 0; s < STAGES - 1; ++s)
         issue(s);
-    }
-    fill_rows(STAGES - 1);
 
-    const uint32_t q = tid & 63, cg = tid >> 6;
+    const uint32_t q = tid % QL, cg = tid / QL; // rows q + QL i; a warp shares one column group
     const float alpha = g.alpha, beta = g.beta;
+    int64_t cn[CPT]; // C offsets of my columns (the same for every tile)
+#pragma unroll
+    for (int j = 0; j < CPT; ++j)
+        cn[j] = T->offCN[cg * CPT + j];
     for (uint32_t it = 0; blockIdx.x + it * gridDim.x < ntiles; ++it) {
         ptx::cp_async_wait<STAGES - 2>();
-        __syncthreads(); // tile `it` visible; stage of tile it-1 free; tables for it+STAGES-1 ready
+        __syncthreads(); // tile `it` and its row table visible; the stage of tile it-1 is free
         issue(it + STAGES - 1);
-        fill_rows(it + STAGES); // read by the issue of the next iteration
         const float* As = reinterpret_cast<const float*>(ring + (it % STAGES) * tile_bytes);
-        float acc[4][CPT];
+        float acc[RPT][CPT];
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < RPT; ++i)
 #pragma unroll
             for (int j = 0; j < CPT; ++j)
                 acc[i][j] = 0.f;
 #pragma unroll 2
         for (uint32_t kc = 0; kc < KC; ++kc) {
-            float4 a[4];
+            float4 a[RPT];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                a[i] = *reinterpret_cast<const float4*>(As + (q + 64 * i) * pitch + kc * 4);
+            for (int i = 0; i < RPT; ++i)
+                a[i] = *reinterpret_cast<const float4*>(As + (q + QL * i) * pitch + kc * 4);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
                 float b[CPT];
                 const float* brow = Bs + (kc * 4 + kk) * NP + cg * CPT;
+                // cg * CPT * 4 bytes is 16-byte aligned when CPT % 4 == 0, else 8-byte aligned
 #pragma unroll
                 for (int j = 0; j < CPT; j += 2) {
-                    const float2 v = *reinterpret_cast<const float2*>(brow + j);
-                    b[j] = v.x;
-                    b[j + 1] = v.y;
+                    if (CPT % 4 == 0 && j % 4 == 0) {
+                        const float4 v = *reinterpret_cast<const float4*>(brow + j);
+                        b[j] = v.x;
+                        b[j + 1] = v.y;
+                        b[j + 2] = v.z;
+                        b[j + 3] = v.w;
+                    } else if (CPT % 4 != 0) {
+                        const float2 v = *reinterpret_cast<const float2*>(brow + j);
+                        b[j] = v.x;
+                        b[j + 1] = v.y;
+                    }
                 }
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < RPT; ++i) {
                     const float av = kk == 0 ? a[i].x : kk == 1 ? a[i].y : kk == 2 ? a[i].z : a[i].w;
 #pragma unroll
                     for (int j = 0; j < CPT; ++j)
@@ -143,21 +149,19 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
         }
         const int64_t* offCM = T->offCM[it % TSLOTS];
 #pragma unroll
-        for (int j = 0; j < CPT; ++j) {
-            const int64_t cn = T->offCN[cg * CPT + j];
-            if (cn < 0)
+        for (int i = 0; i < RPT; ++i) {
+            const int64_t cm = offCM[q + QL * i];
+            if (cm < 0)
                 continue;
-            float old[4];
-            int64_t cm[4];
+            float* crow = g.C + cm;
+            float old[CPT];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                cm[i] = offCM[q + 64 * i];
-                old[i] = (beta != 0.f && cm[i] >= 0) ? __ldcg(g.C + cm[i] + cn) : 0.f;
-            }
+            for (int j = 0; j < CPT; ++j)
+                old[j] = (beta != 0.f && cn[j] >= 0) ? __ldcg(crow + cn[j]) : 0.f;
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (cm[i] >= 0)
-                    g.C[cm[i] + cn] = fmaf(beta, old[i], alpha * acc[i][j]);
+            for (int j = 0; j < CPT; ++j)
+                if (cn[j] >= 0)
+                    crow[cn[j]] = fmaf(beta, old[j], alpha * acc[i][j]);
         }
     }
     ptx::cp_async_wait_all();
