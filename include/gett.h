@@ -197,6 +197,44 @@ GETT_API gett_status_t gett_plan_get_table(const gett_plan_t* plan, int which, i
  */
 GETT_API gett_status_t gett_plan_last_device_status(const gett_plan_t* plan);
 
+/*
+ * gett_contract_noalloc -- the same contraction for callers that cannot allocate
+ * device memory.  (The paper has no counterpart: it is an addition of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree are not allowed or not
+ * wanted -- while a stream is being captured, under an allocator that has claimed
+ * the whole device, inside a latency-critical loop, or in a host callback.  The
+ * plan-based calls above allocate a status word and, for split-K plans, a workspace
+ * when the plan is created.  This call creates no plan object on the device and
+ * calls no allocating routine at all: the contraction runs through the scalar-gather
+ * kernel with the contracted range cut into `split_k` slices, and the slices'
+ * partial sums are kept in an array of GETT_NOALLOC_WORKSPACE_BYTES that is built
+ * into the library image (each GPU that loads the library holds that array until
+ * the process exits).
+ *
+ *   A, B, C   : host descriptors, as for gett_plan_create (read during the call only).
+ *   split_k   : 0 = let the planner choose, 1 = no slicing, s > 1 = s slices.
+ *   A_data, B_data, C_data : device pointers, as for gett_contract.
+ *   cuda_stream : cudaStream_t as void*, NULL = default stream.  Asynchronous.
+ *
+ * Limit: split_k * M * N * 4 bytes must not exceed GETT_NOALLOC_WORKSPACE_BYTES,
+ * otherwise GETT_ERR_UNSUPPORTED is returned and nothing is launched.  Other errors
+ * as for gett_plan_create / gett_contract.
+ *
+ * The first call on each device looks up the device address of the built-in array
+ * (with that device current); make that first call outside any stream capture.
+ * All calls share the one array, and it keeps the previous call's partial sums:
+ * every call overwrites exactly the entries it later reads, so nothing has to be
+ * cleared, but two calls whose kernels overlap on the GPU (different streams) race
+ * on it -- order them on one stream or with events.
+ */
+#define GETT_NOALLOC_WORKSPACE_BYTES (16u << 20)
+GETT_API gett_status_t gett_contract_noalloc(const gett_tensor_desc_t* A, const gett_tensor_desc_t* B,
+                                    const gett_tensor_desc_t* C, gett_dtype_t dtype,
+                                    int32_t split_k, float alpha, const void* A_data,
+                                    const void* B_data, float beta, void* C_data,
+                                    void* cuda_stream);
+
 /* Human-readable name of a status; never NULL. */
 GETT_API const char* gett_status_string(gett_status_t status);
 

@@ -89,6 +89,11 @@ def _load() -> ctypes.CDLL:
                                         ctypes.c_size_t]
     lib.gett_plan_last_device_status.restype = ctypes.c_int
     lib.gett_plan_last_device_status.argtypes = [ctypes.c_void_p]
+    dp2 = ctypes.POINTER(_Desc)
+    lib.gett_contract_noalloc.restype = ctypes.c_int
+    lib.gett_contract_noalloc.argtypes = [dp2, dp2, dp2, ctypes.c_int, ctypes.c_int32, ctypes.c_float,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float,
+                                          ctypes.c_void_p, ctypes.c_void_p]
     lib.gett_status_string.restype = ctypes.c_char_p
     lib.gett_status_string.argtypes = [ctypes.c_int]
     return lib
@@ -147,6 +152,28 @@ def gett_contract(plan: int, alpha: float, A, B, beta: float, C, stream=None) ->
                             ctypes.c_void_p(int(stream)))
     if rc:
         raise GettError(rc, "gett_contract")
+
+
+GETT_NOALLOC_WORKSPACE_BYTES = 16 << 20
+
+
+def gett_contract_noalloc(A, B, C, dtype: int, split_k: int, alpha: float, A_data, B_data,
+                          beta: float, C_data, stream=None) -> None:
+    """The contraction without any device allocation (no plan): descriptors in, launch out.
+    split_k * M * N * 4 bytes must fit GETT_NOALLOC_WORKSPACE_BYTES."""
+    da, ka = _desc(A.labels, A.extents, A.strides)
+    db, kb = _desc(B.labels, B.extents, B.strides)
+    dc, kc = _desc(C.labels, C.extents, C.strides)
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    elif hasattr(stream, "cuda_stream"):
+        stream = stream.cuda_stream
+    rc = _lib.gett_contract_noalloc(ctypes.byref(da), ctypes.byref(db), ctypes.byref(dc), int(dtype),
+                                    int(split_k), float(alpha), _ptr(A_data), _ptr(B_data),
+                                    float(beta), _ptr(C_data), ctypes.c_void_p(int(stream)))
+    if rc:
+        raise GettError(rc, "gett_contract_noalloc")
 
 
 def gett_plan_destroy(plan: Optional[int]) -> None:
