@@ -79,7 +79,9 @@ typedef enum {
 typedef enum {
     GETT_LOAD_SCALAR = 0, /* element-wise gather                                           */
     GETT_LOAD_VEC_FREE = 1, /* 16-byte vectors along the operand's free (M or N) dimension */
-    GETT_LOAD_VEC_K = 2     /* 16-byte vectors along the contracted dimension              */
+    GETT_LOAD_VEC_K = 2,    /* 16-byte vectors along the contracted dimension              */
+    GETT_LOAD_TMA_FREE = 3, /* tensor-map (TMA) boxes, operand's stride-1 mode is free      */
+    GETT_LOAD_TMA_K = 4     /* tensor-map (TMA) boxes, operand's stride-1 mode is contracted */
 } gett_loader_t;
 
 typedef enum {

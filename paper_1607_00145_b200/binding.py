@@ -11,6 +11,7 @@ GETT_MAX_MODES = 12
 GETT_F32, GETT_BF16_F32, GETT_F16_F32 = 0, 1, 2
 GETT_PATH_AUTO, GETT_PATH_SIMT, GETT_PATH_FFMA, GETT_PATH_UMMA = 0, 1, 2, 3
 GETT_LOAD_SCALAR, GETT_LOAD_VEC_FREE, GETT_LOAD_VEC_K = 0, 1, 2
+GETT_LOAD_TMA_FREE, GETT_LOAD_TMA_K = 3, 4
 GETT_EPI_AUTO, GETT_EPI_DIRECT, GETT_EPI_STAGED = 0, 1, 2
 TABLE_NAMES = ("A_M", "A_K", "B_N", "B_K", "C_M", "C_N")
 
@@ -211,7 +212,10 @@ class Plan:
         if opts:
             o = PlanOpts()
             for k, v in opts.items():
-                setattr(o, k, int(v))
+                if k == "reserved0":  # experiment switches (0 in normal use)
+                    o.reserved[0] = int(v)
+                else:
+                    setattr(o, k, int(v))
         self.handle = gett_plan_create(con.A, con.B, con.C, dtype, o)
         self.info = gett_plan_get_info(self.handle)
 

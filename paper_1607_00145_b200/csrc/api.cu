@@ -1,8 +1,10 @@
 // C ABI of the library (declared in include/gett.h): plan life cycle, kernel
 // dispatch, introspection.  Device memory is touched only here (split-K
 // workspace and the status word); gett_contract itself allocates nothing.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstring>
 #include <new>
 
 #include "kernels.h"
@@ -25,6 +27,57 @@ int current_device_sm_count(int* device_out)
     }
     *device_out = dev;
     return sms;
+}
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup, so the library
+// does not link against the driver and still loads on a machine without one.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            p = nullptr;
+        }
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// Tensor map of one operand for this call's base pointer.  False = use the gather loader.
+bool encode_map(const GettTmaRecipe& R, int dtype, const void* base, uint64_t* out_map)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!R.enabled || !fn)
+        return false;
+    cuuint64_t dims[5], strides_bytes[4];
+    cuuint32_t box[5], estr[5];
+    for (int i = 0; i < R.rank; ++i) {
+        dims[i] = R.dims[i];
+        box[i] = R.box[i];
+        estr[i] = 1;
+        if (i > 0)
+            strides_bytes[i - 1] = R.strides[i] * 2;
+    }
+    const CUtensorMapDataType dt = dtype == GETT_BF16_F32 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                                          : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    CUresult rc = fn(reinterpret_cast<CUtensorMap*>(out_map), dt, (cuuint32_t)R.rank, const_cast<void*>(base),
+                     dims, strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS;
+}
+
+int vec_kind(int loader) // the staging layout behind a loader value
+{
+    return loader == GETT_LOAD_TMA_FREE ? GETT_LOAD_VEC_FREE : loader == GETT_LOAD_TMA_K ? GETT_LOAD_VEC_K : loader;
 }
 
 } // namespace
@@ -111,8 +164,8 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     args.dtype = plan->dtype;
     args.a_kmajor = plan->a_kmajor;
     args.b_kmajor = plan->b_kmajor;
-    args.loader_a = plan->info.loader_a;
-    args.loader_b = plan->info.loader_b;
+    args.loader_a = vec_kind(plan->info.loader_a);
+    args.loader_b = vec_kind(plan->info.loader_b);
     args.tile_n = plan->info.tile_n;
     args.stages = plan->info.stages;
     args.epilogue = plan->info.epilogue;
@@ -140,9 +193,22 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
         err = plan->skinny ? gett_launch_ffma_skinny(args, plan->info.grid, plan->info.smem_bytes, stream)
                            : gett_launch_ffma(args, plan->info.grid, plan->info.smem_bytes, stream);
         break;
-    case GETT_PATH_UMMA:
-        err = gett_launch_umma(args, plan->info.grid, plan->info.smem_bytes, stream);
+    case GETT_PATH_UMMA: {
+        alignas(64) GettTmaMaps maps;
+        memset(&maps, 0, sizeof maps);
+        maps.use_a = encode_map(plan->tma_a, plan->dtype, A, maps.map_a) ? 1 : 0;
+        maps.use_b = encode_map(plan->tma_b, plan->dtype, B, maps.map_b) ? 1 : 0;
+        maps.rank_a = plan->tma_a.rank;
+        maps.rank_b = plan->tma_b.rank;
+        for (int i = 0; i < 5; ++i) {
+            maps.which_a[i] = plan->tma_a.which[i];
+            maps.digit_a[i] = plan->tma_a.digit[i];
+            maps.which_b[i] = plan->tma_b.which[i];
+            maps.digit_b[i] = plan->tma_b.digit[i];
+        }
+        err = gett_launch_umma(args, maps, plan->info.grid, plan->info.smem_bytes, stream);
         break;
+    }
     default: return GETT_ERR_UNSUPPORTED;
     }
     if (err == cudaSuccess && args.split_k > 1)

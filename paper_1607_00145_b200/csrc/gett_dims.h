@@ -64,6 +64,18 @@ GETT_HD void gett_decompose(const GettDim& D, uint32_t idx, int64_t& oX, int64_t
     oY = y;
 }
 
+// Per-digit indices of fused index `idx` (first `n` digits are written).
+GETT_HD void gett_digit_indices(const GettDim& D, uint32_t idx, int32_t* out, int n)
+{
+    uint32_t rem = idx;
+#pragma unroll 1
+    for (int d = 0; d < D.ndig && d < n; ++d) {
+        uint32_t q = gett_fastdiv(rem, D.mul[d], D.sh[d]);
+        out[d] = (int32_t)(rem - q * D.ext[d]);
+        rem = q;
+    }
+}
+
 #if !defined(__CUDA_ARCH__)
 // Host only: magic numbers such that floor(n / d) == mulhi(n, mul) >> sh for all n < 2^31.
 inline void gett_magic(uint32_t d, uint32_t& mul, uint32_t& sh)

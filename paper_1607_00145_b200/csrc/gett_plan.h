@@ -49,6 +49,28 @@ struct GettKernelArgs {
     int32_t prod_groups;  // producer groups the tensor-core kernel uses (divides stages)
 };
 
+// Recipe for one operand's TMA tensor map: dimension i of the map follows digit
+// digit[i] of the operand's free dimension (which[i] == 0) or of K (which[i] == 1).
+// Dimension 0 is the operand's stride-1 digit.  A tile is one box (K-major staging)
+// or rows/64 boxes of 64 free indices (MN-major staging).
+struct GettTmaRecipe {
+    int32_t enabled;
+    int32_t rank;
+    uint64_t dims[5];
+    uint64_t strides[5]; // elements; strides[0] == 1
+    uint32_t box[5];
+    int8_t which[5], digit[5];
+};
+
+// What the tensor-core kernel receives besides GettKernelArgs when an operand is
+// loaded through TMA.  `map` is an opaque CUtensorMap (128 bytes, 64-byte aligned).
+struct alignas(64) GettTmaMaps {
+    uint64_t map_a[16];
+    uint64_t map_b[16];
+    int32_t use_a, use_b, rank_a, rank_b;
+    int8_t which_a[5], digit_a[5], which_b[5], digit_b[5];
+};
+
 struct gett_plan {
     int32_t dtype;
     std::vector<GettMode> im, in, ik; // canonical order (what get_info reports)
@@ -60,6 +82,7 @@ struct gett_plan {
     int32_t a_kmajor, b_kmajor;
     int32_t c_vec;
     int32_t skinny; // fp32: B resident in shared memory, A streamed (small N and K)
+    GettTmaRecipe tma_a, tma_b;
     // device side
     float* ws;
     int32_t* status;

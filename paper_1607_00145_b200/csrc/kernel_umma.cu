@@ -334,7 +334,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
 
 template <bool A_VEC_K, bool B_VEC_K, int TILE_N>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
+gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant__ GettTmaMaps tm)
 {
     extern __shared__ uint8_t smem_raw[];
     // stage ring first (1024-byte aligned for the 128-byte swizzle), tables after it
@@ -389,6 +389,11 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
         OperandLoader<B_VEC_K, TILE_N> lb;
         const char* baseA = static_cast<const char*>(g.A);
         const char* baseB = static_cast<const char*>(g.B);
+        // An operand whose tile is a box of a <= 5-D tensor map is fetched by TMA: thread 0
+        // of the group issues the copies and the stage's barrier counts their bytes.
+        const bool tmaA = tm.use_a != 0, tmaB = tm.use_b != 0, all_tma = tmaA && tmaB;
+        const uint32_t tma_bytes = (tmaA ? A_STAGE_BYTES : 0) + (tmaB ? TILE_N * TILE_K * 2 : 0);
+        int32_t fa[5] = {0, 0, 0, 0, 0}, fb[5] = {0, 0, 0, 0, 0}; // digit indices of the tile origin
         uint32_t first = 0; // slab number of the current work item's first slab
         bool alive = true;
         for (uint32_t w = blockIdx.x; w < total_work && pg < ng; w += gridDim.x) {
@@ -396,28 +401,37 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
             // my group's first slab in this item: smallest j with (first + j) % ng == pg
             uint32_t j = (pg + ng - first % ng) % ng;
             if (j < wi.nslab) {
-                ptx::named_barrier(gbar, GROUP_LANES); // the group is done with the previous tables
-                la.setup_tile(g.M, wi.m0, gl, rowA);
-                lb.setup_tile(g.N, wi.n0, gl, rowB);
+                if (!all_tma)
+                    ptx::named_barrier(gbar, GROUP_LANES); // the group is done with the previous tables
+                if (!tmaA)
+                    la.setup_tile(g.M, wi.m0, gl, rowA);
+                else if (gl == 0)
+                    gett_digit_indices(g.M, wi.m0, fa, 5);
+                if (!tmaB)
+                    lb.setup_tile(g.N, wi.n0, gl, rowB);
+                else if (gl == 0)
+                    gett_digit_indices(g.N, wi.n0, fb, 5);
             }
             const bool tile_full = wi.m0 + TILE_M <= g.M.size && wi.n0 + TILE_N <= g.N.size;
             for (; j < wi.nslab; j += ng) {
                 const uint32_t it = first + j;
                 const uint32_t k0 = wi.kbeg + j * TILE_K;
-                ptx::named_barrier(gbar, GROUP_LANES); // previous slab's k table no longer read
-                if (!(g.debug & 16) && gl < TILE_K) {
-                    const uint32_t k = k0 + gl;
-                    uint32_t xa = INVALID16, xb = INVALID16;
-                    if (k < wi.kend) {
-                        int64_t x, y;
-                        gett_decompose(g.K, k, x, y);
-                        xa = (uint32_t)(x >> 3);
-                        xb = (uint32_t)(y >> 3);
+                if (!all_tma) {
+                    ptx::named_barrier(gbar, GROUP_LANES); // previous slab's k table no longer read
+                    if (!(g.debug & 16) && gl < TILE_K) {
+                        const uint32_t k = k0 + gl;
+                        uint32_t xa = INVALID16, xb = INVALID16;
+                        if (k < wi.kend) {
+                            int64_t x, y;
+                            gett_decompose(g.K, k, x, y);
+                            xa = (uint32_t)(x >> 3);
+                            xb = (uint32_t)(y >> 3);
+                        }
+                        kA[gl] = xa;
+                        kB[gl] = xb;
                     }
-                    kA[gl] = xa;
-                    kB[gl] = xb;
+                    ptx::named_barrier(gbar, GROUP_LANES); // tables (rows and k) complete
                 }
-                ptx::named_barrier(gbar, GROUP_LANES); // tables (rows and k) complete
                 const uint32_t s = it % stages;
                 // After a timeout a thread keeps walking the loop (so its group's named
                 // barriers stay matched) but neither waits nor copies any more.
@@ -426,17 +440,56 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g)
                 if (!alive)
                     continue;
                 const uint32_t sa = stage0 + s * sbytes;
+                const uint32_t fullbar = ptx::smem_u32(&T->full[s]);
+                if (gl == 0 && tma_bytes && !(g.debug & 4)) {
+                    int32_t kd[5] = {0, 0, 0, 0, 0}, c[5];
+                    gett_digit_indices(g.K, k0, kd, 5);
+                    ptx::mbar_expect_tx(fullbar, tma_bytes);
+                    if (tmaA) {
+#pragma unroll
+                        for (int i = 0; i < 5; ++i)
+                            c[i] = tm.which_a[i] ? kd[tm.digit_a[i]] : fa[tm.digit_a[i]];
+                        if (A_VEC_K) {
+                            ptx::tma_load(sa, tm.map_a, fullbar, tm.rank_a, c);
+                        } else {
+#pragma unroll
+                            for (int b = 0; b < TILE_M / 64; ++b) {
+                                ptx::tma_load(sa + b * MN_BLOCK_BYTES, tm.map_a, fullbar, tm.rank_a, c);
+                                c[0] += 64;
+                            }
+                        }
+                    }
+                    if (tmaB) {
+#pragma unroll
+                        for (int i = 0; i < 5; ++i)
+                            c[i] = tm.which_b[i] ? kd[tm.digit_b[i]] : fb[tm.digit_b[i]];
+                        if (B_VEC_K) {
+                            ptx::tma_load(sa + A_STAGE_BYTES, tm.map_b, fullbar, tm.rank_b, c);
+                        } else {
+#pragma unroll
+                            for (int b = 0; b < TILE_N / 64; ++b) {
+                                ptx::tma_load(sa + A_STAGE_BYTES + b * MN_BLOCK_BYTES, tm.map_b, fullbar,
+                                              tm.rank_b, c);
+                                c[0] += 64;
+                            }
+                        }
+                    }
+                }
                 if (g.debug & 4) {
                     // experiment switch: no copies at all (measures the rest of the pipeline)
                 } else if (tile_full && k0 + TILE_K <= wi.kend) {
-                    la.template load_slab<true>(baseA, sa, kA, rowA, gl);
-                    lb.template load_slab<true>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+                    if (!tmaA)
+                        la.template load_slab<true>(baseA, sa, kA, rowA, gl);
+                    if (!tmaB)
+                        lb.template load_slab<true>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
                 } else {
-                    la.template load_slab<false>(baseA, sa, kA, rowA, gl);
-                    lb.template load_slab<false>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+                    if (!tmaA)
+                        la.template load_slab<false>(baseA, sa, kA, rowA, gl);
+                    if (!tmaB)
+                        lb.template load_slab<false>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
                 }
                 // full[s] hears from this thread when its copies for the slab have landed
-                ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&T->full[s]));
+                ptx::cp_async_mbar_arrive_noinc(fullbar);
             }
             first += wi.nslab;
         }
@@ -600,9 +653,10 @@ int gett_umma_block() { return NUM_THREADS; }
 int gett_umma_prod_groups(int stages) { return stages >= PROD_GROUPS ? PROD_GROUPS : stages; }
 
 template <bool AK, bool BK>
-static cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
+static cudaError_t launch_tn(const GettKernelArgs& args, const GettTmaMaps& maps, int grid, int smem,
+                             cudaStream_t stream)
 {
-    void (*k)(GettKernelArgs);
+    void (*k)(GettKernelArgs, GettTmaMaps);
     switch (args.tile_n) {
     case 64: k = gett_umma_kernel<AK, BK, 64>; break;
     case 128: k = gett_umma_kernel<AK, BK, 128>; break;
@@ -613,18 +667,19 @@ static cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cud
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess)
         return e;
-    k<<<grid, NUM_THREADS, smem, stream>>>(args);
+    k<<<grid, NUM_THREADS, smem, stream>>>(args, maps);
     return cudaGetLastError();
 }
 
-cudaError_t gett_launch_umma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
+cudaError_t gett_launch_umma(const GettKernelArgs& args, const GettTmaMaps& maps, int grid, int smem,
+                             cudaStream_t stream)
 {
     const bool ak = args.loader_a == GETT_LOAD_VEC_K, bk = args.loader_b == GETT_LOAD_VEC_K;
     if (ak && bk)
-        return launch_tn<true, true>(args, grid, smem, stream);
+        return launch_tn<true, true>(args, maps, grid, smem, stream);
     if (ak)
-        return launch_tn<true, false>(args, grid, smem, stream);
+        return launch_tn<true, false>(args, maps, grid, smem, stream);
     if (bk)
-        return launch_tn<false, true>(args, grid, smem, stream);
-    return launch_tn<false, false>(args, grid, smem, stream);
+        return launch_tn<false, true>(args, maps, grid, smem, stream);
+    return launch_tn<false, false>(args, maps, grid, smem, stream);
 }

@@ -12,7 +12,8 @@ cudaError_t gett_launch_splitk_reduce(const GettKernelArgs& args, int sm_count,
                                       cudaStream_t stream);
 
 // Tensor-core kernel (16-bit inputs, tcgen05 + tensor memory), persistent grid.
-cudaError_t gett_launch_umma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream);
+cudaError_t gett_launch_umma(const GettKernelArgs& args, const GettTmaMaps& maps, int grid, int smem,
+                             cudaStream_t stream);
 
 // Strict-fp32 kernel: 16-byte gathers, register-blocked FFMA.  grid = tiles * split_k.
 cudaError_t gett_launch_ffma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream);

@@ -158,6 +158,52 @@ int64_t min_stride(const std::vector<GettMode>& modes, int which)
 
 uint32_t ceil_div(uint32_t a, uint32_t b) { return (a + b - 1) / b; }
 
+// Tensor-map recipe for one operand of the tensor-core kernel, if its tile (rows free
+// indices x 64 k) is a box: the tile must stay inside digit 0 of the free dimension and
+// of K (one digit only, or a digit-0 extent that the tile size divides), and the free and
+// K digits together must fit the five dimensions a tensor map has.
+void make_tma_recipe(const GettDim& F, bool fX, const GettDim& Kd, bool kX, int loader, uint32_t rows,
+                     GettTmaRecipe& R)
+{
+    memset(&R, 0, sizeof R);
+    if (loader != GETT_LOAD_VEC_FREE && loader != GETT_LOAD_VEC_K)
+        return;
+    if (F.ndig < 1 || Kd.ndig < 1 || F.ndig + Kd.ndig > 5)
+        return;
+    if (F.ndig > 1 && F.ext[0] % rows != 0)
+        return;
+    if (Kd.ndig > 1 && Kd.ext[0] % 64 != 0)
+        return;
+    const int64_t* fs = fX ? F.sX : F.sY;
+    const int64_t* ks = kX ? Kd.sX : Kd.sY;
+    int n = 0;
+    auto push = [&](int which, int d) {
+        const GettDim& D = which ? Kd : F;
+        R.dims[n] = D.ext[d];
+        R.strides[n] = (uint64_t)(which ? ks[d] : fs[d]);
+        R.which[n] = (int8_t)which;
+        R.digit[n] = (int8_t)d;
+        R.box[n] = 1;
+        ++n;
+    };
+    const bool free_inner = loader == GETT_LOAD_VEC_FREE;
+    push(free_inner ? 0 : 1, 0);
+    push(free_inner ? 1 : 0, 0);
+    for (int d = 1; d < F.ndig; ++d)
+        push(0, d);
+    for (int d = 1; d < Kd.ndig; ++d)
+        push(1, d);
+    R.rank = n;
+    R.box[0] = 64;                      // 128 bytes = the swizzle span
+    R.box[1] = free_inner ? 64 : rows;  // MN-major: 64 k rows per box; K-major: all rows in one box
+    if (R.strides[0] != 1)
+        return;
+    for (int i = 1; i < n; ++i)
+        if (R.strides[i] % 8 != 0 || R.strides[i] >= (1ull << 38))
+            return;
+    R.enabled = 1;
+}
+
 // 16-byte vectors of `vec` elements along the first digit of `lead` are legal for
 // carrier X when that digit is stride-1, its extent is a multiple of vec, and every
 // other stride of the tensor (remaining digits of `lead`, all digits of `other`)
@@ -324,6 +370,8 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     info.path = path;
     p->debug = o.reserved[0];
     p->skinny = 0;
+    memset(&p->tma_a, 0, sizeof p->tma_a);
+    memset(&p->tma_b, 0, sizeof p->tma_b);
 
     // ---- blocking (Sec. 3.3) ----
     if (o.tile_m < 0 || o.tile_n < 0 || o.tile_k < 0 || o.stages < 0 || o.split_k < 0)
@@ -436,6 +484,14 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.stages = st;
         info.block = gett_umma_block();
         info.smem_bytes = gett_umma_smem_bytes(tn, st, staged);
+        if (!(p->debug & 32)) { // (debug & 32: experiment switch, gather even where TMA applies)
+            make_tma_recipe(p->M, true, p->K, true, info.loader_a, 128, p->tma_a);
+            make_tma_recipe(p->N, true, p->K, false, info.loader_b, (uint32_t)tn, p->tma_b);
+            if (p->tma_a.enabled)
+                info.loader_a = info.loader_a == GETT_LOAD_VEC_FREE ? GETT_LOAD_TMA_FREE : GETT_LOAD_TMA_K;
+            if (p->tma_b.enabled)
+                info.loader_b = info.loader_b == GETT_LOAD_VEC_FREE ? GETT_LOAD_TMA_FREE : GETT_LOAD_TMA_K;
+        }
     }
     p->tiles_m = ceil_div(p->M.size, (uint32_t)info.tile_m);
     p->tiles_n = ceil_div(p->N.size, (uint32_t)info.tile_n);

@@ -91,6 +91,42 @@ __device__ __forceinline__ void fence_proxy_async_smem()
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// ---- TMA (bulk tensor copies, no multicast) ----
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// One box of a tiled tensor map -> shared memory; `bar` receives the byte count.
+// c[0] is the innermost coordinate (must be a multiple of 16 bytes' worth of elements).
+__device__ __forceinline__ void tma_load(uint32_t dst, const void* map, uint32_t bar, int rank, const int32_t* c)
+{
+    switch (rank) {
+    case 2:
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+                     "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst), "l"(map), "r"(c[0]), "r"(c[1]), "r"(bar)
+                     : "memory");
+        break;
+    case 3:
+        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+                     "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst), "l"(map), "r"(c[0]), "r"(c[1]), "r"(c[2]),
+                     "r"(bar)
+                     : "memory");
+        break;
+    case 4:
+        asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+                     "[%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst), "l"(map), "r"(c[0]), "r"(c[1]),
+                     "r"(c[2]), "r"(c[3]), "r"(bar)
+                     : "memory");
+        break;
+    default:
+        asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+                     "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(dst), "l"(map), "r"(c[0]), "r"(c[1]),
+                     "r"(c[2]), "r"(c[3]), "r"(c[4]), "r"(bar)
+                     : "memory");
+        break;
+    }
+}
+
 __device__ __forceinline__ void named_barrier(uint32_t id, uint32_t nthreads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");

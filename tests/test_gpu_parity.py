@@ -58,6 +58,28 @@ def test_staged_epilogue_when_columns_already_run_along_c():
         assert info.epilogue == g.GETT_EPI_STAGED and info.path == g.GETT_PATH_UMMA
 
 
+@pytest.mark.parametrize("spec,sizes", [
+    ("C[m,n] = A[m,k] * B[k,n]", dict(m=392, n=264, k=200)),                      # 2-D maps, ragged M, N, K
+    ("C[m,n] = A[k,m] * B[n,k]", dict(m=256, n=320, k=136)),                      # K-major A, N-major B
+    ("C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]",
+     dict(m0=128, m1=3, n0=2, n1=128, k0=64, k1=3)),                              # 4-D maps
+    ("C[m0,m1,n0,n1] = A[k0,m0,k1,m1] * B[k0,k1,n0,n1]",
+     dict(m0=256, m1=2, n0=128, n1=3, k0=64, k1=2)),                              # K-major, 4-D maps
+])
+def test_tma_loader_against_gather_loader_and_oracle(spec, sizes):
+    """Tiles that are boxes of a tensor map go through TMA; the same plan with the
+    gather loader (experiment switch 32) must give the same C, and both the oracle's."""
+    con = parse_spec(spec, sizes)
+    for dtype in (BF16_F32, F16_F32):
+        ratio, info = parity_case(con, dtype, "normal", 21, 1.0, 0.5, repeat=2)
+        assert info.path == g.GETT_PATH_UMMA
+        assert info.loader_a in (g.GETT_LOAD_TMA_FREE, g.GETT_LOAD_TMA_K)
+        assert info.loader_b in (g.GETT_LOAD_TMA_FREE, g.GETT_LOAD_TMA_K)
+        ratio2, info2 = parity_case(con, dtype, "normal", 21, 1.0, 0.5, reserved0=32)
+        assert info2.loader_a in (g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_K)
+        parity_case(con, dtype, "normal", 21, 1.0, 0.0, split_k=2)
+
+
 @pytest.mark.parametrize("sizes", [dict(m0=40, m1=33, n0=24, k=24), dict(m0=300, m1=7, n0=5, k=12),
                                    dict(m0=64, m1=9, n0=32, k=64), dict(m0=17, m1=3, n0=1, k=4)])
 def test_tensor_times_small_matrix_kernel(sizes):

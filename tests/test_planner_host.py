@@ -152,7 +152,8 @@ def test_split_k_planning():
 def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
     want = {  # key, dtype -> (path, loader_a, loader_b, epilogue)
         ("cfg1", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_K, g.GETT_EPI_DIRECT),
-        ("cfg2", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_K, g.GETT_EPI_DIRECT),
+        # cfg2: plain matrices, every tile is a box of a 2-D tensor map -> TMA
+        ("cfg2", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_TMA_FREE, g.GETT_LOAD_TMA_K, g.GETT_EPI_DIRECT),
         # cfg3: small N and K -> B is read once into shared memory, element by element
         ("cfg3", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_K, g.GETT_LOAD_SCALAR, g.GETT_EPI_DIRECT),
         ("cfg4", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_DIRECT),
@@ -164,6 +165,12 @@ def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
     # cfg5: the tile is all 8-wide pieces of B's stride-1 mode x the whole of C's stride-1 mode
     i = g.Plan(workload("cfg5").contraction, g.GETT_BF16_F32).info
     assert (i.tile_m, i.tile_n, i.tile_k) == (128, 192, 64) and i.digits_n == 4
+    # cfg4's 128-row tiles straddle the 72-wide modes: not boxes, so the gather loader stays
+    # a 4-D operand whose leading extents are multiples of the tile is a box of a 4-D tensor map
+    boxy = parse_spec("C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]",
+                      dict(m0=128, m1=3, n0=5, n1=256, k0=64, k1=3))
+    i = g.Plan(boxy, g.GETT_BF16_F32).info
+    assert (i.loader_a, i.loader_b) == (g.GETT_LOAD_TMA_FREE, g.GETT_LOAD_TMA_FREE)
     # odd extents cannot be gathered in 16-byte vectors: scalar path
     odd = parse_spec("C[m,n] = A[m,k] * B[k,n]", dict(m=7, n=5, k=3))
     assert g.Plan(odd, g.GETT_BF16_F32).info.path == g.GETT_PATH_SIMT
