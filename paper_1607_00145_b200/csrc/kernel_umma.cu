@@ -51,6 +51,7 @@ constexpr int MAX_STAGES = 8;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t ATOM_BYTES = 1024;      // 8 rows x 128 B
 constexpr uint32_t MN_BLOCK_BYTES = 8192;  // one 64-wide block of an MN-major operand: 64 k rows
+constexpr int RASTER_M = 16;               // tile rows per rasterisation panel
 constexpr int EPI_PITCH = 68;              // floats per staged row: 64 + 4 keeps 128-bit accesses conflict-free
 constexpr int EPI_GROUPS = 256 / 4;          // 16-byte groups per tile row, at most
 constexpr int EPI_DEPTH = 2;                 // staging buffers per warp: old C is fetched EPI_DEPTH-1 chunks ahead
@@ -84,8 +85,16 @@ __device__ __forceinline__ WorkItem decode_work(const GettKernelArgs& g, uint32_
     WorkItem it;
     it.z = w / tiles;
     const uint32_t t = w - it.z * tiles;
-    const uint32_t tn = t / g.tiles_m;
-    it.m0 = (t - tn * g.tiles_m) * TILE_M;
+    // Tiles are numbered panel by panel: a panel is RASTER_M tile rows high and spans all
+    // tile columns, and inside it the row index runs fastest.  The ~148 tiles in flight at
+    // any time then share few distinct rows of A and columns of B, which keeps them in L2.
+    const uint32_t per_panel = RASTER_M * g.tiles_n;
+    const uint32_t panel = t / per_panel;
+    const uint32_t first_m = panel * RASTER_M;
+    const uint32_t rows = min((uint32_t)RASTER_M, g.tiles_m - first_m);
+    const uint32_t in_panel = t - panel * per_panel;
+    const uint32_t tn = in_panel / rows;
+    it.m0 = (first_m + (in_panel - tn * rows)) * TILE_M;
     it.n0 = tn * (uint32_t)g.tile_n;
     it.kbeg = it.z * g.k_per_split;
     it.kend = min(g.K.size, it.kbeg + g.k_per_split);
@@ -418,7 +427,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                 const uint32_t k0 = wi.kbeg + j * TILE_K;
                 if (!all_tma) {
                     ptx::named_barrier(gbar, GROUP_LANES); // previous slab's k table no longer read
-                    if (!(g.debug & 16) && gl < TILE_K) {
+                    if (gl < TILE_K) {
                         const uint32_t k = k0 + gl;
                         uint32_t xa = INVALID16, xb = INVALID16;
                         if (k < wi.kend) {
