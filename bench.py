@@ -50,8 +50,58 @@ def _fp32_peak_tflops(sm_mhz: float) -> float:
     return 148 * 128 * 2 * sm_mhz * 1e6 / 1e12
 
 
+class NvmlSampler:
+    """SM clock and throttle reasons read through NVML (read-only) every few ms."""
+    BITS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+            0x4: "sw_power_cap"}
+
+    def __init__(self, index: int, period: float = 0.005):
+        import pynvml
+        self.nv = pynvml
+        pynvml.nvmlInit()
+        self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+        self.period, self.sm, self.reasons = period, [], set()
+        self.max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        self._stop = threading.Event()
+        self._t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for bit, name in self.BITS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=5)
+
+    def summary(self):
+        if not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": self.max, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.sm)), "sm_max_mhz": self.max,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+def clock_sampler(index: int):
+    try:
+        return NvmlSampler(index)
+    except Exception:
+        return ClockSampler(index)
+
+
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """nvidia-smi clocks and throttle reasons while the timed region runs (fallback)."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
@@ -185,13 +235,15 @@ def time_contraction(torch, g, con, dtype, alpha, beta, dev, steps, warmup, opts
         plan(alpha, a, b, beta, c, stream)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(steps):
-        plan(alpha, a, b, beta, c, stream)
-    e1.record(stream)
-    torch.cuda.synchronize()
+    with clock_sampler(torch.cuda.current_device()) as clk:
+        e0.record(stream)
+        for _ in range(steps):
+            plan(alpha, a, b, beta, c, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
     status = plan.device_status()
     info = plan.info.as_dict()
+    info["clocks"] = clk.summary()
     plan.close()
     if status != 0:
         raise RuntimeError(f"device status {status}")
@@ -243,7 +295,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
            for _ in range(args.steps)]
-    with ClockSampler(local) as clk:
+    with clock_sampler(local) as clk:
         t_wall0 = time.perf_counter()
         for e0, e1 in evs:
             if flush is not None:
@@ -373,16 +425,20 @@ def run_all(torch, g, peaks, fp32_peak, args):
     """Every workload/dtype pair: TFLOP/s, roofline fraction, equal-GEMM ratio."""
     rows = []
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    for key in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "splitk"):
+    for key in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "splitk", "splitk_vec"):
         w = workload(key)
         for dtype in w.dtypes:
             con = w.contraction
             a, b, c = make_inputs(con, dtype, w.dist, w.seed, w.beta)
             dev = (_to_dev(a, torch), _to_dev(b, torch), _to_dev(c, torch))
             variants = [("auto", {})]
-            if key in ("cfg3", "splitk"):
-                variants += [("split_k=1", {"split_k": 1}), ("split_k=2", {"split_k": 2}),
-                             ("split_k=4", {"split_k": 4})]
+            if key == "cfg3":
+                # K = 24 is one slab of the vector kernels; only the scalar path can slice it
+                variants += [("scalar split_k=1", {"path": 1, "split_k": 1}),
+                             ("scalar split_k=2", {"path": 1, "split_k": 2})]
+            if key in ("splitk", "splitk_vec"):
+                variants += [("split_k=1", {"split_k": 1}), ("split_k=4", {"split_k": 4}),
+                             ("split_k=16", {"split_k": 16})]
             for name, opts in variants:
                 try:
                     t, info = time_contraction(torch, g, con, dtype, w.alpha, w.beta, dev,
@@ -392,13 +448,14 @@ def run_all(torch, g, peaks, fp32_peak, args):
                                  "error": str(e)})
                     continue
                 flush.zero_()
-                t_roof, bound = roofline_time_s(con, dtype, w.beta, peaks, fp32_peak)
+                mhz = info["clocks"]["sm_mhz"] or 1965.0
+                t_roof, bound = roofline_time_s(con, dtype, w.beta, peaks, _fp32_peak_tflops(mhz))
                 row = {"workload": key, "dtype": DTYPE_NAMES[dtype], "variant": name,
                        "ms": t * 1e3, "tflops": con.flops() / t / 1e12,
                        "gbs": con.compulsory_bytes(dtype, w.beta) / t / 1e9, "bound": bound,
                        "roofline_frac": t_roof / t, "path": info["path"],
                        "tile": [info["tile_m"], info["tile_n"], info["tile_k"]],
-                       "split_k": info["split_k"]}
+                       "split_k": info["split_k"], "sm_mhz": mhz}
                 if name == "auto" and key != "cfg2" and not args.kernel_only:
                     eg = equal_gemm(con)
                     ga, gb, gc = make_inputs(eg, dtype, w.dist, w.seed, w.beta)

@@ -268,6 +268,10 @@ def workload(key: str, scale: Optional[Dict[str, int]] = None) -> Workload:
         "splitk": ("C[a,b] = A[c,a,d] * B[d,c,b]",
                    dict(a=384, b=376, c=384, d=384), (F32, BF16_F32), "uniform", 5, 1.0, 0.0,
                    "compute"),
+        # the same sizes with layouts the vector kernels can gather (K merges to one mode)
+        "splitk_vec": ("C[a,b] = A[a,c,d] * B[c,d,b]",
+                       dict(a=384, b=376, c=384, d=384), (F32, BF16_F32), "uniform", 5, 1.0, 0.0,
+                       "compute"),
     }
     spec, sizes, dtypes, dist, seed, alpha, beta, bound = table[key]
     sizes = dict(sizes)
