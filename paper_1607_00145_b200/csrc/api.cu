@@ -166,6 +166,7 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     args.b_kmajor = plan->b_kmajor;
     args.loader_a = vec_kind(plan->info.loader_a);
     args.loader_b = vec_kind(plan->info.loader_b);
+    args.tile_m = plan->info.tile_m;
     args.tile_n = plan->info.tile_n;
     args.stages = plan->info.stages;
     args.epilogue = plan->info.epilogue;

@@ -40,6 +40,7 @@ struct GettKernelArgs {
     int32_t a_kmajor;     // A's fastest-varying direction in memory is K (else M)
     int32_t b_kmajor;
     int32_t loader_a, loader_b; // gett_loader_t of the vectorised kernels
+    int32_t tile_m;       // tile height of the tensor-core kernel (128 or 256)
     int32_t tile_n;       // tile width of the tensor-core / FFMA kernels
     int32_t stages;       // depth of the shared-memory ring
     int32_t epilogue;     // gett_epilogue_t
@@ -97,8 +98,8 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* A,
 gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, size_t capacity);
 
 // Geometry of the tensor-core kernel (kernel_umma.cu), needed by the planner.
-int gett_umma_smem_bytes(int tile_n, int stages, int staged);
-int gett_umma_max_stages(int tile_n, int smem_limit, int staged);
+int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged);
+int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged);
 int gett_umma_block();
 int gett_umma_prod_groups(int stages); // producer groups in use; must divide the ring depth
 

@@ -28,9 +28,8 @@
 
 namespace {
 
-constexpr int TILE_M = 128;
+constexpr int MMA_M = 128;            // rows of one tcgen05.mma and of one accumulator buffer
 constexpr int TILE_K = 64;           // 16-bit elements per slab = one 128-byte swizzle row
-constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;
 constexpr int NUM_EPI_WARPS = 8;           // two sets of four: set s takes the CTA's tiles number s, s+2, ...
 constexpr int EPI_SET_THREADS = 128;
 #ifndef GETT_PROD_GROUPS
@@ -65,7 +64,7 @@ constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-by
 struct alignas(16) SmemTables { // the staging rows that follow it hold 128-bit vectors
     int64_t colC[2][256];                     // per epilogue set: C offset of each tile column
     uint32_t kTab[PROD_GROUPS][2][TILE_K];    // per producer group: A / B offsets of the slab's k
-    uint32_t rowTab[PROD_GROUPS][TILE_M + 256]; // per producer group: row offsets (K-major operands)
+    uint32_t rowTab[PROD_GROUPS][256 + 256];  // per producer group: row offsets (K-major operands)
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     int abort_flag;
@@ -73,13 +72,16 @@ struct alignas(16) SmemTables { // the staging rows that follow it hold 128-bit 
 
 static_assert(sizeof(SmemTables) % 16 == 0, "staging area must stay 16-byte aligned");
 
-__host__ __device__ constexpr uint32_t stage_bytes(uint32_t tile_n) { return A_STAGE_BYTES + tile_n * TILE_K * 2; }
+__host__ __device__ constexpr uint32_t stage_bytes(uint32_t tile_m, uint32_t tile_n)
+{
+    return (tile_m + tile_n) * TILE_K * 2;
+}
 
 struct WorkItem {
     uint32_t m0, n0, z, kbeg, kend, nslab;
 };
 
-__device__ __forceinline__ WorkItem decode_work(const GettKernelArgs& g, uint32_t w)
+__device__ __forceinline__ WorkItem decode_work(const GettKernelArgs& g, uint32_t w, uint32_t tile_m)
 {
     const uint32_t tiles = g.tiles_m * g.tiles_n;
     WorkItem it;
@@ -94,7 +96,7 @@ __device__ __forceinline__ WorkItem decode_work(const GettKernelArgs& g, uint32_
     const uint32_t rows = min((uint32_t)RASTER_M, g.tiles_m - first_m);
     const uint32_t in_panel = t - panel * per_panel;
     const uint32_t tn = in_panel / rows;
-    it.m0 = (first_m + (in_panel - tn * rows)) * TILE_M;
+    it.m0 = (first_m + (in_panel - tn * rows)) * tile_m;
     it.n0 = tn * (uint32_t)g.tile_n;
     it.kbeg = it.z * g.k_per_split;
     it.kend = min(g.K.size, it.kbeg + g.k_per_split);
@@ -243,7 +245,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
         if (cj < nchunk) {
             const uint32_t j = cj / NCH, ch = cj - j * NCH;
             if (ch == 0) {
-                const WorkItem wi = decode_work(g, blockIdx.x + (es + 2 * j) * gridDim.x);
+                const WorkItem wi = decode_work(g, blockIdx.x + (es + 2 * j) * gridDim.x, MMA_M);
                 int64_t rc = -1, dummy;
                 const uint32_t m = wi.m0 + eq * 32 + lane;
                 if (m < g.M.size)
@@ -341,7 +343,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
     ptx::cp_async_wait_all();
 }
 
-template <bool A_VEC_K, bool B_VEC_K, int TILE_N>
+template <bool A_VEC_K, bool B_VEC_K, int TILE_N, int TILE_M>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant__ GettTmaMaps tm)
 {
@@ -351,7 +353,9 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
     const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
     uint8_t* smem = smem_raw + pad;
     const uint32_t stages = (uint32_t)g.stages;
-    constexpr uint32_t sbytes = stage_bytes(TILE_N);
+    constexpr uint32_t sbytes = stage_bytes(TILE_M, TILE_N);
+    constexpr uint32_t A_STAGE_BYTES = TILE_M * TILE_K * 2;
+    constexpr bool TWO_HALVES = TILE_M == 2 * MMA_M; // one tile fills both accumulator buffers
     SmemTables* T = reinterpret_cast<SmemTables*>(smem + stages * sbytes);
     const uint32_t stage0 = ptx::smem_u32(smem);
 
@@ -393,7 +397,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
         uint32_t* kA = T->kTab[pg][0];
         uint32_t* kB = T->kTab[pg][1];
         uint32_t* rowA = T->rowTab[pg];
-        uint32_t* rowB = T->rowTab[pg] + TILE_M;
+        uint32_t* rowB = T->rowTab[pg] + 256;
         OperandLoader<A_VEC_K, TILE_M> la;
         OperandLoader<B_VEC_K, TILE_N> lb;
         const char* baseA = static_cast<const char*>(g.A);
@@ -406,7 +410,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
         uint32_t first = 0; // slab number of the current work item's first slab
         bool alive = true;
         for (uint32_t w = blockIdx.x; w < total_work && pg < ng; w += gridDim.x) {
-            const WorkItem wi = decode_work(g, w);
+            const WorkItem wi = decode_work(g, w, TILE_M);
             // my group's first slab in this item: smallest j with (first + j) % ng == pg
             uint32_t j = (pg + ng - first % ng) % ng;
             if (j < wi.nslab) {
@@ -507,7 +511,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
         // ------------------------------ MMA issuer -----------------------------
         if (lane == 0) {
             const uint32_t fmt = g.dtype == GETT_BF16_F32 ? 1u : 0u;
-            const uint32_t idesc = ptx::idesc_f16(fmt, A_VEC_K ? 0u : 1u, B_VEC_K ? 0u : 1u, TILE_M, TILE_N);
+            const uint32_t idesc = ptx::idesc_f16(fmt, A_VEC_K ? 0u : 1u, B_VEC_K ? 0u : 1u, MMA_M, TILE_N);
             // bytes the descriptor start address advances per 16-wide k step
             const uint32_t a_step = A_VEC_K ? 32u : 2u * ATOM_BYTES;
             const uint32_t b_step = B_VEC_K ? 32u : 2u * ATOM_BYTES;
@@ -516,9 +520,14 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
             uint32_t it = 0, local = 0;
             bool alive = true;
             for (uint32_t w = blockIdx.x; w < total_work && alive; w += gridDim.x, ++local) {
-                const WorkItem wi = decode_work(g, w);
-                const uint32_t buf = local & 1;
-                if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[buf]), ((local >> 1) & 1) ^ 1, abort_flag))
+                const WorkItem wi = decode_work(g, w, TILE_M);
+                // 128-row tiles alternate between the two accumulator buffers; a 256-row tile
+                // uses both (rows 0-127 in buffer 0, rows 128-255 in buffer 1)
+                const uint32_t buf = TWO_HALVES ? 0u : (local & 1);
+                const uint32_t par = TWO_HALVES ? (local & 1) : ((local >> 1) & 1);
+                if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[buf]), par ^ 1, abort_flag))
+                    break;
+                if (TWO_HALVES && !ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[1]), par ^ 1, abort_flag))
                     break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * 256;
@@ -535,17 +544,25 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                     ptx::tc_fence_after();
                     const uint32_t sa = stage0 + s * sbytes, sb = sa + A_STAGE_BYTES;
 #pragma unroll
-                    for (uint32_t kk = 0; kk < TILE_K / 16; ++kk) {
-                        const uint64_t ad = A_VEC_K ? ptx::smem_desc_sw128(sa + kk * a_step, 16, ATOM_BYTES)
-                                                    : ptx::smem_desc_sw128(sa + kk * a_step, lbo, sbo);
-                        const uint64_t bd = B_VEC_K ? ptx::smem_desc_sw128(sb + kk * b_step, 16, ATOM_BYTES)
-                                                    : ptx::smem_desc_sw128(sb + kk * b_step, lbo, sbo);
-                        ptx::umma_f16(d_tmem, ad, bd, idesc, (j | kk) ? 1u : 0u);
+                    for (uint32_t h = 0; h < (TWO_HALVES ? 2u : 1u); ++h) {
+                        // rows 128 h .. of the A tile start 16 KB further in either staging layout
+                        const uint32_t sah = sa + h * (MMA_M * TILE_K * 2);
+#pragma unroll
+                        for (uint32_t kk = 0; kk < TILE_K / 16; ++kk) {
+                            const uint64_t ad = A_VEC_K ? ptx::smem_desc_sw128(sah + kk * a_step, 16, ATOM_BYTES)
+                                                        : ptx::smem_desc_sw128(sah + kk * a_step, lbo, sbo);
+                            const uint64_t bd = B_VEC_K ? ptx::smem_desc_sw128(sb + kk * b_step, 16, ATOM_BYTES)
+                                                        : ptx::smem_desc_sw128(sb + kk * b_step, lbo, sbo);
+                            ptx::umma_f16(d_tmem + h * 256, ad, bd, idesc, (j | kk) ? 1u : 0u);
+                        }
                     }
                     ptx::umma_commit(ptx::smem_u32(&T->empty[s])); // stage reusable once these MMAs retire
                 }
-                if (alive)
+                if (alive) {
                     ptx::umma_commit(ptx::smem_u32(&T->acc_full[buf]));
+                    if (TWO_HALVES)
+                        ptx::umma_commit(ptx::smem_u32(&T->acc_full[1]));
+                }
             }
         }
         __syncwarp();
@@ -567,8 +584,14 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
         }
         int64_t* colC = T->colC[es];
         uint32_t j = 0; // counts this set's tiles
-        for (uint32_t w = blockIdx.x + es * gridDim.x; w < total_work && !staged; w += 2 * gridDim.x, ++j) {
-            const WorkItem wi = decode_work(g, w);
+        // 128-row tiles: set es takes every other tile.  256-row tiles: both sets work on
+        // every tile, set es on its rows 128 es .. 128 es + 127.
+        const uint32_t w_first = blockIdx.x + (TWO_HALVES ? 0u : es * gridDim.x);
+        const uint32_t w_step = (TWO_HALVES ? 1u : 2u) * gridDim.x;
+        for (uint32_t w = w_first; w < total_work && !staged; w += w_step, ++j) {
+            WorkItem wi = decode_work(g, w, TILE_M);
+            if (TWO_HALVES)
+                wi.m0 += es * MMA_M;
             const uint32_t buf = es;
             // C offsets of this tile: my row in a register, the columns in shared memory
             int64_t rowC = -1, dummy;
@@ -643,16 +666,16 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
 
 } // namespace
 
-int gett_umma_smem_bytes(int tile_n, int stages, int staged)
+int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged)
 {
-    return 1024 + stages * (int)stage_bytes((uint32_t)tile_n) + (int)sizeof(SmemTables) +
+    return 1024 + stages * (int)stage_bytes((uint32_t)tile_m, (uint32_t)tile_n) + (int)sizeof(SmemTables) +
            (staged ? EPI_STAGE_BYTES : 0);
 }
 
-int gett_umma_max_stages(int tile_n, int smem_limit, int staged)
+int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged)
 {
     int s = (smem_limit - 1024 - (int)sizeof(SmemTables) - (staged ? EPI_STAGE_BYTES : 0)) /
-            (int)stage_bytes((uint32_t)tile_n);
+            (int)stage_bytes((uint32_t)tile_m, (uint32_t)tile_n);
     s = s > MAX_STAGES ? MAX_STAGES : s;
     return s >= PROD_GROUPS ? s - s % PROD_GROUPS : s; // a stage is always served by the same group
 }
@@ -666,12 +689,18 @@ static cudaError_t launch_tn(const GettKernelArgs& args, const GettTmaMaps& maps
                              cudaStream_t stream)
 {
     void (*k)(GettKernelArgs, GettTmaMaps);
-    switch (args.tile_n) {
-    case 64: k = gett_umma_kernel<AK, BK, 64>; break;
-    case 128: k = gett_umma_kernel<AK, BK, 128>; break;
-    case 192: k = gett_umma_kernel<AK, BK, 192>; break;
-    case 256: k = gett_umma_kernel<AK, BK, 256>; break;
-    default: return cudaErrorInvalidValue;
+    if (args.tile_m == 256) {
+        if (args.tile_n != 256)
+            return cudaErrorInvalidValue;
+        k = gett_umma_kernel<AK, BK, 256, 256>;
+    } else {
+        switch (args.tile_n) {
+        case 64: k = gett_umma_kernel<AK, BK, 64, 128>; break;
+        case 128: k = gett_umma_kernel<AK, BK, 128, 128>; break;
+        case 192: k = gett_umma_kernel<AK, BK, 192, 128>; break;
+        case 256: k = gett_umma_kernel<AK, BK, 256, 128>; break;
+        default: return cudaErrorInvalidValue;
+        }
     }
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess)

@@ -419,7 +419,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.smem_bytes = gett_ffma_smem_bytes(tn, st);
         info.epilogue = GETT_EPI_DIRECT;
     } else { // GETT_PATH_UMMA
-        if ((o.tile_m && o.tile_m != 128) || (o.tile_k && o.tile_k != 64))
+        if ((o.tile_m && o.tile_m != 128 && o.tile_m != 256) || (o.tile_k && o.tile_k != 64))
             return GETT_ERR_UNSUPPORTED;
         // Unpacking (Eq. 11).  Direct stores are already coalesced when C's stride-1
         // mode leads the M order (a warp's 32 rows are 32 consecutive floats).  When it
@@ -475,17 +475,28 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
             return GETT_ERR_UNSUPPORTED;
         const int smem_limit = 227 * 1024;
         const int staged = info.epilogue == GETT_EPI_STAGED;
-        int st = o.stages ? o.stages : gett_umma_max_stages(tn, smem_limit, staged);
-        if (st < 1 || st > gett_umma_max_stages(tn, smem_limit, staged) || st % gett_umma_prod_groups(st))
+        // 256-row tiles (both accumulator buffers for one tile) cut the operand bytes per
+        // flop by a third; worth it when the contraction is long enough to be bound by
+        // operand delivery and there are still at least two waves of tiles.  The epilogue
+        // then no longer overlaps the next tile's main loop.
+        int tmh = o.tile_m;
+        if (tmh == 0) {
+            const uint64_t t256 = (uint64_t)ceil_div(p->M.size, 256) * ceil_div(p->N.size, 256);
+            tmh = (tn == 256 && !staged && p->K.size >= 2048 && t256 >= 2ull * sms) ? 256 : 128;
+        }
+        if (tmh == 256 && (tn != 256 || staged))
             return GETT_ERR_UNSUPPORTED;
-        info.tile_m = 128;
+        int st = o.stages ? o.stages : gett_umma_max_stages(tmh, tn, smem_limit, staged);
+        if (st < 1 || st > gett_umma_max_stages(tmh, tn, smem_limit, staged) || st % gett_umma_prod_groups(st))
+            return GETT_ERR_UNSUPPORTED;
+        info.tile_m = tmh;
         info.tile_n = tn;
         info.tile_k = 64;
         info.stages = st;
         info.block = gett_umma_block();
-        info.smem_bytes = gett_umma_smem_bytes(tn, st, staged);
+        info.smem_bytes = gett_umma_smem_bytes(tmh, tn, st, staged);
         if (!(p->debug & 32)) { // (debug & 32: experiment switch, gather even where TMA applies)
-            make_tma_recipe(p->M, true, p->K, true, info.loader_a, 128, p->tma_a);
+            make_tma_recipe(p->M, true, p->K, true, info.loader_a, (uint32_t)tmh, p->tma_a);
             make_tma_recipe(p->N, true, p->K, false, info.loader_b, (uint32_t)tn, p->tma_b);
             if (p->tma_a.enabled)
                 info.loader_a = info.loader_a == GETT_LOAD_VEC_FREE ? GETT_LOAD_TMA_FREE : GETT_LOAD_TMA_K;

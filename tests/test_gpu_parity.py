@@ -80,6 +80,22 @@ def test_tma_loader_against_gather_loader_and_oracle(spec, sizes):
         parity_case(con, dtype, "normal", 21, 1.0, 0.0, split_k=2)
 
 
+@pytest.mark.parametrize("spec,sizes", [
+    ("C[m,n] = A[m,k] * B[k,n]", dict(m=648, n=520, k=200)),                     # TMA, ragged 256-row tiles
+    ("C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]",
+     dict(m0=24, m1=23, n0=11, n1=24, k0=8, k1=19)),                             # gathers, MN-major both
+    ("C[m,n] = A[k,m] * B[n,k]", dict(m=520, n=264, k=136)),                     # K-major A, N-major B
+])
+def test_256_row_tiles(spec, sizes):
+    """One tile in both accumulator buffers (tile_m = 256), forced, against the oracle."""
+    con = parse_spec(spec, sizes)
+    for dtype in (BF16_F32, F16_F32):
+        for extra in ({}, {"reserved0": 32}, {"split_k": 2}):
+            ratio, info = parity_case(con, dtype, "normal", 33, 1.0, 0.5, repeat=2, tile_m=256,
+                                      tile_n=256, **extra)
+            assert info.tile_m == 256 and info.path == g.GETT_PATH_UMMA
+
+
 @pytest.mark.parametrize("sizes", [dict(m0=40, m1=33, n0=24, k=24), dict(m0=300, m1=7, n0=5, k=12),
                                    dict(m0=64, m1=9, n0=32, k=64), dict(m0=17, m1=3, n0=1, k=4)])
 def test_tensor_times_small_matrix_kernel(sizes):
