@@ -9,6 +9,9 @@
 //                                       XOR-swizzled by (row / 4) % 8 so that both the
 //                                       copy and the 128-bit fragment reads are
 //                                       bank-conflict free
+//   no usable stride-1 mode ("SCALAR") -> [k][row], gathered element by element with
+//                                       4-byte cp.async (also chosen on purpose when the
+//                                       vector-friendly order would scatter the stores to C)
 // The macro-kernel is an 8 x (TN/16) register tile per thread fed by 128-bit shared
 // loads (Sec. 3.1: outer products into a register-resident tile); unpacking
 // (Eq. 11) writes alpha*acc + beta*C through C's permutation, as 128-bit stores
@@ -25,33 +28,48 @@ template <int TN>
 struct FfmaSmem {
     int64_t offCM[TM];
     int64_t offCN[TN];
-    uint32_t rowA[TM];       // A row offsets, 16-byte units (INVALID16 beyond M)
+    uint32_t rowA[TM];       // A row offsets in elements (INVALID16 beyond M)
     uint32_t rowB[TN];
-    uint32_t kTab[2][2][TK]; // [parity][A/B][k] offsets of a slab's k, 16-byte units
+    uint32_t kTab[2][2][TK]; // [parity][A/B][k] offsets of a slab's k, in elements
 };
 
 template <int TN>
 __host__ __device__ constexpr int ffma_stage_bytes() { return (TM + TN) * TK * 4; }
 
-// Gather one operand slab: R rows x 32 k.
-template <bool VEC_K, int R>
+// Gather one operand slab: R rows x 32 k.  L is the operand's gett_loader_t.
+template <int L, int R>
 __device__ __forceinline__ void load_operand(const char* __restrict__ base, uint32_t dst,
-                                             const uint32_t* rowTab, const uint32_t* kTab, int tid)
+                                             const uint32_t* rowTab, const uint32_t* kTab, int tid,
+                                             bool k_fastest)
 {
+    if (L == GETT_LOAD_SCALAR) {
+        constexpr int NP = R * TK / NT;
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            const uint32_t q = tid + NT * p;
+            // consecutive threads follow the direction in which the operand is denser in memory
+            const uint32_t k = k_fastest ? q % TK : q / R;
+            const uint32_t r = k_fastest ? q / TK : q % R;
+            const uint32_t r1 = rowTab[r], k1 = kTab[k];
+            const bool ok = r1 != INVALID16 && k1 != INVALID16;
+            ptx::cp_async_4(dst + (k * R + r) * 4, base + (ok ? ((uint64_t)(r1 + k1) << 2) : 0), ok ? 4u : 0u);
+        }
+        return;
+    }
     constexpr int PIECES = R * TK / 4;
     constexpr int NP = (PIECES + NT - 1) / NT;
-    if (VEC_K) {
+    if (L == GETT_LOAD_VEC_K) {
         const uint32_t kc = tid & 7;
-        const uint32_t k16 = kTab[kc * 4];
+        const uint32_t k1 = kTab[kc * 4];
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
             const uint32_t m = (tid >> 3) + 32 * p;
             if (PIECES % NT != 0 && m >= (uint32_t)R)
                 break;
-            const uint32_t r16 = rowTab[m];
-            const bool ok = r16 != INVALID16 && k16 != INVALID16;
+            const uint32_t r1 = rowTab[m];
+            const bool ok = r1 != INVALID16 && k1 != INVALID16;
             ptx::cp_async_16(dst + m * 128 + ((kc ^ ((m >> 2) & 7)) << 4),
-                             base + (ok ? ((uint64_t)(r16 + k16) << 4) : 0), ok ? 16u : 0u);
+                             base + (ok ? ((uint64_t)(r1 + k1) << 2) : 0), ok ? 16u : 0u);
         }
     } else {
         constexpr int PPR = R / 4; // pieces per k row
@@ -61,9 +79,9 @@ __device__ __forceinline__ void load_operand(const char* __restrict__ base, uint
             if (PIECES % NT != 0 && q >= (uint32_t)PIECES)
                 break;
             const uint32_t k = q / PPR, mc = q % PPR;
-            const uint32_t r16 = rowTab[mc * 4], k16 = kTab[k];
-            const bool ok = r16 != INVALID16 && k16 != INVALID16;
-            ptx::cp_async_16(dst + (k * R + mc * 4) * 4, base + (ok ? ((uint64_t)(r16 + k16) << 4) : 0),
+            const uint32_t r1 = rowTab[mc * 4], k1 = kTab[k];
+            const bool ok = r1 != INVALID16 && k1 != INVALID16;
+            ptx::cp_async_16(dst + (k * R + mc * 4) * 4, base + (ok ? ((uint64_t)(r1 + k1) << 2) : 0),
                              ok ? 16u : 0u);
         }
     }
@@ -84,9 +102,10 @@ __device__ __forceinline__ void frag_kmajor(const char* tile, const uint32_t (&r
     }
 }
 
-template <bool A_K, bool B_K, int TN>
+template <int LA, int LB, int TN>
 __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant__ GettKernelArgs g)
 {
+    constexpr bool A_K = LA == GETT_LOAD_VEC_K, B_K = LB == GETT_LOAD_VEC_K; // staged [row][k]
     constexpr int FN = TN / 16;                 // columns per thread (8 or 2)
     constexpr int STAGE = ffma_stage_bytes<TN>();
     extern __shared__ __align__(128) uint8_t smem[];
@@ -115,10 +134,10 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
         if (ok)
             gett_decompose(isA ? g.M : g.N, idx, x, y);
         if (isA) {
-            T->rowA[r] = ok ? (uint32_t)(x >> 2) : INVALID16;
+            T->rowA[r] = ok ? (uint32_t)x : INVALID16;
             T->offCM[r] = ok ? y : -1;
         } else {
-            T->rowB[r - TM] = ok ? (uint32_t)(x >> 2) : INVALID16;
+            T->rowB[r - TM] = ok ? (uint32_t)x : INVALID16;
             T->offCN[r - TM] = ok ? y : -1;
         }
     }
@@ -129,8 +148,8 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
             if (slab < nslab && k < kend) {
                 int64_t x, y;
                 gett_decompose(g.K, k, x, y);
-                xa = (uint32_t)(x >> 2);
-                xb = (uint32_t)(y >> 2);
+                xa = (uint32_t)x;
+                xb = (uint32_t)y;
             }
             T->kTab[slab & 1][0][tid] = xa;
             T->kTab[slab & 1][1][tid] = xb;
@@ -139,9 +158,10 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     auto issue = [&](int slab) {
         if (slab < nslab) {
             const uint32_t dst = smem0 + (slab % stages) * STAGE;
-            load_operand<A_K, TM>(static_cast<const char*>(g.A), dst, T->rowA, T->kTab[slab & 1][0], tid);
-            load_operand<B_K, TN>(static_cast<const char*>(g.B), dst + TM * TK * 4, T->rowB,
-                                  T->kTab[slab & 1][1], tid);
+            load_operand<LA, TM>(static_cast<const char*>(g.A), dst, T->rowA, T->kTab[slab & 1][0], tid,
+                                 g.a_kmajor != 0);
+            load_operand<LB, TN>(static_cast<const char*>(g.B), dst + TM * TK * 4, T->rowB,
+                                 T->kTab[slab & 1][1], tid, g.b_kmajor != 0);
         }
         ptx::cp_async_commit();
     };
@@ -233,6 +253,38 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     // ---- unpack: C <- alpha * acc + beta * C (or the raw slice sums under split-K) ----
     const float alpha = g.alpha, beta = g.beta;
     const bool vec_m = g.c_vec == 1;
+    if (FN == 8 && g.c_vec == 2 && g.split_k == 1) {
+        // four consecutive tile columns are one aligned 16-byte vector of C; the old values
+        // of four rows (eight vectors) are requested together so their latencies overlap
+        int64_t cn[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+            cn[h] = T->offCN[cols[(4 * h) % FN]];
+#pragma unroll
+        for (int i0 = 0; i0 < 8; i0 += 4) {
+            float4 old[4][2];
+            float4* dst[4][2];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int64_t cm = T->offCM[rows[i0 + i]];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    dst[i][h] = (cm >= 0 && cn[h] >= 0) ? reinterpret_cast<float4*>(g.C + cm + cn[h]) : nullptr;
+                    old[i][h] = (beta != 0.f && dst[i][h]) ? __ldcg(dst[i][h]) : make_float4(0, 0, 0, 0);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                    if (dst[i][h])
+                        *dst[i][h] = make_float4(fmaf(beta, old[i][h].x, alpha * acc[i0 + i][(4 * h) % FN]),
+                                                 fmaf(beta, old[i][h].y, alpha * acc[i0 + i][(4 * h + 1) % FN]),
+                                                 fmaf(beta, old[i][h].z, alpha * acc[i0 + i][(4 * h + 2) % FN]),
+                                                 fmaf(beta, old[i][h].w, alpha * acc[i0 + i][(4 * h + 3) % FN]));
+        }
+        return;
+    }
 #pragma unroll
     for (int j = 0; j < FN; ++j) {
         const int64_t cn = T->offCN[cols[j]];
@@ -279,14 +331,14 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     }
 }
 
-template <bool AK, bool BK>
+template <int LA, int LB>
 cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
 {
     void (*k)(GettKernelArgs);
     if (args.tile_n == 128)
-        k = gett_ffma_kernel<AK, BK, 128>;
+        k = gett_ffma_kernel<LA, LB, 128>;
     else if (args.tile_n == 32)
-        k = gett_ffma_kernel<AK, BK, 32>;
+        k = gett_ffma_kernel<LA, LB, 32>;
     else
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -294,6 +346,16 @@ cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cudaStream
         return e;
     k<<<grid, NT, smem, stream>>>(args);
     return cudaGetLastError();
+}
+
+template <int LA>
+cudaError_t launch_b(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
+{
+    switch (args.loader_b) {
+    case GETT_LOAD_VEC_K: return launch_tn<LA, GETT_LOAD_VEC_K>(args, grid, smem, stream);
+    case GETT_LOAD_VEC_FREE: return launch_tn<LA, GETT_LOAD_VEC_FREE>(args, grid, smem, stream);
+    default: return launch_tn<LA, GETT_LOAD_SCALAR>(args, grid, smem, stream);
+    }
 }
 
 } // namespace
@@ -306,12 +368,9 @@ int gett_ffma_smem_bytes(int tile_n, int stages)
 
 cudaError_t gett_launch_ffma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
 {
-    const bool ak = args.loader_a == GETT_LOAD_VEC_K, bk = args.loader_b == GETT_LOAD_VEC_K;
-    if (ak && bk)
-        return launch_tn<true, true>(args, grid, smem, stream);
-    if (ak)
-        return launch_tn<true, false>(args, grid, smem, stream);
-    if (bk)
-        return launch_tn<false, true>(args, grid, smem, stream);
-    return launch_tn<false, false>(args, grid, smem, stream);
+    switch (args.loader_a) {
+    case GETT_LOAD_VEC_K: return launch_b<GETT_LOAD_VEC_K>(args, grid, smem, stream);
+    case GETT_LOAD_VEC_FREE: return launch_b<GETT_LOAD_VEC_FREE>(args, grid, smem, stream);
+    default: return launch_b<GETT_LOAD_SCALAR>(args, grid, smem, stream);
+    }
 }

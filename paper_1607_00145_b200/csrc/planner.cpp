@@ -290,6 +290,22 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     int leadK = find_unit(ik, 0); // A's stride-1 mode, if it is contracted ...
     if (leadK < 0)
         leadK = find_unit(ik, 1); // ... else B's
+    if (dtype == GETT_F32) {
+        // fp32 operands can also be gathered element by element (4-byte cp.async), so when
+        // the contraction is short (C's traffic outweighs the operands') the set that
+        // carries C's stride-1 mode is ordered for C: its canonical order starts with
+        // that mode, and the operand whose own stride-1 mode loses the lead is gathered
+        // by elements (or along K).
+        int64_t ksize = 1;
+        for (const GettMode& m : ik)
+            ksize *= m.ext;
+        if (ksize <= 512) {
+            if (find_unit(im, 2) >= 0 && leadM != find_unit(im, 2))
+                leadM = -1;
+            if (find_unit(in, 2) >= 0 && leadN != find_unit(in, 2))
+                leadN = -1;
+        }
+    }
     p->tm = order_with_lead(im, leadM);
     p->tn = order_with_lead(in, leadN);
     {
@@ -360,13 +376,13 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
                            p->K.size <= (uint32_t)gett_ffma_skinny_max_k() && o.split_k <= 1 &&
                            (o.tile_m == 0 || o.tile_m == gett_ffma_skinny_rows()) && o.tile_n == 0 &&
                            o.tile_k == 0 && o.stages == 0 && o.epilogue != GETT_EPI_STAGED;
-    const bool ffma_ok = dtype == GETT_F32 && (both_vec || skinny_ok);
+    const bool ffma_ok = dtype == GETT_F32; // any layout: operands without usable vectors go scalar
     if (path == GETT_PATH_AUTO)
         path = umma_ok ? GETT_PATH_UMMA : ffma_ok ? GETT_PATH_FFMA : GETT_PATH_SIMT;
     if ((path == GETT_PATH_UMMA && !umma_ok) || (path == GETT_PATH_FFMA && !ffma_ok))
         return GETT_ERR_UNSUPPORTED;
-    // four consecutive tile rows of C form one aligned 16-byte vector
-    p->c_vec = vec_ok(p->M, false, p->N, false, 4) ? 1 : 0;
+    // four consecutive tile rows (1) or columns (2) of C form one aligned 16-byte vector
+    p->c_vec = vec_ok(p->M, false, p->N, false, 4) ? 1 : vec_ok(p->N, false, p->M, false, 4) ? 2 : 0;
     info.path = path;
     p->debug = o.reserved[0];
     p->skinny = 0;
