@@ -185,12 +185,21 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     const uint32_t swA = tx & 7;
     const uint32_t swB = FN == 8 ? (ty & 7) : ((ty * FN) >> 2) & 7;
 
-    float acc[8][FN];
+    // Accumulators are held in pairs so that one packed instruction (two independent
+    // round-to-nearest fp32 FMAs, results identical to two scalar fmaf) updates two of
+    // them.  Pairs run along rows when A's fragment delivers neighbouring rows together
+    // ([k][row] staging), else along columns.
+    constexpr bool PAIR_ROWS = !A_K || B_K;
+    constexpr int PI = PAIR_ROWS ? 4 : 8, PJ = PAIR_ROWS ? FN : FN / 2;
+    float2 accp[PI][PJ];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < PI; ++i)
 #pragma unroll
-        for (int j = 0; j < FN; ++j)
-            acc[i][j] = 0.f;
+        for (int j = 0; j < PJ; ++j)
+            accp[i][j] = make_float2(0.f, 0.f);
+#define ACC(i, j)                                                                       \
+    (PAIR_ROWS ? (((i) & 1) ? accp[(i) / 2 % PI][(j) % PJ].y : accp[(i) / 2 % PI][(j) % PJ].x) \
+               : (((j) & 1) ? accp[(i) % PI][(j) / 2 % PJ].y : accp[(i) % PI][(j) / 2 % PJ].x))
 
     for (int slab = 0; slab < nslab; ++slab) {
         // all but the newest (stages - 2) copy groups have landed => this slab is complete
@@ -239,12 +248,33 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
                 }
             }
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
+            for (int kk = 0; kk < 4; ++kk) {
+                if constexpr (PAIR_ROWS) {
+                    float2 b2[FN];
 #pragma unroll
                     for (int j = 0; j < FN; ++j)
-                        acc[i][j] = fmaf(a[i][kk], b[j][kk], acc[i][j]);
+                        b2[j] = make_float2(b[j][kk], b[j][kk]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 a2 = make_float2(a[2 * i][kk], a[2 * i + 1][kk]);
+#pragma unroll
+                        for (int j = 0; j < FN; ++j)
+                            accp[i][j] = __ffma2_rn(a2, b2[j], accp[i][j]);
+                    }
+                } else {
+                    float2 b2[FN / 2];
+#pragma unroll
+                    for (int j = 0; j < FN / 2; ++j)
+                        b2[j] = make_float2(b[2 * j][kk], b[2 * j + 1][kk]);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float2 a2 = make_float2(a[i][kk], a[i][kk]);
+#pragma unroll
+                        for (int j = 0; j < FN / 2; ++j)
+                            accp[i][j] = __ffma2_rn(a2, b2[j], accp[i][j]);
+                    }
+                }
+            }
         }
     }
     ptx::cp_async_wait_all();
@@ -278,10 +308,10 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
                     if (dst[i][h])
-                        *dst[i][h] = make_float4(fmaf(beta, old[i][h].x, alpha * acc[i0 + i][(4 * h) % FN]),
-                                                 fmaf(beta, old[i][h].y, alpha * acc[i0 + i][(4 * h + 1) % FN]),
-                                                 fmaf(beta, old[i][h].z, alpha * acc[i0 + i][(4 * h + 2) % FN]),
-                                                 fmaf(beta, old[i][h].w, alpha * acc[i0 + i][(4 * h + 3) % FN]));
+                        *dst[i][h] = make_float4(fmaf(beta, old[i][h].x, alpha * ACC(i0 + i, (4 * h) % FN)),
+                                                 fmaf(beta, old[i][h].y, alpha * ACC(i0 + i, (4 * h + 1) % FN)),
+                                                 fmaf(beta, old[i][h].z, alpha * ACC(i0 + i, (4 * h + 2) % FN)),
+                                                 fmaf(beta, old[i][h].w, alpha * ACC(i0 + i, (4 * h + 3) % FN)));
         }
         return;
     }
@@ -298,14 +328,14 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     if (m0 + r0 + i < Msz)
-                        dst[i] = acc[4 * h + i][j];
+                        dst[i] = ACC(4 * h + i, j);
             } else if (vec_m) {
                 const int64_t cm = T->offCM[r0];
                 if (cm < 0)
                     continue;
                 float4* dst = reinterpret_cast<float4*>(g.C + cm + cn);
-                float4 v = make_float4(alpha * acc[4 * h][j], alpha * acc[4 * h + 1][j],
-                                       alpha * acc[4 * h + 2][j], alpha * acc[4 * h + 3][j]);
+                float4 v = make_float4(alpha * ACC(4 * h, j), alpha * ACC(4 * h + 1, j),
+                                       alpha * ACC(4 * h + 2, j), alpha * ACC(4 * h + 3, j));
                 if (beta != 0.f) {
                     const float4 o = *dst;
                     v.x = fmaf(beta, o.x, v.x);
@@ -321,7 +351,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
                     if (cm < 0)
                         continue;
                     float* dst = g.C + cm + cn;
-                    float v = alpha * acc[4 * h + i][j];
+                    float v = alpha * ACC(4 * h + i, j);
                     if (beta != 0.f)
                         v = fmaf(beta, *dst, v);
                     *dst = v;
@@ -357,6 +387,8 @@ cudaError_t launch_b(const GettKernelArgs& args, int grid, int smem, cudaStream_
     default: return launch_tn<LA, GETT_LOAD_SCALAR>(args, grid, smem, stream);
     }
 }
+
+#undef ACC
 
 } // namespace
 

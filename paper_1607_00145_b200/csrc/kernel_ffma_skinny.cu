@@ -107,12 +107,14 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
         __syncthreads(); // tile `it` and its row table visible; the stage of tile it-1 is free
         issue(it + STAGES - 1);
         const float* As = reinterpret_cast<const float*>(ring + (it % STAGES) * tile_bytes);
-        float acc[RPT][CPT];
+        // accumulators are kept as column pairs: one packed instruction performs two
+        // independent round-to-nearest fp32 FMAs (same results as two scalar fmaf)
+        float2 acc[RPT][CPT / 2];
 #pragma unroll
         for (int i = 0; i < RPT; ++i)
 #pragma unroll
-            for (int j = 0; j < CPT; ++j)
-                acc[i][j] = 0.f;
+            for (int j = 0; j < CPT / 2; ++j)
+                acc[i][j] = make_float2(0.f, 0.f);
 #pragma unroll 2
         for (uint32_t kc = 0; kc < KC; ++kc) {
             float4 a[RPT];
@@ -121,29 +123,26 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
                 a[i] = *reinterpret_cast<const float4*>(As + (q + QL * i) * pitch + kc * 4);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
-                float b[CPT];
+                float2 b[CPT / 2];
                 const float* brow = Bs + (kc * 4 + kk) * NP + cg * CPT;
                 // cg * CPT * 4 bytes is 16-byte aligned when CPT % 4 == 0, else 8-byte aligned
 #pragma unroll
                 for (int j = 0; j < CPT; j += 2) {
                     if (CPT % 4 == 0 && j % 4 == 0) {
                         const float4 v = *reinterpret_cast<const float4*>(brow + j);
-                        b[j] = v.x;
-                        b[j + 1] = v.y;
-                        b[j + 2] = v.z;
-                        b[j + 3] = v.w;
+                        b[j / 2] = make_float2(v.x, v.y);
+                        b[j / 2 + 1] = make_float2(v.z, v.w);
                     } else if (CPT % 4 != 0) {
-                        const float2 v = *reinterpret_cast<const float2*>(brow + j);
-                        b[j] = v.x;
-                        b[j + 1] = v.y;
+                        b[j / 2] = *reinterpret_cast<const float2*>(brow + j);
                     }
                 }
 #pragma unroll
                 for (int i = 0; i < RPT; ++i) {
                     const float av = kk == 0 ? a[i].x : kk == 1 ? a[i].y : kk == 2 ? a[i].z : a[i].w;
+                    const float2 a2 = make_float2(av, av);
 #pragma unroll
-                    for (int j = 0; j < CPT; ++j)
-                        acc[i][j] = fmaf(av, b[j], acc[i][j]);
+                    for (int j = 0; j < CPT / 2; ++j)
+                        acc[i][j] = __ffma2_rn(a2, b[j], acc[i][j]);
                 }
             }
         }
@@ -161,7 +160,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
 #pragma unroll
             for (int j = 0; j < CPT; ++j)
                 if (cn[j] >= 0)
-                    crow[cn[j]] = fmaf(beta, old[j], alpha * acc[i][j]);
+                    crow[cn[j]] = fmaf(beta, old[j], alpha * ((j & 1) ? acc[i][j / 2].y : acc[i][j / 2].x));
         }
     }
     ptx::cp_async_wait_all();
