@@ -29,13 +29,14 @@ struct SkinnyTables {
 // 128-bit reads of eight consecutive rows fall into eight different bank groups.
 __host__ __device__ constexpr uint32_t skinny_pitch(uint32_t K) { return K + (K % 8 == 0 ? 4 : 8); }
 
-template <int CPT>
+// KCT: K / 4 when known at compile time (the k loop is then fully unrolled), 0 = run time
+template <int CPT, int KCT>
 __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_constant__ GettKernelArgs g)
 {
     constexpr int NP = 4 * CPT; // padded row of B in shared memory
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t K = g.K.size, N = g.N.size, Msz = g.M.size;
-    const uint32_t KC = K / 4;
+    const uint32_t KC = KCT ? (uint32_t)KCT : K / 4;
     const uint32_t pitch = skinny_pitch(K);
     const uint32_t tile_bytes = ROWS * pitch * 4;
     float* Bs = reinterpret_cast<float*>(smem);                       // [K][NP]
@@ -70,9 +71,15 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
     }
     // Thread `tid` owns rows tid and tid + NT of every tile: it computes their offsets,
     // copies their K/4 pieces, and publishes their C offsets for whoever accumulates them.
+    // Each CTA takes a contiguous run of row tiles, so that per column of C it writes one
+    // sequential stream (better DRAM page locality than tiles strided by the grid size).
+    const uint32_t chunk = (ntiles + gridDim.x - 1) / gridDim.x;
+    const uint32_t t_begin = blockIdx.x * chunk;
+    const uint32_t t_end = min(ntiles, t_begin + chunk);
+    const bool affine_rows = g.M.ndig == 1 && ROWS == NT;
     auto issue = [&](uint32_t it) {
-        const uint32_t t = blockIdx.x + it * gridDim.x;
-        if (t < ntiles) {
+        const uint32_t t = t_begin + it;
+        if (t < t_end) {
 #pragma unroll
             for (int h = 0; h < ROWS / NT; ++h) {
                 const uint32_t row = tid + h * NT;
@@ -84,9 +91,27 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
                 T->offCM[it % TSLOTS][row] = y;
                 const char* src = static_cast<const char*>(g.A) + (ok ? x * 4 : 0);
                 const uint32_t dst = ring_u32 + (it % STAGES) * tile_bytes + row * pitch * 4;
+                if (!affine_rows) {
 #pragma unroll 2
-                for (uint32_t kc = 0; kc < KC; ++kc)
-                    ptx::cp_async_16(dst + kc * 16, src + (ok ? ((uint64_t)T->kA[kc] << 4) : 0), ok ? 16u : 0u);
+                    for (uint32_t kc = 0; kc < KC; ++kc)
+                        ptx::cp_async_16(dst + kc * 16, src + (ok ? ((uint64_t)T->kA[kc] << 4) : 0), ok ? 16u : 0u);
+                }
+            }
+            if (affine_rows) {
+                // M is a single digit: a row's offset is m * stride, so consecutive threads can
+                // take consecutive 16-byte pieces of the tile (full 128-byte lines per warp)
+                const uint32_t dst0 = ring_u32 + (it % STAGES) * tile_bytes;
+#pragma unroll(KCT ? KCT : 2)
+                for (uint32_t p = 0; p < KC; ++p) {
+                    const uint32_t q = tid + NT * p;
+                    const uint32_t row = q / KC, kc = q - row * KC;
+                    const uint32_t m = t * ROWS + row;
+                    const bool ok = m < Msz;
+                    ptx::cp_async_16(dst0 + row * pitch * 4 + kc * 16,
+                                     static_cast<const char*>(g.A) +
+                                         (ok ? ((uint64_t)m * (uint64_t)g.M.sX[0] * 4 + ((uint64_t)T->kA[kc] << 4)) : 0),
+                                     ok ? 16u : 0u);
+                }
             }
         }
         ptx::cp_async_commit();
@@ -102,7 +127,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
         cn[j] = T->offCN[cg * CPT + j];
-    for (uint32_t it = 0; blockIdx.x + it * gridDim.x < ntiles; ++it) {
+    for (uint32_t it = 0; t_begin + it < t_end; ++it) {
         ptx::cp_async_wait<STAGES - 2>();
         __syncthreads(); // tile `it` and its row table visible; the stage of tile it-1 is free
         issue(it + STAGES - 1);
@@ -115,8 +140,8 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
 #pragma unroll
             for (int j = 0; j < CPT / 2; ++j)
                 acc[i][j] = make_float2(0.f, 0.f);
-#pragma unroll 2
-        for (uint32_t kc = 0; kc < KC; ++kc) {
+#pragma unroll(KCT ? KCT : 2)
+        for (uint32_t kc = 0; kc < KC && !(g.debug & 64); ++kc) { // (debug & 64: experiment, no math)
             float4 a[RPT];
 #pragma unroll
             for (int i = 0; i < RPT; ++i)
@@ -150,7 +175,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
 #pragma unroll
         for (int i = 0; i < RPT; ++i) {
             const int64_t cm = offCM[q + QL * i];
-            if (cm < 0)
+            if (cm < 0 || (g.debug & 2)) // (debug & 2: experiment, no stores)
                 continue;
             float* crow = g.C + cm;
             float old[CPT];
@@ -184,13 +209,17 @@ cudaError_t gett_launch_ffma_skinny(const GettKernelArgs& args, int grid, int sm
 {
     const int cpt = skinny_cpt(args.N.size);
     void (*k)(GettKernelArgs);
+    const uint32_t K = args.K.size;
+#define SKINNY_PICK(CPT) k = K == 24 ? gett_ffma_skinny_kernel<CPT, 6> : K == 32 ? gett_ffma_skinny_kernel<CPT, 8> \
+                             : K == 16 ? gett_ffma_skinny_kernel<CPT, 4> : gett_ffma_skinny_kernel<CPT, 0>
     switch (cpt) {
-    case 2: k = gett_ffma_skinny_kernel<2>; break;
-    case 4: k = gett_ffma_skinny_kernel<4>; break;
-    case 6: k = gett_ffma_skinny_kernel<6>; break;
-    case 8: k = gett_ffma_skinny_kernel<8>; break;
+    case 2: SKINNY_PICK(2); break;
+    case 4: SKINNY_PICK(4); break;
+    case 6: SKINNY_PICK(6); break;
+    case 8: SKINNY_PICK(8); break;
     default: return cudaErrorInvalidValue;
     }
+#undef SKINNY_PICK
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess)
         return e;
