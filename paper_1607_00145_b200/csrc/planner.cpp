@@ -533,8 +533,18 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     if (o.split_k > 1) {
         split = std::min<uint32_t>((uint32_t)o.split_k, kslabs);
     } else if (o.split_k == 0 && sm_count > 0 && tiles * 2 <= (uint64_t)sm_count && kslabs >= 8) {
-        uint32_t want = (uint32_t)((2 * (uint64_t)sm_count + tiles - 1) / tiles);
-        split = std::max<uint32_t>(1, std::min<uint32_t>(want, kslabs / 4));
+        // choose the slice count whose (waves of work items) x (slabs per item + a fixed
+        // per-item cost for the epilogue and the reduction) is smallest
+        const uint64_t slots = (uint64_t)sm_count * (path == GETT_PATH_UMMA ? 1 : path == GETT_PATH_FFMA ? 2 : 4);
+        uint64_t best = UINT64_MAX;
+        for (uint32_t s = 1; s <= std::min<uint32_t>(kslabs / 4, 256); ++s) {
+            const uint64_t waves = (tiles * s + slots - 1) / slots;
+            const uint64_t cost = waves * (ceil_div(kslabs, s) + 6) + s / 2;
+            if (cost < best) {
+                best = cost;
+                split = s;
+            }
+        }
     }
     uint32_t slabs_per = ceil_div(kslabs, split);
     split = ceil_div(kslabs, slabs_per); // no empty slice
