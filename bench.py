@@ -250,6 +250,22 @@ def time_contraction(torch, g, con, dtype, alpha, beta, dev, steps, warmup, opts
     return e0.elapsed_time(e1) / 1e3 / steps, info
 
 
+def max_over_ranks(seconds: float, world: int, device) -> float:
+    """Timed-region length of the job: the slowest replica's (all-reduce MAX over ranks)."""
+    if world <= 1:
+        return seconds
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([seconds], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replicas_value(flops_per_replica: float, world: int, sec_per_step: float) -> float:
+    """Whole-job TFLOP/s of `world` independent replicas (no data-path collective)."""
+    return world * flops_per_replica / sec_per_step / 1e12
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -312,14 +328,12 @@ def run_ours(args):
         raise RuntimeError(f"kernel reported status {plan.device_status()}")
     per = np.array([e0.elapsed_time(e1) for e0, e1 in evs]) / 1e3   # seconds per launch
     total = float(per.sum())
+    total = max_over_ranks(total, world, torch.device("cuda", local))
     if world > 1:
-        t = torch.tensor([total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total = float(t.item())
         dist.barrier()
     sec_per_step = total / args.steps
     flops = con.flops()
-    value = world * flops / sec_per_step / 1e12
+    value = replicas_value(flops, world, sec_per_step)
     clocks = clk.summary()
     sm_mhz = clocks["sm_mhz"] or 1965.0
     fp32_peak = _fp32_peak_tflops(sm_mhz)
