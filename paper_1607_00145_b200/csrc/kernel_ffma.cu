@@ -185,6 +185,35 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     const uint32_t swA = tx & 7;
     const uint32_t swB = FN == 8 ? (ty & 7) : ((ty * FN) >> 2) & 7;
 
+    // beta != 0: ask L2 for the old values of this thread's part of C now, so that the
+    // read-modify-write at the end finds them on chip (the request holds no register).
+    // The offset tables were completed before the prologue's first barrier.
+    if (g.beta != 0.f && g.split_k == 1 && stages >= 2) {
+        if (FN == 8 && g.c_vec == 2) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int64_t cm = T->offCM[rows[i]];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int64_t cn = T->offCN[cols[4 * h % FN]];
+                    if (cm >= 0 && cn >= 0)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(g.C + cm + cn));
+                }
+            }
+        } else if (g.c_vec == 1) {
+#pragma unroll
+            for (int j = 0; j < FN; ++j) {
+                const int64_t cn = T->offCN[cols[j]];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int64_t cm = T->offCM[rows[4 * h]];
+                    if (cm >= 0 && cn >= 0)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(g.C + cm + cn));
+                }
+            }
+        }
+    }
+
     // Accumulators are held in pairs so that one packed instruction (two independent
     // round-to-nearest fp32 FMAs, results identical to two scalar fmaf) updates two of
     // them.  Pairs run along rows when A's fragment delivers neighbouring rows together
@@ -215,7 +244,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
         const char* As = reinterpret_cast<const char*>(smem) + (slab % stages) * STAGE;
         const char* Bs = As + TM * TK * 4;
 #pragma unroll
-        for (int k4 = 0; k4 < TK / 4; ++k4) {
+        for (int k4 = 0; k4 < TK / 4 && !(g.debug & 64); ++k4) { // (debug & 64: experiment, no math)
             float a[8][4], b[FN][4];
             if (A_K) {
                 frag_kmajor<8>(As, rows, swA, k4, a);
@@ -283,35 +312,48 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     // ---- unpack: C <- alpha * acc + beta * C (or the raw slice sums under split-K) ----
     const float alpha = g.alpha, beta = g.beta;
     const bool vec_m = g.c_vec == 1;
+    if (g.debug & 2) // experiment: no stores
+        return;
     if (FN == 8 && g.c_vec == 2 && g.split_k == 1) {
-        // four consecutive tile columns are one aligned 16-byte vector of C; the old values
-        // of four rows (eight vectors) are requested together so their latencies overlap
-        int64_t cn[2];
+        // C's stride-1 mode runs along the tile's columns.  The scaled accumulators pass
+        // through shared memory (the stage ring is free now) so that a warp owns whole tile
+        // rows and its 32 lanes cover 128 consecutive columns: the read-modify-write of C
+        // then moves whole runs of C per instruction instead of 16-byte pieces (Eq. 11 as a
+        // transposition).  16-byte groups are XOR-swizzled by (row / 4) % 8: conflict-free
+        // both for the writes (lanes = rows) and for the reads (lanes = column groups).
+        float* S = reinterpret_cast<float*>(smem);
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
-            cn[h] = T->offCN[cols[(4 * h) % FN]];
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t row = rows[i];
 #pragma unroll
-        for (int i0 = 0; i0 < 8; i0 += 4) {
-            float4 old[4][2];
-            float4* dst[4][2];
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t c4 = cols[(4 * h) % FN] >> 2;
+                *reinterpret_cast<float4*>(S + row * TN + ((c4 ^ ((row >> 2) & 7)) << 2)) =
+                    make_float4(alpha * ACC(i, (4 * h) % FN), alpha * ACC(i, (4 * h + 1) % FN),
+                                alpha * ACC(i, (4 * h + 2) % FN), alpha * ACC(i, (4 * h + 3) % FN));
+            }
+        }
+        __syncthreads();
+        const int warp = tid >> 5, lane = tid & 31;
+        const int64_t cn = T->offCN[lane * 4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int64_t cm = T->offCM[rows[i0 + i]];
+        for (int r0 = 0; r0 < 16; r0 += 8) {
+            float4 old[8];
+            float4* dst[8];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    dst[i][h] = (cm >= 0 && cn[h] >= 0) ? reinterpret_cast<float4*>(g.C + cm + cn[h]) : nullptr;
-                    old[i][h] = (beta != 0.f && dst[i][h]) ? __ldcg(dst[i][h]) : make_float4(0, 0, 0, 0);
-                }
+            for (int r = 0; r < 8; ++r) {
+                const int64_t cm = T->offCM[warp * 16 + r0 + r];
+                dst[r] = (cm >= 0 && cn >= 0) ? reinterpret_cast<float4*>(g.C + cm + cn) : nullptr;
+                old[r] = (beta != 0.f && dst[r]) ? __ldcg(dst[r]) : make_float4(0, 0, 0, 0);
             }
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-                    if (dst[i][h])
-                        *dst[i][h] = make_float4(fmaf(beta, old[i][h].x, alpha * ACC(i0 + i, (4 * h) % FN)),
-                                                 fmaf(beta, old[i][h].y, alpha * ACC(i0 + i, (4 * h + 1) % FN)),
-                                                 fmaf(beta, old[i][h].z, alpha * ACC(i0 + i, (4 * h + 2) % FN)),
-                                                 fmaf(beta, old[i][h].w, alpha * ACC(i0 + i, (4 * h + 3) % FN)));
+            for (int r = 0; r < 8; ++r) {
+                const uint32_t row = warp * 16 + r0 + r;
+                const float4 v = *reinterpret_cast<const float4*>(S + row * TN + ((lane ^ ((row >> 2) & 7)) << 2));
+                if (dst[r])
+                    *dst[r] = make_float4(fmaf(beta, old[r].x, v.x), fmaf(beta, old[r].y, v.y),
+                                          fmaf(beta, old[r].z, v.z), fmaf(beta, old[r].w, v.w));
+            }
         }
         return;
     }
