@@ -113,15 +113,15 @@ __device__ __forceinline__ WorkItem decode_work(const GettKernelArgs& g, uint32_
 // VEC_FREE: pieces run along the free dimension (MN-major staging).  Thread gl owns
 //           free-piece fc = gl % FPR of the k rows gl/FPR + KSTEP p; its row offset is
 //           one register per tile, the k offsets come from the group's slab table.
-template <bool VEC_K, int R>
+template <bool VEC_K, int R, int LANES>
 struct OperandLoader {
     static constexpr int FPR = R / 8;                 // pieces per k row (VEC_FREE)
     static constexpr int pow2_floor(int x) { return x >= 64 ? 64 : x >= 32 ? 32 : x >= 16 ? 16 : x >= 8 ? 8 : x >= 4 ? 4 : x >= 2 ? 2 : 1; }
-    static constexpr int KSTEP = pow2_floor(GROUP_LANES / FPR); // k rows per pass (VEC_FREE)
-    static constexpr int RP = GROUP_LANES / 8;                  // rows per pass (VEC_K)
-    static constexpr int ACTIVE = VEC_K ? GROUP_LANES : KSTEP * FPR;
+    static constexpr int KSTEP = pow2_floor(LANES / FPR); // k rows per pass (VEC_FREE)
+    static constexpr int RP = LANES / 8;                  // rows per pass (VEC_K)
+    static constexpr int ACTIVE = VEC_K ? LANES : KSTEP * FPR;
     static constexpr int NP = VEC_K ? (R + RP - 1) / RP : TILE_K / KSTEP;
-    static_assert(ACTIVE <= GROUP_LANES, "tile too wide for one producer group");
+    static_assert(ACTIVE <= LANES, "tile too wide for one producer group");
 
     uint32_t row16;    // VEC_FREE: this thread's row offset (16-byte units), INVALID16 if outside
     uint32_t dst_lane; // byte offset of this thread's piece 0 inside the operand's stage buffer
@@ -132,7 +132,7 @@ struct OperandLoader {
                                                uint32_t* rowTab)
     {
         if (VEC_K) {
-            for (uint32_t r = gl; r < (uint32_t)R; r += GROUP_LANES) {
+            for (uint32_t r = gl; r < (uint32_t)R; r += LANES) {
                 uint32_t v = INVALID16;
                 if (origin + r < D.size) {
                     int64_t x, y;
@@ -179,7 +179,7 @@ struct OperandLoader {
                 }
             }
         } else {
-            if (ACTIVE < GROUP_LANES && gl >= ACTIVE)
+            if (ACTIVE < LANES && gl >= ACTIVE)
                 return;
             const uint32_t fc = gl % FPR, kgroup = gl / FPR;
             const uint32_t dst = stage_dst + dst_lane;
@@ -231,7 +231,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
     int64_t* grp = reinterpret_cast<int64_t*>(S + EPI_DEPTH * 32 * EPI_PITCH);
     const uint32_t s_u32 = ptx::smem_u32(S);
     const float alpha = g.alpha, beta = g.beta;
-    const bool rmw = beta != 0.f;
+    const bool rmw = beta != 0.f && !(g.debug & 128); // (debug & 128: experiment, old C not read)
     // this warp's set handles the CTA's tiles with local number es, es + 2, ...; `j` counts them
     const uint32_t es = warp >> 2, eq = warp & 3;
     const uint32_t ncta = total_work > blockIdx.x ? (total_work - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
@@ -320,7 +320,8 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
                     q.z = fmaf(beta, o.z, q.z);
                     q.w = fmaf(beta, o.w, q.w);
                 }
-                *reinterpret_cast<float4*>(p) = q;
+                if (!(g.debug & 512)) // (debug & 512: experiment, no staging writes)
+                    *reinterpret_cast<float4*>(p) = q;
             }
         }
         if (ch == NCH - 1) { // the accumulator buffer can be overwritten by the set's next tile
@@ -330,15 +331,145 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
         __syncwarp();
         const long long myrow = my_row(j);
 #pragma unroll
-        for (int t = 0; t < 16; ++t) {
+        for (int t = 0; t < 16 && !(g.debug & 256); ++t) { // (debug & 256: experiment, no store phase)
             const uint32_t q = lane + 32 * t, row = q >> 4, s4 = q & 15;
             const long long rc = __shfl_sync(FULL, myrow, row);
             const int64_t cn = grp[(j & 1) * EPI_GROUPS + ch * 16 + s4];
-            if (rc >= 0 && cn >= 0)
+            if (rc >= 0 && cn >= 0 && !(g.debug & 2)) // (debug & 2: experiment, no stores)
                 *reinterpret_cast<float4*>(g.C + rc + cn) =
                     *reinterpret_cast<const float4*>(Sb + row * EPI_PITCH + 4 * s4);
         }
         __syncwarp(); // this staging buffer is free for the next prefetch into it
+    }
+    ptx::cp_async_wait_all();
+}
+
+// The producer role.  A group of LANES threads (index gl inside the group, named barrier
+// gbar) owns the slabs with number it % ng == pg and fills their ring stage.
+template <bool A_VEC_K, bool B_VEC_K, int TILE_N, int TILE_M, int LANES>
+__device__ __forceinline__ void producer_role(const GettKernelArgs& g, const GettTmaMaps& tm, SmemTables* T,
+                                              uint32_t stage0, uint32_t stages, uint32_t total_work,
+                                              volatile int* abort_flag, uint32_t pg, uint32_t ng, uint32_t gl,
+                                              uint32_t gbar)
+{
+    constexpr uint32_t sbytes = stage_bytes(TILE_M, TILE_N);
+    constexpr uint32_t A_STAGE_BYTES = TILE_M * TILE_K * 2;
+    // ------------------------------ producers ------------------------------
+    // Slab number `it` (counted over the CTA's whole work list) belongs to producer
+    // group it % PROD_GROUPS, so PROD_GROUPS slabs are gathered concurrently.  The
+    // ring depth is a multiple of PROD_GROUPS, hence a stage's barriers are always
+    // used by the same group, which therefore observes every one of their phases.
+    uint32_t* kA = T->kTab[pg][0];
+    uint32_t* kB = T->kTab[pg][1];
+    uint32_t* rowA = T->rowTab[pg];
+    uint32_t* rowB = T->rowTab[pg] + 256;
+    OperandLoader<A_VEC_K, TILE_M, LANES> la;
+    OperandLoader<B_VEC_K, TILE_N, LANES> lb;
+    const char* baseA = static_cast<const char*>(g.A);
+    const char* baseB = static_cast<const char*>(g.B);
+    // An operand whose tile is a box of a <= 5-D tensor map is fetched by TMA: thread 0
+    // of the group issues the copies and the stage's barrier counts their bytes.
+    const bool tmaA = tm.use_a != 0, tmaB = tm.use_b != 0, all_tma = tmaA && tmaB;
+    const uint32_t tma_bytes = (tmaA ? A_STAGE_BYTES : 0) + (tmaB ? TILE_N * TILE_K * 2 : 0);
+    int32_t fa[5] = {0, 0, 0, 0, 0}, fb[5] = {0, 0, 0, 0, 0}; // digit indices of the tile origin
+    uint32_t first = 0; // slab number of the current work item's first slab
+    bool alive = true;
+    for (uint32_t w = blockIdx.x; w < total_work && pg < ng; w += gridDim.x) {
+        const WorkItem wi = decode_work(g, w, TILE_M);
+        // my group's first slab in this item: smallest j with (first + j) % ng == pg
+        uint32_t j = (pg + ng - first % ng) % ng;
+        if (j < wi.nslab) {
+            if (!all_tma)
+                ptx::named_barrier(gbar, LANES); // the group is done with the previous tables
+            if (!tmaA)
+                la.setup_tile(g.M, wi.m0, gl, rowA);
+            else if (gl == 0)
+                gett_digit_indices(g.M, wi.m0, fa, 5);
+            if (!tmaB)
+                lb.setup_tile(g.N, wi.n0, gl, rowB);
+            else if (gl == 0)
+                gett_digit_indices(g.N, wi.n0, fb, 5);
+        }
+        const bool tile_full = wi.m0 + TILE_M <= g.M.size && wi.n0 + TILE_N <= g.N.size;
+        for (; j < wi.nslab; j += ng) {
+            const uint32_t it = first + j;
+            const uint32_t k0 = wi.kbeg + j * TILE_K;
+            if (!all_tma) {
+                ptx::named_barrier(gbar, LANES); // previous slab's k table no longer read
+                if (gl < TILE_K) {
+                    const uint32_t k = k0 + gl;
+                    uint32_t xa = INVALID16, xb = INVALID16;
+                    if (k < wi.kend) {
+                        int64_t x, y;
+                        gett_decompose(g.K, k, x, y);
+                        xa = (uint32_t)(x >> 3);
+                        xb = (uint32_t)(y >> 3);
+                    }
+                    kA[gl] = xa;
+                    kB[gl] = xb;
+                }
+                ptx::named_barrier(gbar, LANES); // tables (rows and k) complete
+            }
+            const uint32_t s = it % stages;
+            // After a timeout a thread keeps walking the loop (so its group's named
+            // barriers stay matched) but neither waits nor copies any more.
+            if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->empty[s]), ((it / stages) & 1) ^ 1, abort_flag))
+                alive = false;
+            if (!alive)
+                continue;
+            const uint32_t sa = stage0 + s * sbytes;
+            const uint32_t fullbar = ptx::smem_u32(&T->full[s]);
+            if (gl == 0 && tma_bytes && !(g.debug & 4)) {
+                int32_t kd[5] = {0, 0, 0, 0, 0}, c[5];
+                gett_digit_indices(g.K, k0, kd, 5);
+                ptx::mbar_expect_tx(fullbar, tma_bytes);
+                if (tmaA) {
+#pragma unroll
+                    for (int i = 0; i < 5; ++i)
+                        c[i] = tm.which_a[i] ? kd[tm.digit_a[i]] : fa[tm.digit_a[i]];
+                    if (A_VEC_K) {
+                        ptx::tma_load(sa, tm.map_a, fullbar, tm.rank_a, c);
+                    } else {
+#pragma unroll
+                        for (int b = 0; b < TILE_M / 64; ++b) {
+                            ptx::tma_load(sa + b * MN_BLOCK_BYTES, tm.map_a, fullbar, tm.rank_a, c);
+                            c[0] += 64;
+                        }
+                    }
+                }
+                if (tmaB) {
+#pragma unroll
+                    for (int i = 0; i < 5; ++i)
+                        c[i] = tm.which_b[i] ? kd[tm.digit_b[i]] : fb[tm.digit_b[i]];
+                    if (B_VEC_K) {
+                        ptx::tma_load(sa + A_STAGE_BYTES, tm.map_b, fullbar, tm.rank_b, c);
+                    } else {
+#pragma unroll
+                        for (int b = 0; b < TILE_N / 64; ++b) {
+                            ptx::tma_load(sa + A_STAGE_BYTES + b * MN_BLOCK_BYTES, tm.map_b, fullbar,
+                                          tm.rank_b, c);
+                            c[0] += 64;
+                        }
+                    }
+                }
+            }
+            if (g.debug & 4) {
+                // experiment switch: no copies at all (measures the rest of the pipeline)
+            } else if (tile_full && k0 + TILE_K <= wi.kend) {
+                if (!tmaA)
+                    la.template load_slab<true>(baseA, sa, kA, rowA, gl);
+                if (!tmaB)
+                    lb.template load_slab<true>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+            } else {
+                if (!tmaA)
+                    la.template load_slab<false>(baseA, sa, kA, rowA, gl);
+                if (!tmaB)
+                    lb.template load_slab<false>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+            }
+            // full[s] hears from this thread when its copies for the slab have landed
+            ptx::cp_async_mbar_arrive_noinc(fullbar);
+        }
+        first += wi.nslab;
     }
     ptx::cp_async_wait_all();
 }
@@ -365,7 +496,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < stages; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&T->full[s]), GROUP_LANES); // the slab's producer group
+            ptx::mbar_init(ptx::smem_u32(&T->full[s]), g.prod_groups == 1 ? PROD_THREADS : GROUP_LANES); // the slab's producers
             ptx::mbar_init(ptx::smem_u32(&T->empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -385,128 +516,20 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
     const uint32_t tmem_base = T->tmem_base;
 
     if (warp >= PROD_WARP0) {
-        // ------------------------------ producers ------------------------------
-        // Slab number `it` (counted over the CTA's whole work list) belongs to producer
-        // group it % PROD_GROUPS, so PROD_GROUPS slabs are gathered concurrently.  The
-        // ring depth is a multiple of PROD_GROUPS, hence a stage's barriers are always
-        // used by the same group, which therefore observes every one of their phases.
-        const uint32_t pg = (warp - PROD_WARP0) / WARPS_PER_GROUP;
-        const uint32_t ng = (uint32_t)g.prod_groups; // groups in use: divides the ring depth
-        const uint32_t gl = threadIdx.x - (PROD_WARP0 + pg * WARPS_PER_GROUP) * 32;
-        const uint32_t gbar = 3 + pg; // named barrier of this group
-        uint32_t* kA = T->kTab[pg][0];
-        uint32_t* kB = T->kTab[pg][1];
-        uint32_t* rowA = T->rowTab[pg];
-        uint32_t* rowB = T->rowTab[pg] + 256;
-        OperandLoader<A_VEC_K, TILE_M> la;
-        OperandLoader<B_VEC_K, TILE_N> lb;
-        const char* baseA = static_cast<const char*>(g.A);
-        const char* baseB = static_cast<const char*>(g.B);
-        // An operand whose tile is a box of a <= 5-D tensor map is fetched by TMA: thread 0
-        // of the group issues the copies and the stage's barrier counts their bytes.
-        const bool tmaA = tm.use_a != 0, tmaB = tm.use_b != 0, all_tma = tmaA && tmaB;
-        const uint32_t tma_bytes = (tmaA ? A_STAGE_BYTES : 0) + (tmaB ? TILE_N * TILE_K * 2 : 0);
-        int32_t fa[5] = {0, 0, 0, 0, 0}, fb[5] = {0, 0, 0, 0, 0}; // digit indices of the tile origin
-        uint32_t first = 0; // slab number of the current work item's first slab
-        bool alive = true;
-        for (uint32_t w = blockIdx.x; w < total_work && pg < ng; w += gridDim.x) {
-            const WorkItem wi = decode_work(g, w, TILE_M);
-            // my group's first slab in this item: smallest j with (first + j) % ng == pg
-            uint32_t j = (pg + ng - first % ng) % ng;
-            if (j < wi.nslab) {
-                if (!all_tma)
-                    ptx::named_barrier(gbar, GROUP_LANES); // the group is done with the previous tables
-                if (!tmaA)
-                    la.setup_tile(g.M, wi.m0, gl, rowA);
-                else if (gl == 0)
-                    gett_digit_indices(g.M, wi.m0, fa, 5);
-                if (!tmaB)
-                    lb.setup_tile(g.N, wi.n0, gl, rowB);
-                else if (gl == 0)
-                    gett_digit_indices(g.N, wi.n0, fb, 5);
-            }
-            const bool tile_full = wi.m0 + TILE_M <= g.M.size && wi.n0 + TILE_N <= g.N.size;
-            for (; j < wi.nslab; j += ng) {
-                const uint32_t it = first + j;
-                const uint32_t k0 = wi.kbeg + j * TILE_K;
-                if (!all_tma) {
-                    ptx::named_barrier(gbar, GROUP_LANES); // previous slab's k table no longer read
-                    if (gl < TILE_K) {
-                        const uint32_t k = k0 + gl;
-                        uint32_t xa = INVALID16, xb = INVALID16;
-                        if (k < wi.kend) {
-                            int64_t x, y;
-                            gett_decompose(g.K, k, x, y);
-                            xa = (uint32_t)(x >> 3);
-                            xb = (uint32_t)(y >> 3);
-                        }
-                        kA[gl] = xa;
-                        kB[gl] = xb;
-                    }
-                    ptx::named_barrier(gbar, GROUP_LANES); // tables (rows and k) complete
-                }
-                const uint32_t s = it % stages;
-                // After a timeout a thread keeps walking the loop (so its group's named
-                // barriers stay matched) but neither waits nor copies any more.
-                if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->empty[s]), ((it / stages) & 1) ^ 1, abort_flag))
-                    alive = false;
-                if (!alive)
-                    continue;
-                const uint32_t sa = stage0 + s * sbytes;
-                const uint32_t fullbar = ptx::smem_u32(&T->full[s]);
-                if (gl == 0 && tma_bytes && !(g.debug & 4)) {
-                    int32_t kd[5] = {0, 0, 0, 0, 0}, c[5];
-                    gett_digit_indices(g.K, k0, kd, 5);
-                    ptx::mbar_expect_tx(fullbar, tma_bytes);
-                    if (tmaA) {
-#pragma unroll
-                        for (int i = 0; i < 5; ++i)
-                            c[i] = tm.which_a[i] ? kd[tm.digit_a[i]] : fa[tm.digit_a[i]];
-                        if (A_VEC_K) {
-                            ptx::tma_load(sa, tm.map_a, fullbar, tm.rank_a, c);
-                        } else {
-#pragma unroll
-                            for (int b = 0; b < TILE_M / 64; ++b) {
-                                ptx::tma_load(sa + b * MN_BLOCK_BYTES, tm.map_a, fullbar, tm.rank_a, c);
-                                c[0] += 64;
-                            }
-                        }
-                    }
-                    if (tmaB) {
-#pragma unroll
-                        for (int i = 0; i < 5; ++i)
-                            c[i] = tm.which_b[i] ? kd[tm.digit_b[i]] : fb[tm.digit_b[i]];
-                        if (B_VEC_K) {
-                            ptx::tma_load(sa + A_STAGE_BYTES, tm.map_b, fullbar, tm.rank_b, c);
-                        } else {
-#pragma unroll
-                            for (int b = 0; b < TILE_N / 64; ++b) {
-                                ptx::tma_load(sa + A_STAGE_BYTES + b * MN_BLOCK_BYTES, tm.map_b, fullbar,
-                                              tm.rank_b, c);
-                                c[0] += 64;
-                            }
-                        }
-                    }
-                }
-                if (g.debug & 4) {
-                    // experiment switch: no copies at all (measures the rest of the pipeline)
-                } else if (tile_full && k0 + TILE_K <= wi.kend) {
-                    if (!tmaA)
-                        la.template load_slab<true>(baseA, sa, kA, rowA, gl);
-                    if (!tmaB)
-                        lb.template load_slab<true>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
-                } else {
-                    if (!tmaA)
-                        la.template load_slab<false>(baseA, sa, kA, rowA, gl);
-                    if (!tmaB)
-                        lb.template load_slab<false>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
-                }
-                // full[s] hears from this thread when its copies for the slab have landed
-                ptx::cp_async_mbar_arrive_noinc(fullbar);
-            }
-            first += wi.nslab;
+        // Producers.  With a ring of one stage (tiles of a single slab) all producer warps
+        // form one wide group and share every slab; otherwise groups of WARPS_PER_GROUP
+        // warps own whole slabs round-robin.  The ring depth is a multiple of the group
+        // count, so a stage's barriers are always used by the same group.
+        const uint32_t ng = (uint32_t)g.prod_groups;
+        if (ng == 1) {
+            producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, PROD_THREADS>(
+                g, tm, T, stage0, stages, total_work, abort_flag, 0, 1, threadIdx.x - PROD_WARP0 * 32, 3);
+        } else {
+            const uint32_t pg = (warp - PROD_WARP0) / WARPS_PER_GROUP;
+            producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, GROUP_LANES>(
+                g, tm, T, stage0, stages, total_work, abort_flag, pg, ng,
+                threadIdx.x - (PROD_WARP0 + pg * WARPS_PER_GROUP) * 32, 3 + pg);
         }
-        ptx::cp_async_wait_all();
     } else if (warp == MMA_WARP) {
         // ------------------------------ MMA issuer -----------------------------
         if (lane == 0) {
