@@ -98,8 +98,8 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* A,
 gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, size_t capacity);
 
 // Geometry of the tensor-core kernel (kernel_umma.cu), needed by the planner.
-int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged);
-int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged);
+int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged_cv); // staged_cv: 0, 1 or 8
+int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged_cv);
 int gett_umma_block();
 int gett_umma_prod_groups(int stages); // producer groups in use; must divide the ring depth
 

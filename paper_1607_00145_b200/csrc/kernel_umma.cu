@@ -54,8 +54,12 @@ constexpr int RASTER_M = 16;               // tile rows per rasterisation panel
 constexpr int EPI_PITCH = 68;              // floats per staged row: 64 + 4 keeps 128-bit accesses conflict-free
 constexpr int EPI_GROUPS = 256 / 4;          // 16-byte groups per tile row, at most
 constexpr int EPI_DEPTH = 2;                 // staging buffers per warp: old C is fetched EPI_DEPTH-1 chunks ahead
-constexpr int EPI_WARP_BYTES = EPI_DEPTH * (32 * EPI_PITCH * 4 + EPI_GROUPS * 8); // chunk buffers + group tables
-constexpr int EPI_STAGE_BYTES = NUM_EPI_WARPS * EPI_WARP_BYTES;
+// staging bytes of one epilogue warp: chunk buffers + group tables (cv as in StagedShape)
+__host__ __device__ constexpr int epi_pitch(int tile_n, int cv) { return cv == 8 ? tile_n / 4 + 4 : EPI_PITCH; }
+__host__ __device__ constexpr int epi_warp_bytes(int tile_n, int cv)
+{
+    return EPI_DEPTH * (32 * epi_pitch(tile_n, cv) * 4 + EPI_GROUPS * 8);
+}
 
 constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-byte-unit offset tables
 
@@ -200,19 +204,34 @@ struct OperandLoader {
 };
 
 // ---- staged epilogue (Eq. 11 as a transposition through shared memory) ----
-// Within a 64-column chunk of the accumulator the columns are re-ordered into "slots"
-// so that four consecutive slots are four consecutive floats of C:
-//   CV == 1: the tile's columns already run along C's stride-1 mode (slot = column)
-//   CV == 8: the first N digit is the 8-wide piece of B's stride-1 mode and the second
-//            digit is C's stride-1 mode, i.e. column = a + 8 n'  ->  slot = 8 a + n'
-template <int CV>
-__device__ __forceinline__ uint32_t col_of_slot(uint32_t slot)
-{
-    return CV == 1 ? slot : (slot >> 3) + ((slot & 7) << 3);
-}
+// The accumulator is walked in chunks of up to 64 columns, and inside a chunk the columns
+// are re-ordered into "slots" so that four consecutive slots are four consecutive floats of C:
+//   CV == 1: the tile's columns already run along C's stride-1 mode; a chunk is 64
+//            consecutive columns and slot = column.
+//   CV == 8: the first N digit a (extent 8) is the 8-wide piece of B's stride-1 mode and the
+//            second digit is C's stride-1 mode, i.e. column = a + 8 p with p running along
+//            C.  A chunk is a pair of a values over ALL p of the tile (TILE_N / 4 columns,
+//            read from tensor memory two at a time with a stride of 8 columns), slot =
+//            (a & 1) * TILE_N/8 + p: each row of the chunk is two runs of TILE_N/8
+//            consecutive floats of C, so the reads and writes of C cover whole runs of its
+//            stride-1 mode instead of 32-byte pieces of them.
+template <int TILE_N, int CV>
+struct StagedShape {
+    static constexpr uint32_t NP = TILE_N / 8;                      // CV == 8: pieces (values of p) per tile
+    static constexpr uint32_t NCH = CV == 8 ? 4 : TILE_N / 64;      // chunks per tile
+    static constexpr uint32_t SLOTS = CV == 8 ? TILE_N / 4 : 64;    // slots per row of a chunk
+    static constexpr uint32_t PITCH = epi_pitch(TILE_N, CV);        // SLOTS + 4 keeps 128-bit accesses conflict-free
+    static constexpr uint32_t GPR = SLOTS / 4;                      // 16-byte groups per row of a chunk
+    static_assert(PITCH == SLOTS + 4, "staging pitch");
+    // first tile column of the 16-byte group number e (e = chunk * GPR + group in the row)
+    static __device__ __forceinline__ uint32_t col_of_group(uint32_t e)
+    {
+        return CV == 8 ? e / (NP / 4) + 32 * (e % (NP / 4)) : 4 * e;
+    }
+};
 
-// Staged epilogue, run by each epilogue warp on its own 32 tile rows, one 64-column
-// chunk at a time, software-pipelined one chunk ahead (across tile boundaries):
+// Staged epilogue, run by each epilogue warp on its own 32 tile rows, one chunk at a
+// time, software-pipelined one chunk ahead (across tile boundaries):
 //   prepare(c+1): (first chunk of a tile) C offsets of my row and of the tile's 16-byte
 //                 groups; if beta != 0, cp.async the old C values of chunk c+1 into the
 //                 other staging buffer -- the reads of C never wait for the accumulator
@@ -225,10 +244,11 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
                                                 uint32_t tmem_base, uint32_t warp, uint32_t lane,
                                                 uint32_t total_work, volatile int* abort_flag)
 {
-    constexpr uint32_t NCH = TILE_N / 64;
+    using Sh = StagedShape<TILE_N, CV>;
+    constexpr uint32_t NCH = Sh::NCH, PITCH = Sh::PITCH, GPR = Sh::GPR, NP = Sh::NP;
     constexpr uint32_t FULL = 0xFFFFFFFFu;
-    float* S = reinterpret_cast<float*>(epi_smem + warp * EPI_WARP_BYTES);
-    int64_t* grp = reinterpret_cast<int64_t*>(S + EPI_DEPTH * 32 * EPI_PITCH);
+    float* S = reinterpret_cast<float*>(epi_smem + warp * epi_warp_bytes(TILE_N, CV));
+    int64_t* grp = reinterpret_cast<int64_t*>(S + EPI_DEPTH * 32 * PITCH);
     const uint32_t s_u32 = ptx::smem_u32(S);
     const float alpha = g.alpha, beta = g.beta;
     const bool rmw = beta != 0.f && !(g.debug & 128); // (debug & 128: experiment, old C not read)
@@ -253,7 +273,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
                 rowC_0 = (j & 1) ? rowC_0 : rc;
                 rowC_1 = (j & 1) ? rc : rowC_1;
                 for (uint32_t e = lane; e < TILE_N / 4; e += 32) {
-                    const uint32_t col = (e >> 4) * 64 + col_of_slot<CV>(4 * (e & 15));
+                    const uint32_t col = Sh::col_of_group(e);
                     int64_t x, y = -1;
                     if (wi.n0 + col < g.N.size)
                         gett_decompose(g.N, wi.n0 + col, x, y);
@@ -263,18 +283,55 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
             }
             if (rmw) {
                 const long long myrow = my_row(j);
-                const uint32_t dst = s_u32 + (cj & 1) * (32 * EPI_PITCH * 4);
+                const uint32_t dst = s_u32 + (cj & 1) * (32 * PITCH * 4);
+                const int64_t* gch = grp + (j & 1) * EPI_GROUPS + ch * GPR;
+                // four copies at a time: offsets first, then the copies back to back
 #pragma unroll
-                for (int t = 0; t < 16; ++t) {
-                    const uint32_t q = lane + 32 * t, row = q >> 4, s4 = q & 15;
-                    const long long rc = __shfl_sync(FULL, myrow, row);
-                    const int64_t cn = grp[(j & 1) * EPI_GROUPS + ch * 16 + s4];
-                    const bool ok = rc >= 0 && cn >= 0;
-                    ptx::cp_async_16(dst + (row * EPI_PITCH + 4 * s4) * 4, ok ? g.C + rc + cn : g.C, ok ? 16u : 0u);
+                for (uint32_t t0 = 0; t0 < GPR; t0 += 4) {
+                    const float* src[4];
+                    uint32_t d[4];
+#pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k) {
+                        const uint32_t q = lane + 32 * (t0 + k), row = q / GPR, gi = q - row * GPR;
+                        const long long rc = __shfl_sync(FULL, myrow, row);
+                        const int64_t cn = gch[gi];
+                        src[k] = (rc >= 0 && cn >= 0) ? g.C + rc + cn : nullptr;
+                        d[k] = dst + (row * PITCH + 4 * gi) * 4;
+                    }
+#pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k)
+                        ptx::cp_async_16(d[k], src[k] ? src[k] : g.C, src[k] ? 16u : 0u);
                 }
             }
         }
         ptx::cp_async_commit();
+    };
+
+    // alpha * acc (+ beta * old, read from the same staging slots) -> staging.  Four
+    // 16-byte groups at a time: the old values are read first, then the results written,
+    // so that the loads do not queue up behind the stores to the same buffer.
+    auto combine4 = [&](float* const (&p)[4], float4 (&q)[4]) {
+        float4 o[4];
+        if (rmw) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                o[k] = *reinterpret_cast<const float4*>(p[k]);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            q[k].x *= alpha;
+            q[k].y *= alpha;
+            q[k].z *= alpha;
+            q[k].w *= alpha;
+            if (rmw) {
+                q[k].x = fmaf(beta, o[k].x, q[k].x);
+                q[k].y = fmaf(beta, o[k].y, q[k].y);
+                q[k].z = fmaf(beta, o[k].z, q[k].z);
+                q[k].w = fmaf(beta, o[k].w, q[k].w);
+            }
+            if (!(g.debug & 512)) // (debug & 512: experiment, no staging writes)
+                *reinterpret_cast<float4*>(p[k]) = q[k];
+        }
     };
 
     prepare(0);
@@ -288,40 +345,57 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
                 break;
             ptx::tc_fence_after();
         }
-        float* Sb = S + (ci & 1) * (32 * EPI_PITCH);
-        float* Srow = Sb + lane * EPI_PITCH;
-        const uint32_t taddr = tmem_base + ((eq * 32u) << 16) + buf * 256 + ch * 64;
+        float* Sb = S + (ci & 1) * (32 * PITCH);
+        float* Srow = Sb + lane * PITCH;
+        const uint32_t tacc = tmem_base + ((eq * 32u) << 16) + buf * 256;
+        if (CV == 1) {
 #pragma unroll
-        for (uint32_t h = 0; h < 2; ++h) {
-            uint32_t v[32];
-            ptx::tmem_ld_32x32(taddr + h * 32, v);
-            ptx::tmem_wait_ld();
+            for (uint32_t h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                ptx::tmem_ld_32x32(tacc + ch * 64 + h * 32, v);
+                ptx::tmem_wait_ld();
 #pragma unroll
-            for (int a = 0; a < 8; ++a) {
-                float4 q;
-                float* p;
-                if (CV == 1) {
-                    q = make_float4(__uint_as_float(v[4 * a]), __uint_as_float(v[4 * a + 1]),
-                                    __uint_as_float(v[4 * a + 2]), __uint_as_float(v[4 * a + 3]));
-                    p = Srow + h * 32 + 4 * a;
-                } else {
-                    q = make_float4(__uint_as_float(v[a]), __uint_as_float(v[a + 8]),
-                                    __uint_as_float(v[a + 16]), __uint_as_float(v[a + 24]));
-                    p = Srow + a * 8 + h * 4;
+                for (int u0 = 0; u0 < 8; u0 += 4) {
+                    float* p[4];
+                    float4 q[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int u = u0 + k;
+                        p[k] = Srow + h * 32 + 4 * u;
+                        q[k] = make_float4(__uint_as_float(v[4 * u]), __uint_as_float(v[4 * u + 1]),
+                                           __uint_as_float(v[4 * u + 2]), __uint_as_float(v[4 * u + 3]));
+                    }
+                    combine4(p, q);
                 }
-                q.x *= alpha;
-                q.y *= alpha;
-                q.z *= alpha;
-                q.w *= alpha;
-                if (rmw) {
-                    const float4 o = *reinterpret_cast<const float4*>(p);
-                    q.x = fmaf(beta, o.x, q.x);
-                    q.y = fmaf(beta, o.y, q.y);
-                    q.z = fmaf(beta, o.z, q.z);
-                    q.w = fmaf(beta, o.w, q.w);
+            }
+        } else {
+            // columns 2 ch + aa + 8 p: half of the tile's p values at a time
+            constexpr uint32_t HP = NP / 2;
+            static_assert(HP % 4 == 0 && HP <= 16, "tile widths 64, 128, 192, 256");
+#pragma unroll
+            for (uint32_t h = 0; h < 2; ++h) {
+                uint32_t v[2 * HP];
+#pragma unroll
+                for (uint32_t i = 0; i < HP; ++i)
+                    ptx::tmem_ld_32x2(tacc + 2 * ch + 8 * (h * HP + i), v[2 * i], v[2 * i + 1]);
+                ptx::tmem_wait_ld();
+                // 2 * HP / 4 groups: group u covers a = 2 ch + u / (HP / 4), p = h HP + 4 (u % (HP / 4)) ...
+                constexpr uint32_t NG = HP / 2, Q = HP / 4;
+                static_assert(NG % 2 == 0, "groups are combined two or four at a time");
+#pragma unroll
+                for (uint32_t u0 = 0; u0 < NG; u0 += 4) {
+                    float* p[4];
+                    float4 q[4];
+#pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k) {
+                        const uint32_t u = u0 + k < NG ? u0 + k : NG - 1; // (NG = 2 or 6: the tail repeats the last group)
+                        const uint32_t aa = u / Q, i4 = u % Q;
+                        p[k] = Srow + aa * NP + h * HP + 4 * i4;
+                        q[k] = make_float4(__uint_as_float(v[8 * i4 + aa]), __uint_as_float(v[8 * i4 + 2 + aa]),
+                                           __uint_as_float(v[8 * i4 + 4 + aa]), __uint_as_float(v[8 * i4 + 6 + aa]));
+                    }
+                    combine4(p, q);
                 }
-                if (!(g.debug & 512)) // (debug & 512: experiment, no staging writes)
-                    *reinterpret_cast<float4*>(p) = q;
             }
         }
         if (ch == NCH - 1) { // the accumulator buffer can be overwritten by the set's next tile
@@ -330,14 +404,24 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
         }
         __syncwarp();
         const long long myrow = my_row(j);
+        const int64_t* gch = grp + (j & 1) * EPI_GROUPS + ch * GPR;
+        // four groups at a time: staging reads first, then the global stores
 #pragma unroll
-        for (int t = 0; t < 16 && !(g.debug & 256); ++t) { // (debug & 256: experiment, no store phase)
-            const uint32_t q = lane + 32 * t, row = q >> 4, s4 = q & 15;
-            const long long rc = __shfl_sync(FULL, myrow, row);
-            const int64_t cn = grp[(j & 1) * EPI_GROUPS + ch * 16 + s4];
-            if (rc >= 0 && cn >= 0 && !(g.debug & 2)) // (debug & 2: experiment, no stores)
-                *reinterpret_cast<float4*>(g.C + rc + cn) =
-                    *reinterpret_cast<const float4*>(Sb + row * EPI_PITCH + 4 * s4);
+        for (uint32_t t0 = 0; t0 < GPR && !(g.debug & 256); t0 += 4) { // (debug & 256: experiment, no store phase)
+            float4 val[4];
+            float* dstp[4];
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k) {
+                const uint32_t q = lane + 32 * (t0 + k), row = q / GPR, gi = q - row * GPR;
+                const long long rc = __shfl_sync(FULL, myrow, row);
+                const int64_t cn = gch[gi];
+                dstp[k] = (rc >= 0 && cn >= 0 && !(g.debug & 2)) ? g.C + rc + cn : nullptr; // (debug & 2: no stores)
+                val[k] = *reinterpret_cast<const float4*>(Sb + row * PITCH + 4 * gi);
+            }
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k)
+                if (dstp[k])
+                    *reinterpret_cast<float4*>(dstp[k]) = val[k];
         }
         __syncwarp(); // this staging buffer is free for the next prefetch into it
     }
@@ -689,15 +773,16 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
 
 } // namespace
 
-int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged)
+int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged_cv)
 {
     return 1024 + stages * (int)stage_bytes((uint32_t)tile_m, (uint32_t)tile_n) + (int)sizeof(SmemTables) +
-           (staged ? EPI_STAGE_BYTES : 0);
+           (staged_cv ? NUM_EPI_WARPS * epi_warp_bytes(tile_n, staged_cv) : 0);
 }
 
-int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged)
+int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged_cv)
 {
-    int s = (smem_limit - 1024 - (int)sizeof(SmemTables) - (staged ? EPI_STAGE_BYTES : 0)) /
+    int s = (smem_limit - 1024 - (int)sizeof(SmemTables) -
+             (staged_cv ? NUM_EPI_WARPS * epi_warp_bytes(tile_n, staged_cv) : 0)) /
             (int)stage_bytes((uint32_t)tile_m, (uint32_t)tile_n);
     s = s > MAX_STAGES ? MAX_STAGES : s;
     return s >= PROD_GROUPS ? s - s % PROD_GROUPS : s; // a stage is always served by the same group

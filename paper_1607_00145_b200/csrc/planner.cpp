@@ -502,15 +502,15 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         }
         if (tmh == 256 && (tn != 256 || staged))
             return GETT_ERR_UNSUPPORTED;
-        int st = o.stages ? o.stages : gett_umma_max_stages(tmh, tn, smem_limit, staged);
-        if (st < 1 || st > gett_umma_max_stages(tmh, tn, smem_limit, staged) || st % gett_umma_prod_groups(st))
+        int st = o.stages ? o.stages : gett_umma_max_stages(tmh, tn, smem_limit, staged_cv);
+        if (st < 1 || st > gett_umma_max_stages(tmh, tn, smem_limit, staged_cv) || st % gett_umma_prod_groups(st))
             return GETT_ERR_UNSUPPORTED;
         info.tile_m = tmh;
         info.tile_n = tn;
         info.tile_k = 64;
         info.stages = st;
         info.block = gett_umma_block();
-        info.smem_bytes = gett_umma_smem_bytes(tmh, tn, st, staged);
+        info.smem_bytes = gett_umma_smem_bytes(tmh, tn, st, staged_cv);
         if (!(p->debug & 32)) { // (debug & 32: experiment switch, gather even where TMA applies)
             make_tma_recipe(p->M, true, p->K, true, info.loader_a, (uint32_t)tmh, p->tma_a);
             make_tma_recipe(p->N, true, p->K, false, info.loader_b, (uint32_t)tn, p->tma_b);
