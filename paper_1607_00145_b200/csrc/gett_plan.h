@@ -44,8 +44,9 @@ struct GettKernelArgs {
     int32_t tile_n;       // tile width of the tensor-core / FFMA kernels
     int32_t stages;       // depth of the shared-memory ring
     int32_t epilogue;     // gett_epilogue_t
-    int32_t c_vec;        // direct epilogue: 1 = four consecutive tile rows are one aligned 16-byte
-                          // vector of C; staged epilogue: column-to-slot pattern (1 or 8)
+    int32_t c_vec;        // four consecutive tile rows (1) or columns (2) are one aligned 16-byte
+                          // vector of C; column-to-slot pattern of the staged epilogues: 1 or 8
+                          // (tensor-core kernel), 4 (fp32 kernel: column = a + 4 p, p along C)
     int32_t debug;        // opts.reserved[0]: experiment switches, 0 in normal use
     int32_t prod_groups;  // producer groups the tensor-core kernel uses (divides stages)
 };
@@ -104,7 +105,7 @@ int gett_umma_block();
 int gett_umma_prod_groups(int stages); // producer groups in use; must divide the ring depth
 
 // Geometry of the fp32 kernel (kernel_ffma.cu).
-int gett_ffma_smem_bytes(int tile_n, int stages);
+int gett_ffma_smem_bytes(int tile_m, int tile_n, int stages);
 
 // fp32 kernel for N <= 32, K <= gett_ffma_skinny_max_k(), A K-major (kernel_ffma_skinny.cu).
 int gett_ffma_skinny_smem_bytes(int N, int K);

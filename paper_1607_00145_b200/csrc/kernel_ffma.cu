@@ -1,7 +1,7 @@
 // Strict-fp32 contraction kernel: 16-byte cp.async gathers, register-blocked FFMA.
 //
-// One CTA of 256 threads owns a 128 x TN tile of the fused (M, N) output and walks its
-// K range in slabs of 32 through a ring of shared-memory stages (Listing 4 with the
+// One CTA of 2 TM threads owns a TM x TN tile (TM = 128 or 64) of the fused (M, N) output
+// and walks its K range in slabs of 32 through a ring of shared-memory stages (Listing 4 with the
 // m-/n-loops spread over the grid).  Packing (Eq. 9 / Eq. 10) is the gather of
 // 16-byte pieces of the A and B sub-tensors into one of two shared layouts:
 //   stride-1 mode free  ("VEC_FREE") -> [k][row]  rows contiguous, as the FMA loop reads it
@@ -21,10 +21,10 @@
 
 namespace {
 
-constexpr int TM = 128, TK = 32, NT = 256;
+constexpr int TK = 32;
 constexpr uint32_t INVALID16 = 0xFFFFFFFFu;
 
-template <int TN>
+template <int TM, int TN>
 struct FfmaSmem {
     int64_t offCM[TM];
     int64_t offCN[TN];
@@ -33,11 +33,11 @@ struct FfmaSmem {
     uint32_t kTab[2][2][TK]; // [parity][A/B][k] offsets of a slab's k, in elements
 };
 
-template <int TN>
+template <int TM, int TN>
 __host__ __device__ constexpr int ffma_stage_bytes() { return (TM + TN) * TK * 4; }
 
-// Gather one operand slab: R rows x 32 k.  L is the operand's gett_loader_t.
-template <int L, int R>
+// Gather one operand slab: R rows x 32 k, by NT threads.  L is the operand's gett_loader_t.
+template <int L, int R, int NT>
 __device__ __forceinline__ void load_operand(const char* __restrict__ base, uint32_t dst,
                                              const uint32_t* rowTab, const uint32_t* kTab, int tid,
                                              bool k_fastest)
@@ -63,7 +63,7 @@ __device__ __forceinline__ void load_operand(const char* __restrict__ base, uint
         const uint32_t k1 = kTab[kc * 4];
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
-            const uint32_t m = (tid >> 3) + 32 * p;
+            const uint32_t m = (tid >> 3) + (NT / 8) * p;
             if (PIECES % NT != 0 && m >= (uint32_t)R)
                 break;
             const uint32_t r1 = rowTab[m];
@@ -102,15 +102,16 @@ __device__ __forceinline__ void frag_kmajor(const char* tile, const uint32_t (&r
     }
 }
 
-template <int LA, int LB, int TN>
-__global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant__ GettKernelArgs g)
+template <int LA, int LB, int TN, int TM>
+__global__ void __launch_bounds__(2 * TM, 256 / TM) gett_ffma_kernel(const __grid_constant__ GettKernelArgs g)
 {
+    constexpr int NT = 2 * TM;
     constexpr bool A_K = LA == GETT_LOAD_VEC_K, B_K = LB == GETT_LOAD_VEC_K; // staged [row][k]
     constexpr int FN = TN / 16;                 // columns per thread (8 or 2)
-    constexpr int STAGE = ffma_stage_bytes<TN>();
+    constexpr int STAGE = ffma_stage_bytes<TM, TN>();
     extern __shared__ __align__(128) uint8_t smem[];
     const int stages = g.stages;
-    FfmaSmem<TN>* T = reinterpret_cast<FfmaSmem<TN>*>(smem + stages * STAGE);
+    FfmaSmem<TM, TN>* T = reinterpret_cast<FfmaSmem<TM, TN>*>(smem + stages * STAGE);
     const uint32_t smem0 = ptx::smem_u32(smem);
 
     const uint32_t tiles = g.tiles_m * g.tiles_n;
@@ -123,7 +124,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     const uint32_t kend = min(g.K.size, kbeg + g.k_per_split);
     const int nslab = (int)((kend - kbeg + TK - 1) / TK);
     const int tid = threadIdx.x;
-    const int tx = tid & 15, ty = tid >> 4;
+    const int tx = tid % (TM / 8), ty = tid / (TM / 8); // TM/8 x 16 threads, 8 x FN outputs each
 
     // ---- per-tile tables ----
     for (int r = tid; r < TM + TN; r += NT) {
@@ -158,9 +159,9 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     auto issue = [&](int slab) {
         if (slab < nslab) {
             const uint32_t dst = smem0 + (slab % stages) * STAGE;
-            load_operand<LA, TM>(static_cast<const char*>(g.A), dst, T->rowA, T->kTab[slab & 1][0], tid,
+            load_operand<LA, TM, NT>(static_cast<const char*>(g.A), dst, T->rowA, T->kTab[slab & 1][0], tid,
                                  g.a_kmajor != 0);
-            load_operand<LB, TN>(static_cast<const char*>(g.B), dst + TM * TK * 4, T->rowB,
+            load_operand<LB, TN, NT>(static_cast<const char*>(g.B), dst + TM * TK * 4, T->rowB,
                                  T->kTab[slab & 1][1], tid, g.b_kmajor != 0);
         }
         ptx::cp_async_commit();
@@ -178,7 +179,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     uint32_t rows[8], cols[FN];
 #pragma unroll
     for (int i = 0; i < 8; ++i)
-        rows[i] = (i < 4 ? 0 : 64) + tx * 4 + (i & 3);
+        rows[i] = (i < 4 ? 0 : TM / 2) + tx * 4 + (i & 3);
 #pragma unroll
     for (int j = 0; j < FN; ++j)
         cols[j] = FN == 8 ? (j < 4 ? 0 : 64) + ty * 4 + (j & 3) : ty * FN + j;
@@ -189,16 +190,15 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     // read-modify-write at the end finds them on chip (the request holds no register).
     // The offset tables were completed before the prologue's first barrier.
     if (g.beta != 0.f && g.split_k == 1 && stages >= 2) {
-        if (FN == 8 && g.c_vec == 2) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int64_t cm = T->offCM[rows[i]];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int64_t cn = T->offCN[cols[4 * h % FN]];
-                    if (cm >= 0 && cn >= 0)
-                        asm volatile("prefetch.global.L2 [%0];" ::"l"(g.C + cm + cn));
-                }
+        if (FN == 8 && (g.c_vec == 2 || g.c_vec == 4)) {
+            // the same (row, 16-byte group) assignment as the unpacking below
+            const int warp = tid >> 5, lane = tid & 31;
+            const int64_t cn = T->offCN[g.c_vec == 4 ? (lane >> 3) + 16 * (lane & 7) : lane * 4];
+#pragma unroll 4
+            for (int r = 0; r < 16; ++r) {
+                const int64_t cm = T->offCM[warp * 16 + r];
+                if (cm >= 0 && cn >= 0)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(g.C + cm + cn));
             }
         } else if (g.c_vec == 1) {
 #pragma unroll
@@ -253,7 +253,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
                 for (int kk = 0; kk < 4; ++kk) {
                     const float* row = reinterpret_cast<const float*>(As) + (k4 * 4 + kk) * TM;
                     const float4 lo = *reinterpret_cast<const float4*>(row + tx * 4);
-                    const float4 hi = *reinterpret_cast<const float4*>(row + 64 + tx * 4);
+                    const float4 hi = *reinterpret_cast<const float4*>(row + TM / 2 + tx * 4);
                     a[0][kk] = lo.x; a[1][kk] = lo.y; a[2][kk] = lo.z; a[3][kk] = lo.w;
                     a[4][kk] = hi.x; a[5][kk] = hi.y; a[6][kk] = hi.z; a[7][kk] = hi.w;
                 }
@@ -314,28 +314,44 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_kernel(const __grid_constant_
     const bool vec_m = g.c_vec == 1;
     if (g.debug & 2) // experiment: no stores
         return;
-    if (FN == 8 && g.c_vec == 2 && g.split_k == 1) {
+    if (FN == 8 && (g.c_vec == 2 || g.c_vec == 4) && g.split_k == 1) {
         // C's stride-1 mode runs along the tile's columns.  The scaled accumulators pass
         // through shared memory (the stage ring is free now) so that a warp owns whole tile
-        // rows and its 32 lanes cover 128 consecutive columns: the read-modify-write of C
-        // then moves whole runs of C per instruction instead of 16-byte pieces (Eq. 11 as a
-        // transposition).  16-byte groups are XOR-swizzled by (row / 4) % 8: conflict-free
-        // both for the writes (lanes = rows) and for the reads (lanes = column groups).
+        // rows and its 32 lanes cover the row's 128 "slots", four consecutive slots being
+        // one 16-byte vector of C: the read-modify-write of C then moves whole runs of C
+        // per instruction instead of 16-byte pieces (Eq. 11 as a transposition).
+        //   c_vec == 2: slot = column
+        //   c_vec == 4: column = a + 4 p (a: piece of B's stride-1 mode, p along C's)
+        //               -> slot = 32 a + p
+        // 16-byte groups are XOR-swizzled by (row / 4) % 8: conflict-free for the 128-bit
+        // writes (lanes = rows) and reads (lanes = groups), two-way for the scalar writes.
         float* S = reinterpret_cast<float*>(smem);
+        if (g.c_vec == 2) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t row = rows[i];
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t row = rows[i];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint32_t c4 = cols[(4 * h) % FN] >> 2;
-                *reinterpret_cast<float4*>(S + row * TN + ((c4 ^ ((row >> 2) & 7)) << 2)) =
-                    make_float4(alpha * ACC(i, (4 * h) % FN), alpha * ACC(i, (4 * h + 1) % FN),
-                                alpha * ACC(i, (4 * h + 2) % FN), alpha * ACC(i, (4 * h + 3) % FN));
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t c4 = cols[(4 * h) % FN] >> 2;
+                    *reinterpret_cast<float4*>(S + row * TN + ((c4 ^ ((row >> 2) & 7)) << 2)) =
+                        make_float4(alpha * ACC(i, (4 * h) % FN), alpha * ACC(i, (4 * h + 1) % FN),
+                                    alpha * ACC(i, (4 * h + 2) % FN), alpha * ACC(i, (4 * h + 3) % FN));
+                }
+            }
+        } else {
+            // cols[j] = (j < 4 ? 0 : 64) + 4 ty + j % 4  ->  a = j % 4, p = ty + (j < 4 ? 0 : 16)
+            const uint32_t sw = (uint32_t)(tx & 7) << 2; // (row / 4) % 8 of all my rows
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float* Srow = S + ((i < 4 ? 0 : TM / 2) + tx * 4 + (i & 3)) * TN;
+#pragma unroll
+                for (int j = 0; j < FN; ++j)
+                    Srow[((j & 3) * (TN / 4) + (j < 4 ? 0 : 16) + ty) ^ sw] = alpha * ACC(i, j);
             }
         }
         __syncthreads();
         const int warp = tid >> 5, lane = tid & 31;
-        const int64_t cn = T->offCN[lane * 4];
+        const int64_t cn = T->offCN[g.c_vec == 4 ? (lane >> 3) + 16 * (lane & 7) : lane * 4];
 #pragma unroll
         for (int r0 = 0; r0 < 16; r0 += 8) {
             float4 old[8];
@@ -407,16 +423,18 @@ template <int LA, int LB>
 cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
 {
     void (*k)(GettKernelArgs);
-    if (args.tile_n == 128)
-        k = gett_ffma_kernel<LA, LB, 128>;
-    else if (args.tile_n == 32)
-        k = gett_ffma_kernel<LA, LB, 32>;
+    if (args.tile_n == 128 && args.tile_m == 128)
+        k = gett_ffma_kernel<LA, LB, 128, 128>;
+    else if (args.tile_n == 128 && args.tile_m == 64)
+        k = gett_ffma_kernel<LA, LB, 128, 64>;
+    else if (args.tile_n == 32 && args.tile_m == 128)
+        k = gett_ffma_kernel<LA, LB, 32, 128>;
     else
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess)
         return e;
-    k<<<grid, NT, smem, stream>>>(args);
+    k<<<grid, 2 * args.tile_m, smem, stream>>>(args);
     return cudaGetLastError();
 }
 
@@ -434,10 +452,12 @@ cudaError_t launch_b(const GettKernelArgs& args, int grid, int smem, cudaStream_
 
 } // namespace
 
-int gett_ffma_smem_bytes(int tile_n, int stages)
+int gett_ffma_smem_bytes(int tile_m, int tile_n, int stages)
 {
-    return tile_n == 128 ? stages * ffma_stage_bytes<128>() + (int)sizeof(FfmaSmem<128>)
-                         : stages * ffma_stage_bytes<32>() + (int)sizeof(FfmaSmem<32>);
+    if (tile_m == 64)
+        return stages * ffma_stage_bytes<64, 128>() + (int)sizeof(FfmaSmem<64, 128>);
+    return tile_n == 128 ? stages * ffma_stage_bytes<128, 128>() + (int)sizeof(FfmaSmem<128, 128>)
+                         : stages * ffma_stage_bytes<128, 32>() + (int)sizeof(FfmaSmem<128, 32>);
 }
 
 cudaError_t gett_launch_ffma(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)

@@ -290,6 +290,14 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     int leadK = find_unit(ik, 0); // A's stride-1 mode, if it is contracted ...
     if (leadK < 0)
         leadK = find_unit(ik, 1); // ... else B's
+    // Sec. 3.2.1 applied to I_n: B's stride-1 mode and C's stride-1 mode are two different
+    // modes of I_n, and B's can be split into pieces of one 16-byte vector (vecB elements).
+    auto n_split_ok = [&](int64_t vecB) {
+        const int unitCn = find_unit(in, 2);
+        return leadN >= 0 && unitCn >= 0 && unitCn != leadN && in[leadN].ext % vecB == 0 &&
+               in[leadN].ext > vecB && o.epilogue != GETT_EPI_DIRECT &&
+               (dtype != GETT_F32 || in[unitCn].ext % 4 == 0);
+    };
     if (dtype == GETT_F32) {
         // fp32 operands can also be gathered element by element (4-byte cp.async), so when
         // the contraction is short (C's traffic outweighs the operands') the set that
@@ -302,7 +310,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         if (ksize <= 512) {
             if (find_unit(im, 2) >= 0 && leadM != find_unit(im, 2))
                 leadM = -1;
-            if (find_unit(in, 2) >= 0 && leadN != find_unit(in, 2))
+            if (find_unit(in, 2) >= 0 && leadN != find_unit(in, 2) && !n_split_ok(4))
                 leadN = -1;
         }
     }
@@ -314,8 +322,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         // mode right after that piece, so that a tile holds vectors of B and runs of C.
         const int unitCn = find_unit(in, 2);
         const int64_t vecB = dtype == GETT_F32 ? 4 : 8;
-        if (leadN >= 0 && unitCn >= 0 && unitCn != leadN && in[leadN].ext % vecB == 0 &&
-            in[leadN].ext > vecB && o.epilogue != GETT_EPI_DIRECT && dtype != GETT_F32) {
+        if (n_split_ok(vecB)) {
             std::vector<GettDigit> t;
             t.push_back({leadN, vecB, 1});
             t.push_back({unitCn, in[unitCn].ext, 1});
@@ -383,6 +390,20 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         return GETT_ERR_UNSUPPORTED;
     // four consecutive tile rows (1) or columns (2) of C form one aligned 16-byte vector
     p->c_vec = vec_ok(p->M, false, p->N, false, 4) ? 1 : vec_ok(p->N, false, p->M, false, 4) ? 2 : 0;
+    // every C stride except that of N digit `skip_n_digit` is a multiple of four elements
+    auto others_mult4 = [&](int skip_n_digit) {
+        for (int d = 0; d < p->M.ndig; ++d)
+            if (p->M.sY[d] % 4)
+                return false;
+        for (int d = 0; d < p->N.ndig; ++d)
+            if (d != skip_n_digit && p->N.sY[d] % 4)
+                return false;
+        return true;
+    };
+    // fp32, columns = a + 4 p with p running along C's stride-1 mode (the N order above):
+    // four consecutive p of one a are one aligned 16-byte vector of C
+    const bool split4 = dtype == GETT_F32 && p->c_vec == 0 && p->N.ndig >= 2 && p->N.ext[0] == 4 &&
+                        p->N.sY[1] == 1 && p->N.ext[1] % 4 == 0 && others_mult4(1);
     info.path = path;
     p->debug = o.reserved[0];
     p->skinny = 0;
@@ -418,22 +439,37 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.epilogue = GETT_EPI_DIRECT;
         info.loader_b = GETT_LOAD_SCALAR; // B is read once, element by element
     } else if (path == GETT_PATH_FFMA) {
-        if ((o.tile_m && o.tile_m != 128) || (o.tile_k && o.tile_k != 32) ||
-            (o.epilogue && o.epilogue != GETT_EPI_DIRECT))
+        if ((o.tile_m && o.tile_m != 128 && o.tile_m != 64) || (o.tile_k && o.tile_k != 32))
             return GETT_ERR_UNSUPPORTED;
         int tn = o.tile_n ? o.tile_n : (p->N.size <= 32 ? 32 : 128);
         if (tn != 32 && tn != 128)
             return GETT_ERR_UNSUPPORTED;
-        int st = o.stages ? o.stages : (tn == 128 ? 3 : 4);
+        if (split4 && tn == 128)
+            p->c_vec = 4; // unpacking through the shared-memory transpose with the slot pattern
+        if (o.epilogue == GETT_EPI_STAGED && p->c_vec != 4)
+            return GETT_ERR_UNSUPPORTED;
+        // A short contraction (a few slabs) leaves a CTA's life dominated by latencies --
+        // offset tables, the first copies, the read-modify-write of C -- that only other
+        // resident CTAs can hide: 64-row tiles (128 threads) fit four CTAs per SM instead
+        // of two.  Long contractions keep the 128-row tile's higher flops per byte.
+        int tmh = o.tile_m;
+        if (tmh == 0)
+            tmh = (tn == 128 && p->K.size <= 128 &&
+                   (uint64_t)ceil_div(p->M.size, 64) * ceil_div(p->N.size, 128) >= 8ull * sms)
+                      ? 64
+                      : 128;
+        if (tmh == 64 && tn != 128)
+            return GETT_ERR_UNSUPPORTED;
+        int st = o.stages ? o.stages : (tmh == 64 ? 2 : tn == 128 ? 3 : 4);
         if (st < 2 || st > 4)
             return GETT_ERR_UNSUPPORTED;
-        info.tile_m = 128;
+        info.tile_m = tmh;
         info.tile_n = tn;
         info.tile_k = 32;
         info.stages = st;
-        info.block = 256;
-        info.smem_bytes = gett_ffma_smem_bytes(tn, st);
-        info.epilogue = GETT_EPI_DIRECT;
+        info.block = 2 * tmh;
+        info.smem_bytes = gett_ffma_smem_bytes(tmh, tn, st);
+        info.epilogue = p->c_vec == 4 ? GETT_EPI_STAGED : GETT_EPI_DIRECT;
     } else { // GETT_PATH_UMMA
         if ((o.tile_m && o.tile_m != 128 && o.tile_m != 256) || (o.tile_k && o.tile_k != 64))
             return GETT_ERR_UNSUPPORTED;
@@ -441,15 +477,6 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         // mode leads the M order (a warp's 32 rows are 32 consecutive floats).  When it
         // is a mode of I_n instead, the accumulator goes through a shared-memory
         // transpose if four consecutive "slots" are one aligned 16-byte vector of C.
-        auto others_mult4 = [&](int skip_n_digit) {
-            for (int d = 0; d < p->M.ndig; ++d)
-                if (p->M.sY[d] % 4)
-                    return false;
-            for (int d = 0; d < p->N.ndig; ++d)
-                if (d != skip_n_digit && p->N.sY[d] % 4)
-                    return false;
-            return true;
-        };
         int staged_cv = 0;
         if (!(p->M.ndig >= 1 && p->M.sY[0] == 1)) {
             if (p->N.ndig >= 2 && p->N.ext[0] == 8 && p->N.sY[1] == 1 && p->N.ext[1] % 4 == 0 &&

@@ -40,13 +40,14 @@ def test_reduced_workloads(key, dtype, path):
 @pytest.mark.parametrize("dtype", DTYPES)
 @pytest.mark.parametrize("epilogue", [g.GETT_EPI_AUTO, g.GETT_EPI_DIRECT])
 def test_cfg5_shape_with_split_stride_one_mode(dtype, epilogue):
-    """B's stride-1 mode (16) is split into 8-wide pieces around C's stride-1 mode (12):
-    exercises the staged epilogue (16-bit inputs) against the direct one."""
+    """B's stride-1 mode (16) is split into pieces of one 16-byte vector around C's stride-1
+    mode (12): exercises the staged epilogues against the direct ones."""
     w = workload("cfg5", dict(m0=2, m1=16, m2=5, n0=12, n1=3, n2=16, k=72))
     ratio, info = parity_case(w.contraction, dtype, w.dist, w.seed, w.alpha, w.beta, repeat=2,
                               epilogue=epilogue)
-    if dtype != F32 and epilogue == g.GETT_EPI_AUTO:
+    if epilogue == g.GETT_EPI_AUTO: # fp32 too: 4-wide pieces of B's mode, slots through shared memory
         assert info.epilogue == g.GETT_EPI_STAGED
+        assert info.loader_b == g.GETT_LOAD_VEC_FREE
     parity_case(w.contraction, dtype, w.dist, w.seed, -0.5, 0.0, epilogue=epilogue)
 
 
@@ -94,6 +95,23 @@ def test_256_row_tiles(spec, sizes):
             ratio, info = parity_case(con, dtype, "normal", 33, 1.0, 0.5, repeat=2, tile_m=256,
                                       tile_n=256, **extra)
             assert info.tile_m == 256 and info.path == g.GETT_PATH_UMMA
+
+
+@pytest.mark.parametrize("spec,sizes", [
+    ("C[m,n] = A[m,k] * B[k,n]", dict(m=200, n=136, k=88)),                        # A free-major, B K-major
+    ("C[m,n] = A[k,m] * B[n,k]", dict(m=136, n=264, k=72)),                        # A K-major, B free-major
+    ("C[n0,m2,m1,n2,m0,n1] = A[m1,k,m0,m2] * B[n2,n0,k,n1]",
+     dict(m0=2, m1=16, m2=5, n0=12, n1=3, n2=16, k=72)),                           # slots through shared memory
+    ("C[m0,n0,m1] = A[m0,k,m1] * B[k,n0]", dict(m0=24, m1=7, n0=40, k=48)),        # rows along C
+    ("C[a,b] = A[c,a,d] * B[d,c,b]", dict(a=90, b=70, c=5, d=7)),                  # scalar gathers
+])
+def test_fp32_64_row_tiles(spec, sizes):
+    """The strict-fp32 kernel with 64-row tiles (128 threads, four CTAs per SM), forced."""
+    con = parse_spec(spec, sizes)
+    for alpha, beta in [(1.0, 0.0), (0.5, 2.0)]:
+        ratio, info = parity_case(con, F32, "uniform", 17, alpha, beta, repeat=2, tile_m=64)
+        assert info.path == g.GETT_PATH_FFMA and info.tile_m == 64
+    parity_case(con, F32, "uniform", 17, 1.0, 0.5, tile_m=64, split_k=2)
 
 
 @pytest.mark.parametrize("sizes", [dict(m0=40, m1=33, n0=24, k=24), dict(m0=300, m1=7, n0=5, k=12),
