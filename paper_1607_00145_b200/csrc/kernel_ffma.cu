@@ -124,7 +124,9 @@ __global__ void __launch_bounds__(2 * TM, 256 / TM) gett_ffma_kernel(const __gri
     const uint32_t kend = min(g.K.size, kbeg + g.k_per_split);
     const int nslab = (int)((kend - kbeg + TK - 1) / TK);
     const int tid = threadIdx.x;
-    const int tx = tid % (TM / 8), ty = tid / (TM / 8); // TM/8 x 16 threads, 8 x FN outputs each
+    // TM/8 x 16 threads with 8 x FN outputs each.  A warp is 8 (along M) x 4 (along N) of
+    // them: its fragment reads touch 128 + 64 distinct bytes per k (one wavefront each).
+    const int tx = ((tid >> 5) % (TM / 64)) * 8 + (tid & 7), ty = ((tid >> 5) / (TM / 64)) * 4 + ((tid >> 3) & 3);
 
     // ---- per-tile tables ----
     for (int r = tid; r < TM + TN; r += NT) {

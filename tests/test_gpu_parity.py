@@ -51,6 +51,15 @@ def test_cfg5_shape_with_split_stride_one_mode(dtype, epilogue):
     parity_case(w.contraction, dtype, w.dist, w.seed, -0.5, 0.0, epilogue=epilogue)
 
 
+@pytest.mark.parametrize("n2,tile_m", [(12, 128), (12, 64), (24, 128), (40, 64)])
+def test_fp32_split_of_b_mode(n2, tile_m):
+    """fp32: B's stride-1 mode is cut into pieces of 4 (one 16-byte vector) around C's stride-1 mode."""
+    w = workload("cfg5", dict(m0=3, m1=16, m2=4, n0=12, n1=2, n2=n2, k=40))
+    for alpha, beta in [(1.0, 1.0), (-0.5, 0.0)]:
+        ratio, info = parity_case(w.contraction, F32, w.dist, w.seed, alpha, beta, repeat=2, tile_m=tile_m)
+        assert info.epilogue == g.GETT_EPI_STAGED and info.loader_b == g.GETT_LOAD_VEC_FREE
+
+
 def test_staged_epilogue_when_columns_already_run_along_c():
     # B is K-major, C's stride-1 mode is a mode of I_n: slots are the columns themselves
     con = parse_spec("C[n0,m,n1] = A[m,k] * B[k,n1,n0]", dict(m=136, n0=24, n1=7, k=80))
