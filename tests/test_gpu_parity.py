@@ -51,6 +51,19 @@ def test_cfg5_shape_with_split_stride_one_mode(dtype, epilogue):
     parity_case(w.contraction, dtype, w.dist, w.seed, -0.5, 0.0, epilogue=epilogue)
 
 
+@pytest.mark.parametrize("tile_n", [64, 128, 192, 256])
+@pytest.mark.parametrize("n0", [8, 24, 28])
+def test_staged_epilogue_strided_chunks_every_tile_width(tile_n, n0):
+    """Column = a + 8 p: every tile width (8, 16, 24, 32 values of p per tile), with C's stride-1
+    extent smaller than, equal to and not dividing the tile's p range; ragged M, N and K."""
+    w = workload("cfg5", dict(m0=3, m1=8, m2=7, n0=n0, n1=2, n2=24, k=72))
+    for dtype in (BF16_F32, F16_F32):
+        for alpha, beta in [(1.0, 1.0), (2.0, 0.0)]:
+            ratio, info = parity_case(w.contraction, dtype, w.dist, w.seed, alpha, beta, repeat=2, tile_n=tile_n)
+            assert info.epilogue == g.GETT_EPI_STAGED and info.tile_n == tile_n
+    parity_case(w.contraction, BF16_F32, w.dist, w.seed, 1.0, 0.5, tile_n=tile_n, split_k=2)
+
+
 @pytest.mark.parametrize("n2,tile_m", [(12, 128), (12, 64), (24, 128), (40, 64)])
 def test_fp32_split_of_b_mode(n2, tile_m):
     """fp32: B's stride-1 mode is cut into pieces of 4 (one 16-byte vector) around C's stride-1 mode."""
