@@ -88,15 +88,20 @@ typedef enum {
     GETT_EPI_AUTO = 0,
     GETT_EPI_DIRECT = 1, /* each thread stores its accumulators straight to C              */
     GETT_EPI_STAGED = 2  /* accumulators pass through a shared-memory transpose so that
-                            stores run along C's stride-1 mode (Eq. 11 as a transposition) */
+                            stores run along C's stride-1 mode (Eq. 11 as a transposition);
+                            available when that mode is a mode of I_n and four consecutive
+                            tile columns -- or, after B's stride-1 mode has been split into
+                            16-byte pieces around it (Sec. 3.2.1), four consecutive values of
+                            it -- are one aligned 16-byte vector of C.  GETT_EPI_DIRECT also
+                            switches that split off.                                        */
 } gett_epilogue_t;
 
 /* Planner overrides; zero-initialise for "auto".  Unsupported combinations make
  * gett_plan_create return GETT_ERR_UNSUPPORTED rather than being silently changed. */
 typedef struct {
     int32_t path;     /* gett_path_t                                     */
-    int32_t tile_m;   /* 0 = auto                                        */
-    int32_t tile_n;   /* 0 = auto                                        */
+    int32_t tile_m;   /* 0 = auto; UMMA 128 | 256, FFMA 128 | 64 (256: small-N kernel), SIMT 64 */
+    int32_t tile_n;   /* 0 = auto; UMMA 64 | 128 | 192 | 256, FFMA 128 | 32, SIMT 64            */
     int32_t tile_k;   /* 0 = auto (K elements per pipeline stage)        */
     int32_t stages;   /* 0 = auto                                        */
     int32_t split_k;  /* 0 = auto, 1 = never, s > 1 = exactly s slices   */

@@ -14,8 +14,9 @@
 //                                       vector-friendly order would scatter the stores to C)
 // The macro-kernel is an 8 x (TN/16) register tile per thread fed by 128-bit shared
 // loads (Sec. 3.1: outer products into a register-resident tile); unpacking
-// (Eq. 11) writes alpha*acc + beta*C through C's permutation, as 128-bit stores
-// along M when C's stride-1 mode leads the M order.
+// (Eq. 11) writes alpha*acc + beta*C through C's permutation: as 128-bit stores
+// along M when C's stride-1 mode leads the M order, through a shared-memory transpose
+// (whole tile rows per warp, 128-bit accesses along C) when it runs along the columns.
 #include "kernels.h"
 #include "ptx_sm100.cuh"
 
