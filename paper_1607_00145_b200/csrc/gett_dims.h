@@ -64,6 +64,20 @@ GETT_HD void gett_decompose(const GettDim& D, uint32_t idx, int64_t& oX, int64_t
     oY = y;
 }
 
+// The offset in the second carrier alone (M, N: the offset in C), for the unpacking code.
+GETT_HD int64_t gett_offset_y(const GettDim& D, uint32_t idx)
+{
+    int64_t y = 0;
+    uint32_t rem = idx;
+#pragma unroll 1
+    for (int d = 0; d < D.ndig; ++d) {
+        uint32_t q = gett_fastdiv(rem, D.mul[d], D.sh[d]);
+        y += (int64_t)(rem - q * D.ext[d]) * D.sY[d];
+        rem = q;
+    }
+    return y;
+}
+
 // Per-digit indices of fused index `idx` (first `n` digits are written).
 GETT_HD void gett_digit_indices(const GettDim& D, uint32_t idx, int32_t* out, int n)
 {

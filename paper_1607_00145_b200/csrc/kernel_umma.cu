@@ -266,17 +266,17 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
             const uint32_t j = cj / NCH, ch = cj - j * NCH;
             if (ch == 0) {
                 const WorkItem wi = decode_work(g, blockIdx.x + (es + 2 * j) * gridDim.x, MMA_M);
-                int64_t rc = -1, dummy;
+                int64_t rc = -1;
                 const uint32_t m = wi.m0 + eq * 32 + lane;
                 if (m < g.M.size)
-                    gett_decompose(g.M, m, dummy, rc);
+                    rc = gett_offset_y(g.M, m);
                 rowC_0 = (j & 1) ? rowC_0 : rc;
                 rowC_1 = (j & 1) ? rc : rowC_1;
                 for (uint32_t e = lane; e < TILE_N / 4; e += 32) {
                     const uint32_t col = Sh::col_of_group(e);
-                    int64_t x, y = -1;
+                    int64_t y = -1;
                     if (wi.n0 + col < g.N.size)
-                        gett_decompose(g.N, wi.n0 + col, x, y);
+                        y = gett_offset_y(g.N, wi.n0 + col);
                     grp[(j & 1) * EPI_GROUPS + e] = y;
                 }
                 __syncwarp();
@@ -701,14 +701,14 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                 wi.m0 += es * MMA_M;
             const uint32_t buf = es;
             // C offsets of this tile: my row in a register, the columns in shared memory
-            int64_t rowC = -1, dummy;
+            int64_t rowC = -1;
             if (wi.m0 + et < g.M.size)
-                gett_decompose(g.M, wi.m0 + et, dummy, rowC);
+                rowC = gett_offset_y(g.M, wi.m0 + et);
             ptx::named_barrier(1 + es, EPI_SET_THREADS); // previous tile's column table no longer read
             for (uint32_t c = et; c < TILE_N; c += EPI_SET_THREADS) {
-                int64_t x, y = -1;
+                int64_t y = -1;
                 if (wi.n0 + c < g.N.size)
-                    gett_decompose(g.N, wi.n0 + c, x, y);
+                    y = gett_offset_y(g.N, wi.n0 + c);
                 colC[c] = y;
             }
             ptx::named_barrier(1 + es, EPI_SET_THREADS);
