@@ -294,9 +294,22 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     // modes of I_n, and B's can be split into pieces of one 16-byte vector (vecB elements).
     auto n_split_ok = [&](int64_t vecB) {
         const int unitCn = find_unit(in, 2);
-        return leadN >= 0 && unitCn >= 0 && unitCn != leadN && in[leadN].ext % vecB == 0 &&
-               in[leadN].ext > vecB && o.epilogue != GETT_EPI_DIRECT &&
-               (dtype != GETT_F32 || in[unitCn].ext % 4 == 0);
+        if (!(leadN >= 0 && unitCn >= 0 && unitCn != leadN && in[leadN].ext % vecB == 0 &&
+              in[leadN].ext > vecB && o.epilogue != GETT_EPI_DIRECT))
+            return false;
+        if (dtype != GETT_F32)
+            return true;
+        // fp32 gives up C's order for the split, so the split must pay off in the unpacking:
+        // four consecutive values of C's mode have to be one aligned 16-byte vector of C
+        if (in[unitCn].ext % 4)
+            return false;
+        for (const GettMode& m : im)
+            if (m.sC % 4)
+                return false;
+        for (int i = 0; i < (int)in.size(); ++i)
+            if (i != unitCn && in[i].sC % 4)
+                return false;
+        return true;
     };
     if (dtype == GETT_F32) {
         // fp32 operands can also be gathered element by element (4-byte cp.async), so when

@@ -165,6 +165,22 @@ def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
     # cfg5: the tile is all 8-wide pieces of B's stride-1 mode x the whole of C's stride-1 mode
     i = g.Plan(workload("cfg5").contraction, g.GETT_BF16_F32).info
     assert (i.tile_m, i.tile_n, i.tile_k) == (128, 192, 64) and i.digits_n == 4
+    # cfg5 fp32: B's mode is cut into 4-wide pieces (one 16-byte vector of fp32) around C's mode,
+    # the unpacking goes through the slot-permuted transpose, short K -> 64-row tiles
+    i = g.Plan(workload("cfg5").contraction, g.GETT_F32).info
+    assert (i.path, i.loader_a, i.loader_b, i.epilogue) == \
+        (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_STAGED)
+    assert (i.tile_m, i.tile_n, i.tile_k, i.block) == (64, 128, 32, 128) and i.digits_n == 4
+    # ... asked for direct stores, the split is off and the N order follows C: B goes scalar
+    i = g.Plan(workload("cfg5").contraction, g.GETT_F32, epilogue=g.GETT_EPI_DIRECT).info
+    assert (i.loader_b, i.epilogue) == (g.GETT_LOAD_SCALAR, g.GETT_EPI_DIRECT)
+    # ... and when a stride of C is not a multiple of four the split would not pay off either
+    w5 = workload("cfg5", dict(m0=3, m1=8, m2=5, n0=8, n1=3, n2=8, k=40)).contraction
+    padded = Contraction(w5.name, w5.A, w5.B,
+                         TensorSpec(w5.C.labels, w5.C.extents, [1, 9, 9 * 5, 9 * 5 * 8, 9 * 5 * 8 * 8, 9 * 5 * 8 * 8 * 3]),
+                         w5.label_names)
+    i = g.Plan(padded, g.GETT_F32).info
+    assert (i.loader_b, i.epilogue) == (g.GETT_LOAD_SCALAR, g.GETT_EPI_DIRECT)
     # cfg4's 128-row tiles straddle the 72-wide modes: not boxes, so the gather loader stays
     # a 4-D operand whose leading extents are multiples of the tile is a box of a 4-D tensor map
     boxy = parse_spec("C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]",
