@@ -46,19 +46,36 @@ def test_merged_super_indices():
     assert T.merged_extents(con) == ([24, 576], [576, 24], [24])
 
 
+def _golden(name):
+    import os
+    out = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", name)) as f:
+        for line in f:
+            line = line.split("#")[0].split()
+            if line:
+                out[line[0]] = int(line[1])
+    return out
+
+
 def test_listing8_constants_follow_from_first_mode_fastest_strides():
+    """The numbers the paper prints for its merged-index example (fixture with the citation)."""
+    gold = _golden("listing8_constants.txt")
     con = parse_spec("C[a,b,c,i,j,k] = A[i,j,m,c] * B[m,k,a,b]",
                      dict(a=24, b=24, c=24, i=24, j=24, k=24, m=24))
     sA = dict(zip(_names(con, con.A.labels), con.A.strides))
     sB = dict(zip(_names(con, con.B.labels), con.B.strides))
     sC = dict(zip(_names(con, con.C.labels), con.C.strides))
-    assert sA["m"] == 576                  # ldb_ = i_UP            (A as (ij) x m)
-    assert sB["a"] == 24 * 24              # lda_ = m_UP * k_UP     (B as m x (ab) per k)
-    assert sC["i"] == 576 * 24             # ldc_ = a_UP * c_UP
-    assert sB["k"] == 24                   # &B[k * m_UP]
-    assert sA["c"] == 576 * 24             # &A[c * i_UP * m_UP]
-    assert sC["c"] == 576 and sC["k"] == 576 * 24 * 576   # &C[c*a_UP + k*a_UP*c_UP*i_UP]
-    assert sC["k"] == 7962624 and sC["i"] == 13824
+    m_ext, n_ext, k_ext = T.merged_extents(con)
+    # I_m = {c, (i,j)}, I_n = {(a,b), k}, I_k = {m}: the merged extents are the example's *_UP
+    assert m_ext == [gold["c_UP"], gold["i_UP"]] and n_ext == [gold["a_UP"], gold["k_UP"]]
+    assert k_ext == [gold["m_UP"]]
+    assert sB["a"] == gold["lda"] == gold["m_UP"] * gold["k_UP"]          # B as m x (ab) per k
+    assert sA["m"] == gold["ldb"] == gold["i_UP"]                         # A as (ij) x m
+    assert sC["i"] == gold["ldc"] == gold["a_UP"] * gold["c_UP"]
+    assert sB["k"] == gold["B_per_k"] == gold["m_UP"]
+    assert sA["c"] == gold["A_per_c"] == gold["i_UP"] * gold["m_UP"]
+    assert sC["c"] == gold["C_per_c"] == gold["a_UP"]
+    assert sC["k"] == gold["C_per_k"] == gold["a_UP"] * gold["c_UP"] * gold["i_UP"]
 
 
 def _grid(*axes):
