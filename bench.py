@@ -394,6 +394,8 @@ def run_ours(args):
                "roofline": roofline, "clocks": clocks}
         if args.all:
             out["workloads"] = run_all(torch, g, peaks, fp32_peak, args)
+        if args.pool:
+            out.update(run_pool(torch, g, peaks, args))
     elif rank == 0:
         # ---- end to end through the C ABI with host buffers ----
         pin = [torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
@@ -550,6 +552,43 @@ def run_all(torch, g, peaks, fp32_peak, args):
     return rows
 
 
+def run_pool(torch, g, peaks, args):
+    """The seeded pool of synthetic contractions (workloads.pool): per item and dtype the plan,
+    TFLOP/s, roofline fraction and the ratio to the equal-sized GEMM through the same library
+    (the paper's Sec. 7 statistic), plus the distribution of that ratio."""
+    from workloads import pool
+    rows = []
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for w in pool():
+        con = w.contraction
+        for dtype in w.dtypes:
+            a, b, c = make_inputs(con, dtype, w.dist, w.seed, w.beta)
+            dev = (_to_dev(a, torch), _to_dev(b, torch), _to_dev(c, torch))
+            t, info = time_contraction(torch, g, con, dtype, w.alpha, w.beta, dev, args.all_steps, 3)
+            flush.zero_()
+            mhz = info["clocks"]["sm_mhz"] or 1965.0
+            t_roof, bound = roofline_time_s(con, dtype, w.beta, peaks, _fp32_peak_tflops(mhz))
+            eg = equal_gemm(con)
+            ga, gb, gc = make_inputs(eg, dtype, w.dist, w.seed, w.beta)
+            gdev = (_to_dev(ga, torch), _to_dev(gb, torch), _to_dev(gc, torch))
+            t_eq, _ = time_contraction(torch, g, eg, dtype, w.alpha, w.beta, gdev, args.all_steps, 3)
+            M, N, K = con.mnk()
+            rows.append({"item": w.key, "spec": con.name, "dtype": DTYPE_NAMES[dtype], "mnk": [M, N, K],
+                         "ms": t * 1e3, "tflops": con.flops() / t / 1e12, "bound": bound,
+                         "roofline_frac": t_roof / t, "path": info["path"],
+                         "loaders": [info["loader_a"], info["loader_b"]], "epilogue": info["epilogue"],
+                         "tile": [info["tile_m"], info["tile_n"], info["tile_k"]],
+                         "split_k": info["split_k"], "speedup_vs_equal_gemm": t_eq / t})
+            del dev, gdev
+    out = {"pool": rows}
+    for name in sorted(DTYPE_BY_NAME):
+        r = np.array([x["speedup_vs_equal_gemm"] for x in rows if x["dtype"] == name])
+        if r.size:
+            out[f"ratio_to_equal_gemm_{name}"] = {"min": float(r.min()), "median": float(np.median(r)),
+                                                  "max": float(r.max()), "n": int(r.size)}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -561,6 +600,8 @@ def main():
     ap.add_argument("--path", type=int, default=0, help="force a gett_path_t")
     ap.add_argument("--split-k", type=int, default=0)
     ap.add_argument("--scale", default="", help="override extents, e.g. m=4096,n=4096 (profiling)")
+    ap.add_argument("--pool", action="store_true",
+                    help="with --kernel-only: also time the seeded pool of synthetic contractions")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end, equal-GEMM and CPU legs (profiling runs)")
     ap.add_argument("--all", action="store_true", help="also time every workload")

@@ -173,6 +173,7 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     args.debug = plan->debug;
     args.c_vec = plan->c_vec;
     args.prod_groups = plan->info.path == GETT_PATH_UMMA ? gett_umma_prod_groups(plan->info.stages) : 0;
+    args.epi_lean = plan->epi_lean;
 
     int path = plan->info.path;
     // the vectorised kernels need 16-byte aligned operand bases; otherwise gather scalars

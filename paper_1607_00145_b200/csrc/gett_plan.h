@@ -49,6 +49,7 @@ struct GettKernelArgs {
                           // (tensor-core kernel), 4 (fp32 kernel: column = a + 4 p, p along C)
     int32_t debug;        // opts.reserved[0]: experiment switches, 0 in normal use
     int32_t prod_groups;  // producer groups the tensor-core kernel uses (divides stages)
+    int32_t epi_lean;     // staged epilogue of the tensor-core kernel with one narrow staging buffer per warp
 };
 
 // Recipe for one operand's TMA tensor map: dimension i of the map follows digit
@@ -84,6 +85,7 @@ struct gett_plan {
     int32_t a_kmajor, b_kmajor;
     int32_t c_vec;
     int32_t skinny; // fp32: B resident in shared memory, A streamed (small N and K)
+    int32_t epi_lean; // see GettKernelArgs
     GettTmaRecipe tma_a, tma_b;
     // device side
     float* ws;
@@ -99,8 +101,8 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* A,
 gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, size_t capacity);
 
 // Geometry of the tensor-core kernel (kernel_umma.cu), needed by the planner.
-int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged_cv); // staged_cv: 0, 1 or 8
-int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged_cv);
+int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged_cv, int lean); // staged_cv: 0, 1 or 8
+int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged_cv, int lean);
 int gett_umma_block();
 int gett_umma_prod_groups(int stages); // producer groups in use; must divide the ring depth
 

@@ -54,11 +54,14 @@ constexpr int RASTER_M = 16;               // tile rows per rasterisation panel
 constexpr int EPI_PITCH = 68;              // floats per staged row: 64 + 4 keeps 128-bit accesses conflict-free
 constexpr int EPI_GROUPS = 256 / 4;          // 16-byte groups per tile row, at most
 constexpr int EPI_DEPTH = 2;                 // staging buffers per warp: old C is fetched EPI_DEPTH-1 chunks ahead
-// staging bytes of one epilogue warp: chunk buffers + group tables (cv as in StagedShape)
-__host__ __device__ constexpr int epi_pitch(int tile_n, int cv) { return cv == 8 ? tile_n / 4 + 4 : EPI_PITCH; }
-__host__ __device__ constexpr int epi_warp_bytes(int tile_n, int cv)
+// staging bytes of one epilogue warp: chunk buffers + group tables (cv, lean as in StagedShape)
+__host__ __device__ constexpr int epi_pitch(int tile_n, int cv, int lean)
 {
-    return EPI_DEPTH * (32 * epi_pitch(tile_n, cv) * 4 + EPI_GROUPS * 8);
+    return cv == 8 ? tile_n / 4 + 4 : lean ? 32 + 4 : EPI_PITCH;
+}
+__host__ __device__ constexpr int epi_warp_bytes(int tile_n, int cv, int lean)
+{
+    return (lean ? 1 : EPI_DEPTH) * 32 * epi_pitch(tile_n, cv, lean) * 4 + EPI_DEPTH * EPI_GROUPS * 8;
 }
 
 constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-byte-unit offset tables
@@ -215,12 +218,17 @@ struct OperandLoader {
 //            (a & 1) * TILE_N/8 + p: each row of the chunk is two runs of TILE_N/8
 //            consecutive floats of C, so the reads and writes of C cover whole runs of its
 //            stride-1 mode instead of 32-byte pieces of them.
-template <int TILE_N, int CV>
+// LEAN: one staging buffer per warp instead of two (the old C of a chunk is requested when
+// the previous chunk is done, not one chunk ahead) and 32-column chunks for CV == 1: a third
+// of the shared memory, for long contractions, where the operand ring needs the space and
+// the unpacking hides behind the next tile's main loop anyway.
+template <int TILE_N, int CV, int LEAN>
 struct StagedShape {
     static constexpr uint32_t NP = TILE_N / 8;                      // CV == 8: pieces (values of p) per tile
-    static constexpr uint32_t NCH = CV == 8 ? 4 : TILE_N / 64;      // chunks per tile
-    static constexpr uint32_t SLOTS = CV == 8 ? TILE_N / 4 : 64;    // slots per row of a chunk
-    static constexpr uint32_t PITCH = epi_pitch(TILE_N, CV);        // SLOTS + 4 keeps 128-bit accesses conflict-free
+    static constexpr uint32_t SLOTS = CV == 8 ? TILE_N / 4 : LEAN ? 32 : 64; // slots per row of a chunk
+    static constexpr uint32_t NCH = CV == 8 ? 4 : TILE_N / SLOTS;   // chunks per tile
+    static constexpr uint32_t DEPTH = LEAN ? 1 : EPI_DEPTH;         // staging buffers
+    static constexpr uint32_t PITCH = epi_pitch(TILE_N, CV, LEAN);  // SLOTS + 4 keeps 128-bit accesses conflict-free
     static constexpr uint32_t GPR = SLOTS / 4;                      // 16-byte groups per row of a chunk
     static_assert(PITCH == SLOTS + 4, "staging pitch");
     // first tile column of the 16-byte group number e (e = chunk * GPR + group in the row)
@@ -239,16 +247,16 @@ struct StagedShape {
 //                 one row per lane), result written back to staging with 128-bit stores;
 //                 then the warp re-reads staging with lanes running along C and issues
 //                 128-bit global stores
-template <int TILE_N, int CV>
+template <int TILE_N, int CV, int LEAN>
 __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTables* T, uint8_t* epi_smem,
                                                 uint32_t tmem_base, uint32_t warp, uint32_t lane,
                                                 uint32_t total_work, volatile int* abort_flag)
 {
-    using Sh = StagedShape<TILE_N, CV>;
-    constexpr uint32_t NCH = Sh::NCH, PITCH = Sh::PITCH, GPR = Sh::GPR, NP = Sh::NP;
+    using Sh = StagedShape<TILE_N, CV, LEAN>;
+    constexpr uint32_t NCH = Sh::NCH, PITCH = Sh::PITCH, GPR = Sh::GPR, NP = Sh::NP, DEPTH = Sh::DEPTH;
     constexpr uint32_t FULL = 0xFFFFFFFFu;
-    float* S = reinterpret_cast<float*>(epi_smem + warp * epi_warp_bytes(TILE_N, CV));
-    int64_t* grp = reinterpret_cast<int64_t*>(S + EPI_DEPTH * 32 * PITCH);
+    float* S = reinterpret_cast<float*>(epi_smem + warp * epi_warp_bytes(TILE_N, CV, LEAN));
+    int64_t* grp = reinterpret_cast<int64_t*>(S + DEPTH * 32 * PITCH);
     const uint32_t s_u32 = ptx::smem_u32(S);
     const float alpha = g.alpha, beta = g.beta;
     const bool rmw = beta != 0.f && !(g.debug & 128); // (debug & 128: experiment, old C not read)
@@ -283,7 +291,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
             }
             if (rmw) {
                 const long long myrow = my_row(j);
-                const uint32_t dst = s_u32 + (cj & 1) * (32 * PITCH * 4);
+                const uint32_t dst = s_u32 + (cj & (DEPTH - 1)) * (32 * PITCH * 4);
                 const int64_t* gch = grp + (j & 1) * EPI_GROUPS + ch * GPR;
                 // four copies at a time: offsets first, then the copies back to back
 #pragma unroll
@@ -334,25 +342,31 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
         }
     };
 
-    prepare(0);
+    if (DEPTH == 2)
+        prepare(0);
     for (uint32_t ci = 0; ci < nchunk; ++ci) {
-        prepare(ci + 1);
-        ptx::cp_async_wait<1>(); // chunk ci's old C has landed (my copies) ...
-        __syncwarp();            // ... and everybody else's
+        if (DEPTH == 2) {
+            prepare(ci + 1);
+            ptx::cp_async_wait<1>(); // chunk ci's old C has landed (my copies) ...
+        } else {
+            prepare(ci);
+            ptx::cp_async_wait<0>();
+        }
+        __syncwarp(); // ... and everybody else's
         const uint32_t j = ci / NCH, ch = ci - j * NCH, buf = es; // tile es + 2j uses accumulator es
         if (ch == 0) {
             if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag))
                 break;
             ptx::tc_fence_after();
         }
-        float* Sb = S + (ci & 1) * (32 * PITCH);
+        float* Sb = S + (ci & (DEPTH - 1)) * (32 * PITCH);
         float* Srow = Sb + lane * PITCH;
         const uint32_t tacc = tmem_base + ((eq * 32u) << 16) + buf * 256;
         if (CV == 1) {
 #pragma unroll
-            for (uint32_t h = 0; h < 2; ++h) {
+            for (uint32_t h = 0; h < Sh::SLOTS / 32; ++h) {
                 uint32_t v[32];
-                ptx::tmem_ld_32x32(tacc + ch * 64 + h * 32, v);
+                ptx::tmem_ld_32x32(tacc + ch * Sh::SLOTS + h * 32, v);
                 ptx::tmem_wait_ld();
 #pragma unroll
                 for (int u0 = 0; u0 < 8; u0 += 4) {
@@ -684,10 +698,14 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
         const bool staged = g.epilogue == GETT_EPI_STAGED && g.split_k == 1;
         if (staged) {
             uint8_t* epi_smem = smem + stages * sbytes + sizeof(SmemTables);
-            if (g.c_vec == 8)
-                epilogue_staged<TILE_N, 8>(g, T, epi_smem, tmem_base, warp, lane, total_work, abort_flag);
+            if (g.c_vec == 8 && g.epi_lean)
+                epilogue_staged<TILE_N, 8, 1>(g, T, epi_smem, tmem_base, warp, lane, total_work, abort_flag);
+            else if (g.c_vec == 8)
+                epilogue_staged<TILE_N, 8, 0>(g, T, epi_smem, tmem_base, warp, lane, total_work, abort_flag);
+            else if (g.epi_lean)
+                epilogue_staged<TILE_N, 1, 1>(g, T, epi_smem, tmem_base, warp, lane, total_work, abort_flag);
             else
-                epilogue_staged<TILE_N, 1>(g, T, epi_smem, tmem_base, warp, lane, total_work, abort_flag);
+                epilogue_staged<TILE_N, 1, 0>(g, T, epi_smem, tmem_base, warp, lane, total_work, abort_flag);
         }
         int64_t* colC = T->colC[es];
         uint32_t j = 0; // counts this set's tiles
@@ -773,16 +791,16 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
 
 } // namespace
 
-int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged_cv)
+int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged_cv, int lean)
 {
     return 1024 + stages * (int)stage_bytes((uint32_t)tile_m, (uint32_t)tile_n) + (int)sizeof(SmemTables) +
-           (staged_cv ? NUM_EPI_WARPS * epi_warp_bytes(tile_n, staged_cv) : 0);
+           (staged_cv ? NUM_EPI_WARPS * epi_warp_bytes(tile_n, staged_cv, lean) : 0);
 }
 
-int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged_cv)
+int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged_cv, int lean)
 {
     int s = (smem_limit - 1024 - (int)sizeof(SmemTables) -
-             (staged_cv ? NUM_EPI_WARPS * epi_warp_bytes(tile_n, staged_cv) : 0)) /
+             (staged_cv ? NUM_EPI_WARPS * epi_warp_bytes(tile_n, staged_cv, lean) : 0)) /
             (int)stage_bytes((uint32_t)tile_m, (uint32_t)tile_n);
     s = s > MAX_STAGES ? MAX_STAGES : s;
     return s >= PROD_GROUPS ? s - s % PROD_GROUPS : s; // a stage is always served by the same group

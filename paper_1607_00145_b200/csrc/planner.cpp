@@ -420,6 +420,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     info.path = path;
     p->debug = o.reserved[0];
     p->skinny = 0;
+    p->epi_lean = 0;
     memset(&p->tma_a, 0, sizeof p->tma_a);
     memset(&p->tma_b, 0, sizeof p->tma_b);
 
@@ -530,6 +531,17 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         if (tn != 64 && tn != 128 && tn != 192 && tn != 256)
             return GETT_ERR_UNSUPPORTED;
         const int smem_limit = 227 * 1024;
+        // The staging rows take shared memory from the operand ring.  A long contraction
+        // needs the ring (three stages, or one per slab) more than it needs the old values of
+        // C one chunk ahead: its unpacking hides behind the next tile's main loop, so it gets
+        // the lean staging (one narrow buffer per warp).
+        int lean = 0;
+        if (staged_cv) {
+            const int need = (int)std::min<uint32_t>(3, ceil_div(p->K.size, 64));
+            if (gett_umma_max_stages(128, tn, smem_limit, staged_cv, 0) < need)
+                lean = 1;
+        }
+        p->epi_lean = lean;
         const int staged = info.epilogue == GETT_EPI_STAGED;
         // 256-row tiles (both accumulator buffers for one tile) cut the operand bytes per
         // flop by a third; worth it when the contraction is long enough to be bound by
@@ -542,15 +554,15 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         }
         if (tmh == 256 && (tn != 256 || staged))
             return GETT_ERR_UNSUPPORTED;
-        int st = o.stages ? o.stages : gett_umma_max_stages(tmh, tn, smem_limit, staged_cv);
-        if (st < 1 || st > gett_umma_max_stages(tmh, tn, smem_limit, staged_cv) || st % gett_umma_prod_groups(st))
+        int st = o.stages ? o.stages : gett_umma_max_stages(tmh, tn, smem_limit, staged_cv, lean);
+        if (st < 1 || st > gett_umma_max_stages(tmh, tn, smem_limit, staged_cv, lean) || st % gett_umma_prod_groups(st))
             return GETT_ERR_UNSUPPORTED;
         info.tile_m = tmh;
         info.tile_n = tn;
         info.tile_k = 64;
         info.stages = st;
         info.block = gett_umma_block();
-        info.smem_bytes = gett_umma_smem_bytes(tmh, tn, st, staged_cv);
+        info.smem_bytes = gett_umma_smem_bytes(tmh, tn, st, staged_cv, lean);
         if (!(p->debug & 32)) { // (debug & 32: experiment switch, gather even where TMA applies)
             make_tma_recipe(p->M, true, p->K, true, info.loader_a, (uint32_t)tmh, p->tma_a);
             make_tma_recipe(p->N, true, p->K, false, info.loader_b, (uint32_t)tn, p->tma_b);

@@ -283,6 +283,52 @@ def workload(key: str, scale: Optional[Dict[str, int]] = None) -> Workload:
 WORKLOAD_KEYS = ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5")
 
 
+def pool(seed: int = 2016, per_family: int = 5) -> List[Workload]:
+    """A seeded pool of synthetic contractions with random mode orders, one family per kind of
+    shape the paper's benchmark contains (its own contraction strings and input files are not
+    reproduced here): plain matrices in the four transposition variants, a large tensor times
+    a small matrix, 4-D tensors with two free and two contracted modes each, the 6-D / 4-D / 4-D
+    coupled-cluster shape with one contracted mode, and mixed 3- to 5-D cases.  Extents are
+    drawn from the values the paper's families use (24, 48, 72, 96, 312, ...).  Every tensor
+    is packed with its first listed mode stride-1; the order of the modes inside A, B and C
+    is a random permutation, so the pool exercises every loader / epilogue combination."""
+    rng = np.random.default_rng(seed)
+    out: List[Workload] = []
+
+    def emit(family: str, m: Dict[str, int], n: Dict[str, int], k: Dict[str, int], beta: float):
+        sizes = {**m, **n, **k}
+        am, bn, cm = list(m) + list(k), list(k) + list(n), list(m) + list(n)
+        for lst in (am, bn, cm):
+            rng.shuffle(lst)
+        spec = f"C[{','.join(cm)}] = A[{','.join(am)}] * B[{','.join(bn)}]"
+        key = f"{family}{sum(1 for w in out if w.key.startswith(family))}"
+        w = _wl(key, spec, sizes, (F32, BF16_F32), "uniform", 100 + len(out), 1.0, beta, "pool")
+        w.contraction.name = spec + "  " + ",".join(f"{k_}={v}" for k_, v in sizes.items())
+        out.append(w)
+
+    pick = lambda vals: int(rng.choice(vals))
+    for i in range(per_family):
+        # plain matrices
+        emit("gemm", {"m": pick([2048, 3072, 4096])}, {"n": pick([2048, 3072, 4096])},
+             {"k": pick([1024, 2048, 4096])}, float(i % 2))
+        # tensor times small matrix (either operand may be the small one after the shuffle)
+        e = pick([24, 32, 48])
+        emit("ttm", {"a": pick([312, 296, 256]), "b": pick([312, 296, 256]), "c": pick([8, 16, 24])},
+             {"u": e}, {"k": pick([24, 32, 48])}, 0.0)
+        # two free and two contracted modes per operand, one extent
+        e = pick([48, 72, 96])
+        emit("d4", {"a": e, "b": e}, {"c": e, "d": e}, {"k": e, "l": e}, 0.0)
+        # coupled-cluster shape: three free modes per operand, one contracted mode
+        e = pick([16, 24])
+        emit("cc", {"a": e, "b": e, "c": e}, {"i": e, "j": e, "l": e}, {"k": pick([24, 48, 64])},
+             float((i + 1) % 2))
+        # mixed ranks and extents
+        emit("mix", {"a": pick([40, 72, 120]), "b": pick([24, 56, 64])},
+             {"c": pick([48, 96, 312])} if i % 2 else {"c": pick([48, 96]), "d": pick([8, 24, 40])},
+             {"k": pick([32, 72, 200]), "l": pick([8, 24])}, 0.0)
+    return out
+
+
 def draw(dist: str, seed: int, tensor: str, n: int) -> np.ndarray:
     tid = TENSOR_ID[tensor]
     if dist == "uniform":
