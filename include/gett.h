@@ -126,7 +126,10 @@ typedef struct {
     int64_t workspace_bytes;          /* split-K partial sums owned by the plan            */
     int64_t tiles;                    /* output tiles (M tiles x N tiles)                  */
     int32_t device;                   /* CUDA device the plan is bound to, -1 = none       */
-    int32_t reserved[7];
+    int32_t swapped;                  /* 1: the kernel runs with the operands exchanged (its rows
+                                         run over I_n, its columns over I_m; tile_m and tile_n are
+                                         the kernel's).  Everything else here is the caller's view. */
+    int32_t reserved[6];
 } gett_plan_info_t;
 
 typedef enum {

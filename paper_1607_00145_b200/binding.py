@@ -52,7 +52,8 @@ class PlanInfo(ctypes.Structure):
                 ("digits_m", ctypes.c_int32), ("digits_n", ctypes.c_int32),
                 ("digits_k", ctypes.c_int32),
                 ("workspace_bytes", ctypes.c_int64), ("tiles", ctypes.c_int64),
-                ("device", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7)]
+                ("device", ctypes.c_int32), ("swapped", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 6)]
 
     def as_dict(self) -> Dict[str, object]:
         out = {}

@@ -6,6 +6,7 @@
 
 #include <cstring>
 #include <new>
+#include <utility>
 
 #include "kernels.h"
 
@@ -139,6 +140,8 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
 {
     if (!plan || !A || !B || !C)
         return GETT_ERR_INVALID_ARG;
+    if (plan->swapped) // the kernels run with the operands exchanged
+        std::swap(A, B);
     if (plan->info.device < 0)
         return GETT_ERR_CUDA;
     const uintptr_t es = plan->dtype == GETT_F32 ? 4 : 2;
@@ -164,8 +167,9 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     args.dtype = plan->dtype;
     args.a_kmajor = plan->a_kmajor;
     args.b_kmajor = plan->b_kmajor;
-    args.loader_a = vec_kind(plan->info.loader_a);
-    args.loader_b = vec_kind(plan->info.loader_b);
+    // (info is the caller's view: with exchanged operands its loader_a describes the kernels' B)
+    args.loader_a = vec_kind(plan->swapped ? plan->info.loader_b : plan->info.loader_a);
+    args.loader_b = vec_kind(plan->swapped ? plan->info.loader_a : plan->info.loader_b);
     args.tile_m = plan->info.tile_m;
     args.tile_n = plan->info.tile_n;
     args.stages = plan->info.stages;

@@ -87,8 +87,8 @@ extern "C" gett_status_t gett_contract_noalloc(const gett_tensor_desc_t* A, cons
     args.M = plan.M;
     args.N = plan.N;
     args.K = plan.K;
-    args.A = A_data;
-    args.B = B_data;
+    args.A = plan.swapped ? B_data : A_data; // (the plan may have exchanged the operands)
+    args.B = plan.swapped ? A_data : B_data;
     args.C = static_cast<float*>(C_data);
     args.ws = scratch;
     args.status = nullptr;

@@ -280,6 +280,34 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     std::stable_sort(in.begin(), in.end(), byC);
     std::stable_sort(ik.begin(), ik.end(), byA);
     p->dtype = dtype;
+
+    // ---- which operand gives the kernel its rows ----
+    // The kernels unpack along their columns (the N-side split below, the staged epilogues).
+    // If C's stride-1 mode belongs to A but is not A's own stride-1 mode, exchange the roles of
+    // A and B (C = A B is also C = B A with rows and columns exchanged): that mode becomes a
+    // column mode, and A's stride-1 mode can be split around it.  The lists keep their order;
+    // only the carriers change places.
+    p->swapped = 0;
+    {
+        const int unitCm = find_unit(im, 2), unitAm = find_unit(im, 0);
+        const int64_t vec = dtype == GETT_F32 ? 4 : 8;
+        bool want = unitCm >= 0 && unitAm >= 0 && unitCm != unitAm && im[unitAm].ext % vec == 0 &&
+                    im[unitAm].ext > vec && im[unitCm].ext % 4 == 0 && o.epilogue != GETT_EPI_DIRECT &&
+                    !(o.reserved[0] & 8192); // (experiment switch: never exchange)
+        if (want && dtype == GETT_F32) { // the same alignment the fp32 split asks for
+            for (const GettMode& m : in)
+                want = want && m.sC % 4 == 0;
+            for (int i = 0; i < (int)im.size(); ++i)
+                want = want && (i == unitCm || im[i].sC % 4 == 0);
+        }
+        if (want) {
+            std::swap(im, in);
+            for (std::vector<GettMode>* v : {&im, &in, &ik})
+                for (GettMode& m : *v)
+                    std::swap(m.sA, m.sB);
+            p->swapped = 1;
+        }
+    }
     p->im = im;
     p->in = in;
     p->ik = ik;
@@ -610,6 +638,16 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.grid = (int32_t)std::min<uint64_t>(tiles * split, (uint64_t)sms);
     if (p->skinny) // persistent: two CTAs per SM stream the row tiles
         info.grid = (int32_t)std::min<uint64_t>(p->tiles_m, 2ull * sms);
+    info.swapped = p->swapped;
+    if (p->swapped) { // report the caller's view
+        std::swap(info.M, info.N);
+        std::swap(info.n_m, info.n_n);
+        std::swap(info.merged_m, info.merged_n);
+        std::swap(info.digits_m, info.digits_n);
+        std::swap(info.loader_a, info.loader_b);
+        for (int i = 0; i < GETT_MAX_MODES; ++i)
+            std::swap(info.labels_m[i], info.labels_n[i]);
+    }
     return GETT_OK;
 }
 
@@ -621,6 +659,17 @@ gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, si
     const std::vector<GettDigit>* digits;
     const GettDim* D;
     bool wantX;
+    if (p->swapped) { // the caller's A is the kernels' B: rows <-> columns, X <-> Y for K
+        switch (which) {
+        case GETT_TABLE_A_M: which = GETT_TABLE_B_N; break;
+        case GETT_TABLE_C_M: which = GETT_TABLE_C_N; break;
+        case GETT_TABLE_B_N: which = GETT_TABLE_A_M; break;
+        case GETT_TABLE_C_N: which = GETT_TABLE_C_M; break;
+        case GETT_TABLE_A_K: which = GETT_TABLE_B_K; break;
+        case GETT_TABLE_B_K: which = GETT_TABLE_A_K; break;
+        default: break;
+        }
+    }
     switch (which) {
     case GETT_TABLE_A_M: modes = &p->im; digits = &p->tm; D = &p->M; wantX = true; break;
     case GETT_TABLE_C_M: modes = &p->im; digits = &p->tm; D = &p->M; wantX = false; break;
