@@ -134,6 +134,24 @@ def test_contract_without_device_reports_cuda_error_not_a_crash():
     assert e.value.status == 7
 
 
+def test_operands_are_exchanged_when_c_runs_along_a_mode_of_a_that_is_not_a_s_own():
+    # C's stride-1 mode `a` belongs to A, whose own stride-1 mode is `b`
+    con = parse_spec("C[a,b,j,l,c,i] = A[b,c,k,a] * B[j,i,k,l]",
+                     dict(a=24, b=24, c=8, i=8, j=24, l=8, k=40))
+    for dtype in (g.GETT_BF16_F32, g.GETT_F32):
+        p = _tables_match(con, dtype)          # the tables stay the caller's, bit for bit
+        i = p.info
+        assert i.swapped == 1 and (i.M, i.N, i.K) == con.mnk()
+        im, in_, ik = T.classify(con)
+        assert i.as_dict()["labels_m"] == im and i.as_dict()["labels_n"] == in_
+        assert i.loader_a == g.GETT_LOAD_VEC_FREE and i.epilogue == g.GETT_EPI_STAGED
+        # asked for direct stores there is nothing to gain from the exchange
+        assert g.Plan(con, dtype, epilogue=g.GETT_EPI_DIRECT).info.swapped == 0
+    # A's stride-1 mode is also C's: rows already run along C, no exchange
+    assert g.Plan(workload("cfg4").contraction, g.GETT_BF16_F32).info.swapped == 0
+    assert g.Plan(workload("cfg3").contraction, g.GETT_F32).info.swapped == 0
+
+
 def test_split_k_planning():
     con = workload("splitk").contraction
     auto = g.Plan(con, g.GETT_F32)
