@@ -537,9 +537,13 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         int tn = o.tile_n;
         if (tn == 0 && staged_cv == 8) {
             // one tile = all 8-wide pieces x the whole of C's stride-1 mode, if that is a legal width
+            // (the widest legal width that holds whole runs: fewer, larger tiles)
             const uint32_t want = 8 * p->N.ext[1];
-            if (want == 64 || want == 128 || want == 192 || want == 256)
-                tn = (int)want;
+            for (uint32_t cand : {256u, 192u, 128u, 64u})
+                if (cand % want == 0) {
+                    tn = (int)cand;
+                    break;
+                }
         }
         if (tn == 0) {
             // fewest waves x per-tile cost; ties go to the wider tile
