@@ -281,7 +281,16 @@ __global__ void __launch_bounds__(2 * TM, 256 / TM) gett_ffma_kernel(const __gri
             }
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
-                if constexpr (PAIR_ROWS) {
+                if constexpr (A_K && B_K) {
+                    // both fragments deliver 4 k of ONE row / column per load: neither operand
+                    // has neighbours in adjacent registers, and building the pairs costs more
+                    // issue slots than the packed instruction saves -> plain FMAs
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+#pragma unroll
+                        for (int j = 0; j < FN; ++j)
+                            ACC(i, j) = fmaf(a[i][kk], b[j][kk], ACC(i, j));
+                } else if constexpr (PAIR_ROWS) {
                     float2 b2[FN];
 #pragma unroll
                     for (int j = 0; j < FN; ++j)
