@@ -113,5 +113,6 @@ int gett_ffma_smem_bytes(int tile_m, int tile_n, int stages);
 
 // fp32 kernel for N <= 32, K <= gett_ffma_skinny_max_k(), A K-major (kernel_ffma_skinny.cu).
 int gett_ffma_skinny_smem_bytes(int N, int K);
+int gett_ffma_skinny_mn_smem_bytes(int N, int K); // ... A staged MN-major (its stride-1 mode is free)
 int gett_ffma_skinny_rows();
 int gett_ffma_skinny_max_k();

@@ -191,9 +191,184 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
     ptx::cp_async_wait_all();
 }
 
+// ---- the same regime with A staged MN-major (A's stride-1 mode is a free mode) ----
+// A tile is [k][256 rows] in shared memory, filled with 16-byte pieces of four consecutive
+// rows; a thread owns the four rows 4 q .. 4 q + 3 (one 128-bit read per k delivers all four)
+// and CPT columns, and writes C with 128-bit stores along the rows when four consecutive rows
+// are one aligned vector of C.
+struct SkinnyMnTables {
+    int64_t offCM[TSLOTS][ROWS]; // C offset of each tile row (-1 beyond M)
+    int64_t offCN[32];
+    uint32_t kA[KMAX];           // A offset of each k, 16-byte units
+};
+
+// KT: K when known at compile time (the k loop is then fully unrolled), 0 = run time
+template <int CPT, int KT>
+__global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_mn_kernel(const __grid_constant__ GettKernelArgs g)
+{
+    constexpr int NP = 4 * CPT; // padded row of B in shared memory
+    constexpr uint32_t NONE = 0xFFFFFFFFu;
+    extern __shared__ __align__(16) uint8_t smem[];
+    const uint32_t K = KT ? (uint32_t)KT : g.K.size, N = g.N.size, Msz = g.M.size;
+    const uint32_t tile_bytes = K * ROWS * 4;
+    float* Bs = reinterpret_cast<float*>(smem);                       // [K][NP]
+    uint8_t* ring = smem + K * NP * 4;
+    SkinnyMnTables* T = reinterpret_cast<SkinnyMnTables*>(ring + STAGES * tile_bytes);
+    const uint32_t ring_u32 = ptx::smem_u32(ring);
+    const int tid = threadIdx.x;
+    const uint32_t ntiles = g.tiles_m;
+
+    for (uint32_t i = tid; i < K * NP; i += NT) {
+        const uint32_t k = i / NP, n = i - k * NP;
+        float v = 0.f;
+        if (n < N) {
+            int64_t bn, cn, ak, bk;
+            gett_decompose(g.N, n, bn, cn);
+            gett_decompose(g.K, k, ak, bk);
+            v = __ldg(static_cast<const float*>(g.B) + bn + bk);
+        }
+        Bs[i] = v;
+    }
+    if (tid < 32) {
+        int64_t bn, cn = -1;
+        if ((uint32_t)tid < N)
+            gett_decompose(g.N, tid, bn, cn);
+        T->offCN[tid] = cn;
+    }
+    if ((uint32_t)tid < K) {
+        int64_t ak, bk;
+        gett_decompose(g.K, tid, ak, bk);
+        T->kA[tid] = (uint32_t)(ak >> 2);
+    }
+    const uint32_t chunk = (ntiles + gridDim.x - 1) / gridDim.x;
+    const uint32_t t_begin = blockIdx.x * chunk;
+    const uint32_t t_end = min(ntiles, t_begin + chunk);
+    // Thread tid publishes the C offset of tile row tid, and copies the pieces (k, quad) with
+    // quad = tid % 64 (rows 4 quad ..), k = tid / 64 + 4 p: lanes run along the rows.
+    const uint32_t quad = tid & 63, kq = tid >> 6;
+    auto issue = [&](uint32_t it) {
+        const uint32_t t = t_begin + it;
+        if (t < t_end) {
+            const uint32_t m = t * ROWS + tid;
+            T->offCM[it % TSLOTS][tid] = m < Msz ? gett_offset_y(g.M, m) : -1;
+            const uint32_t mq = t * ROWS + 4 * quad;
+            uint32_t x4 = NONE; // (M's leading extent is a multiple of 4: a quad is inside M or outside)
+            if (mq < Msz) {
+                int64_t x, y;
+                gett_decompose(g.M, mq, x, y);
+                x4 = (uint32_t)(x >> 2);
+            }
+            const uint32_t dst = ring_u32 + (it % STAGES) * tile_bytes + quad * 16;
+            const char* base = static_cast<const char*>(g.A);
+#pragma unroll(KT ? KT / 4 : 2)
+            for (uint32_t k = kq; k < K; k += NT / 64) {
+                const bool ok = x4 != NONE;
+                ptx::cp_async_16(dst + k * (ROWS * 4), base + (ok ? ((uint64_t)(x4 + T->kA[k]) << 4) : 0),
+                                 ok ? 16u : 0u);
+            }
+        }
+        ptx::cp_async_commit();
+    };
+
+    __syncthreads(); // kA ready
+    for (uint32_t s = 0; s < STAGES - 1; ++s)
+        issue(s);
+
+    const uint32_t q = tid % QL, cg = tid / QL; // rows 4 q ..; a warp shares one column group
+    const float alpha = g.alpha, beta = g.beta;
+    const bool vec_rows = g.c_vec == 1;
+    int64_t cn[CPT];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j)
+        cn[j] = T->offCN[cg * CPT + j];
+    for (uint32_t it = 0; t_begin + it < t_end; ++it) {
+        ptx::cp_async_wait<STAGES - 2>();
+        __syncthreads(); // tile `it` and its row table visible; the stage of tile it-1 is free
+        issue(it + STAGES - 1);
+        const float* As = reinterpret_cast<const float*>(ring + (it % STAGES) * tile_bytes) + 4 * q;
+        float2 acc[4][CPT / 2]; // column pairs: one packed instruction = two independent fp32 FMAs
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < CPT / 2; ++j)
+                acc[i][j] = make_float2(0.f, 0.f);
+#pragma unroll(KT ? KT : 4)
+        for (uint32_t k = 0; k < K && !(g.debug & 64); ++k) { // (debug & 64: experiment, no math)
+            const float4 a = *reinterpret_cast<const float4*>(As + k * ROWS);
+            float2 b[CPT / 2];
+            const float* brow = Bs + k * NP + cg * CPT;
+#pragma unroll
+            for (int j = 0; j < CPT; j += 2) {
+                if (CPT % 4 == 0 && j % 4 == 0) {
+                    const float4 v = *reinterpret_cast<const float4*>(brow + j);
+                    b[j / 2] = make_float2(v.x, v.y);
+                    b[j / 2 + 1] = make_float2(v.z, v.w);
+                } else if (CPT % 4 != 0) {
+                    b[j / 2] = *reinterpret_cast<const float2*>(brow + j);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float av = i == 0 ? a.x : i == 1 ? a.y : i == 2 ? a.z : a.w;
+                const float2 a2 = make_float2(av, av);
+#pragma unroll
+                for (int j = 0; j < CPT / 2; ++j)
+                    acc[i][j] = __ffma2_rn(a2, b[j], acc[i][j]);
+            }
+        }
+        if (g.debug & 2) // (experiment: no stores)
+            continue;
+        const int64_t* offCM = T->offCM[it % TSLOTS] + 4 * q;
+        if (vec_rows) {
+            const int64_t cm = offCM[0];
+            if (cm < 0)
+                continue;
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) {
+                if (cn[j] < 0)
+                    continue;
+                float4* dst = reinterpret_cast<float4*>(g.C + cm + cn[j]);
+                float4 v;
+                v.x = alpha * ((j & 1) ? acc[0][j / 2].y : acc[0][j / 2].x);
+                v.y = alpha * ((j & 1) ? acc[1][j / 2].y : acc[1][j / 2].x);
+                v.z = alpha * ((j & 1) ? acc[2][j / 2].y : acc[2][j / 2].x);
+                v.w = alpha * ((j & 1) ? acc[3][j / 2].y : acc[3][j / 2].x);
+                if (beta != 0.f) {
+                    const float4 o = __ldcg(dst);
+                    v.x = fmaf(beta, o.x, v.x);
+                    v.y = fmaf(beta, o.y, v.y);
+                    v.z = fmaf(beta, o.z, v.z);
+                    v.w = fmaf(beta, o.w, v.w);
+                }
+                *dst = v;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int64_t cm = offCM[i];
+                if (cm < 0)
+                    continue;
+                float* crow = g.C + cm;
+#pragma unroll
+                for (int j = 0; j < CPT; ++j)
+                    if (cn[j] >= 0) {
+                        const float v = alpha * ((j & 1) ? acc[i][j / 2].y : acc[i][j / 2].x);
+                        crow[cn[j]] = beta != 0.f ? fmaf(beta, __ldcg(crow + cn[j]), v) : v;
+                    }
+            }
+        }
+    }
+    ptx::cp_async_wait_all();
+}
+
 } // namespace
 
 static int skinny_cpt(uint32_t N) { return (int)((N + 3) / 4 + 1) & ~1; } // even, 4 * cpt >= N
+
+int gett_ffma_skinny_mn_smem_bytes(int N, int K)
+{
+    return K * 4 * skinny_cpt((uint32_t)N) * 4 + STAGES * K * ROWS * 4 + (int)sizeof(SkinnyMnTables);
+}
 
 int gett_ffma_skinny_smem_bytes(int N, int K)
 {
@@ -210,6 +385,23 @@ cudaError_t gett_launch_ffma_skinny(const GettKernelArgs& args, int grid, int sm
     const int cpt = skinny_cpt(args.N.size);
     void (*k)(GettKernelArgs);
     const uint32_t K = args.K.size;
+    if (args.loader_a == GETT_LOAD_VEC_FREE) { // A staged MN-major
+#define SKINNY_MN_PICK(CPT) k = K == 24 ? gett_ffma_skinny_mn_kernel<CPT, 24> : K == 32 ? gett_ffma_skinny_mn_kernel<CPT, 32> \
+                                : K == 48 ? gett_ffma_skinny_mn_kernel<CPT, 48> : gett_ffma_skinny_mn_kernel<CPT, 0>
+        switch (cpt) {
+        case 2: SKINNY_MN_PICK(2); break;
+        case 4: SKINNY_MN_PICK(4); break;
+        case 6: SKINNY_MN_PICK(6); break;
+        case 8: SKINNY_MN_PICK(8); break;
+        default: return cudaErrorInvalidValue;
+        }
+#undef SKINNY_MN_PICK
+        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess)
+            return e;
+        k<<<grid, NT, smem, stream>>>(args);
+        return cudaGetLastError();
+    }
 #define SKINNY_PICK(CPT) k = K == 24 ? gett_ffma_skinny_kernel<CPT, 6> : K == 32 ? gett_ffma_skinny_kernel<CPT, 8> \
                              : K == 16 ? gett_ffma_skinny_kernel<CPT, 4> : gett_ffma_skinny_kernel<CPT, 0>
     switch (cpt) {

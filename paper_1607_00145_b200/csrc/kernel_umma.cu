@@ -362,7 +362,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
         float* Sb = S + (ci & (DEPTH - 1)) * (32 * PITCH);
         float* Srow = Sb + lane * PITCH;
         const uint32_t tacc = tmem_base + ((eq * 32u) << 16) + buf * 256;
-        if (CV == 1) {
+        if constexpr (CV == 1) {
 #pragma unroll
             for (uint32_t h = 0; h < Sh::SLOTS / 32; ++h) {
                 uint32_t v[32];

@@ -420,7 +420,9 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     const bool umma_ok = dtype != GETT_F32 && both_vec;
     // fp32 with small N and K and a K-major A: B is read once element by element, so
     // only A has to be gatherable in 16-byte vectors
-    const bool skinny_ok = dtype == GETT_F32 && info.loader_a == GETT_LOAD_VEC_K && p->N.size <= 32 &&
+    const bool skinny_ok = dtype == GETT_F32 &&
+                           (info.loader_a == GETT_LOAD_VEC_K || info.loader_a == GETT_LOAD_VEC_FREE) &&
+                           p->N.size <= 32 &&
                            p->K.size <= (uint32_t)gett_ffma_skinny_max_k() && o.split_k <= 1 &&
                            (o.tile_m == 0 || o.tile_m == gett_ffma_skinny_rows()) && o.tile_n == 0 &&
                            o.tile_k == 0 && o.stages == 0 && o.epilogue != GETT_EPI_STAGED;
@@ -477,7 +479,9 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.tile_k = (int)p->K.size;
         info.stages = 3;
         info.block = 256;
-        info.smem_bytes = gett_ffma_skinny_smem_bytes((int)p->N.size, (int)p->K.size);
+        info.smem_bytes = info.loader_a == GETT_LOAD_VEC_K
+                              ? gett_ffma_skinny_smem_bytes((int)p->N.size, (int)p->K.size)
+                              : gett_ffma_skinny_mn_smem_bytes((int)p->N.size, (int)p->K.size);
         info.epilogue = GETT_EPI_DIRECT;
         info.loader_b = GETT_LOAD_SCALAR; // B is read once, element by element
     } else if (path == GETT_PATH_FFMA) {

@@ -150,6 +150,21 @@ def test_tensor_times_small_matrix_kernel(sizes):
         assert info.tile_m == 128
 
 
+@pytest.mark.parametrize("spec,sizes,vec_rows", [
+    ("C[m0,m1,n0] = A[m0,k,m1] * B[n0,k]", dict(m0=72, m1=11, n0=24, k=24), True),     # rows run along C
+    ("C[m0,n0,m1] = A[m0,m1,k] * B[k,n0]", dict(m0=40, m1=29, n0=17, k=48), True),     # odd N
+    ("C[n0,m0,m1] = A[m0,k,m1] * B[k,n0]", dict(m0=24, m1=37, n0=8, k=20), False),     # C runs along n0
+    ("C[m0,m1,n0] = A[m0,k,m1] * B[n0,k]", dict(m0=256, m1=5, n0=32, k=64), True),     # widest N and K
+    ("C[m0,m1,n0] = A[m0,k,m1] * B[n0,k]", dict(m0=8, m1=300, n0=12, k=7), True),      # K not a multiple of 4
+])
+def test_tensor_times_small_matrix_kernel_a_free_major(spec, sizes, vec_rows):
+    """The small-N, small-K fp32 kernel with A staged MN-major (A's stride-1 mode is free)."""
+    con = parse_spec(spec, sizes)
+    for alpha, beta in [(1.0, 0.0), (0.5, 2.0)]:
+        ratio, info = parity_case(con, F32, "uniform", 23, alpha, beta, repeat=2, epilogue=g.GETT_EPI_DIRECT)
+        assert info.path == g.GETT_PATH_FFMA and info.tile_m == 256 and info.loader_a == g.GETT_LOAD_VEC_FREE
+
+
 @pytest.mark.parametrize("seed", range(48))
 def test_fuzz_random_contractions(seed):
     rng = np.random.default_rng(5000 + seed)
