@@ -1,5 +1,5 @@
 // Strict-fp32 kernel for the bandwidth-bound "tensor times small matrix" regime:
-// N <= 32, K <= 64, A staged K-major (its stride-1 mode is contracted).
+// N <= 64, K <= 64, A staged K-major (its stride-1 mode is contracted).
 //
 // The whole of B (K x N) stays in shared memory for the life of the CTA, so the
 // loop nest of Listing 4 degenerates to the m-loop alone: persistent CTAs stream
@@ -21,7 +21,7 @@ constexpr int TSLOTS = STAGES + 1;
 
 struct SkinnyTables {
     int64_t offCM[TSLOTS][ROWS]; // C offset of each tile row (-1 beyond M)
-    int64_t offCN[32];
+    int64_t offCN[64];
     uint32_t kA[KMAX / 4];       // A offset of each 4-wide k piece, 16-byte units
 };
 
@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
         }
         Bs[i] = v;
     }
-    if (tid < 32) {
+    if (tid < 64) {
         int64_t bn, cn = -1;
         if ((uint32_t)tid < N)
             gett_decompose(g.N, tid, bn, cn);
@@ -198,7 +198,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
 // are one aligned vector of C.
 struct SkinnyMnTables {
     int64_t offCM[TSLOTS][ROWS]; // C offset of each tile row (-1 beyond M)
-    int64_t offCN[32];
+    int64_t offCN[64];
     uint32_t kA[KMAX];           // A offset of each k, 16-byte units
 };
 
@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_mn_kernel(const __grid
         }
         Bs[i] = v;
     }
-    if (tid < 32) {
+    if (tid < 64) {
         int64_t bn, cn = -1;
         if ((uint32_t)tid < N)
             gett_decompose(g.N, tid, bn, cn);
@@ -393,6 +393,10 @@ cudaError_t gett_launch_ffma_skinny(const GettKernelArgs& args, int grid, int sm
         case 4: SKINNY_MN_PICK(4); break;
         case 6: SKINNY_MN_PICK(6); break;
         case 8: SKINNY_MN_PICK(8); break;
+        case 10: SKINNY_MN_PICK(10); break;
+        case 12: SKINNY_MN_PICK(12); break;
+        case 14: SKINNY_MN_PICK(14); break;
+        case 16: SKINNY_MN_PICK(16); break;
         default: return cudaErrorInvalidValue;
         }
 #undef SKINNY_MN_PICK
@@ -409,6 +413,10 @@ cudaError_t gett_launch_ffma_skinny(const GettKernelArgs& args, int grid, int sm
     case 4: SKINNY_PICK(4); break;
     case 6: SKINNY_PICK(6); break;
     case 8: SKINNY_PICK(8); break;
+    case 10: SKINNY_PICK(10); break;
+    case 12: SKINNY_PICK(12); break;
+    case 14: SKINNY_PICK(14); break;
+    case 16: SKINNY_PICK(16); break;
     default: return cudaErrorInvalidValue;
     }
 #undef SKINNY_PICK

@@ -291,7 +291,15 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     {
         const int unitCm = find_unit(im, 2), unitAm = find_unit(im, 0);
         const int64_t vec = dtype == GETT_F32 ? 4 : 8;
-        bool want = unitCm >= 0 && unitAm >= 0 && unitCm != unitAm && im[unitAm].ext % vec == 0 &&
+        // (fp32 with small N and K keeps A on the row side: the small-N kernel streams it, and the
+        //  same split is applied to I_m below)
+        int64_t nsz = 1, ksz = 1;
+        for (const GettMode& m : in)
+            nsz *= m.ext;
+        for (const GettMode& m : ik)
+            ksz *= m.ext;
+        const bool small_nk = dtype == GETT_F32 && nsz <= 64 && ksz <= gett_ffma_skinny_max_k();
+        bool want = !small_nk && unitCm >= 0 && unitAm >= 0 && unitCm != unitAm && im[unitAm].ext % vec == 0 &&
                     im[unitAm].ext > vec && im[unitCm].ext % 4 == 0 && o.epilogue != GETT_EPI_DIRECT &&
                     !(o.reserved[0] & 8192); // (experiment switch: never exchange)
         if (want && dtype == GETT_F32) { // the same alignment the fp32 split asks for
@@ -339,6 +347,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
                 return false;
         return true;
     };
+    bool m_split = false;
     if (dtype == GETT_F32) {
         // fp32 operands can also be gathered element by element (4-byte cp.async), so when
         // the contraction is short (C's traffic outweighs the operands') the set that
@@ -348,14 +357,39 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         int64_t ksize = 1;
         for (const GettMode& m : ik)
             ksize *= m.ext;
+        // Small N and K (the small-N kernel streams A, four consecutive rows per thread and
+        // consecutive threads on consecutive row quads): if C's stride-1 mode is a mode of I_m
+        // other than A's stride-1 mode, split A's mode into 4-wide pieces and put C's mode
+        // right after the piece (Sec. 3.2.1 on I_m): A is still copied in 16-byte vectors and
+        // a warp's stores run along C.
+        int64_t nsize = 1;
+        for (const GettMode& m : in)
+            nsize *= m.ext;
+        const int unitCm = find_unit(im, 2);
+        m_split = leadM >= 0 && unitCm >= 0 && unitCm != leadM && im[leadM].ext % 4 == 0 && nsize <= 64 &&
+                  ksize <= gett_ffma_skinny_max_k() && o.split_k <= 1 && o.tile_n == 0 && o.tile_k == 0 &&
+                  o.stages == 0 && (o.tile_m == 0 || o.tile_m == gett_ffma_skinny_rows()) &&
+                  (o.path == GETT_PATH_AUTO || o.path == GETT_PATH_FFMA);
         if (ksize <= 512) {
-            if (find_unit(im, 2) >= 0 && leadM != find_unit(im, 2))
+            if (find_unit(im, 2) >= 0 && leadM != find_unit(im, 2) && !m_split)
                 leadM = -1;
             if (find_unit(in, 2) >= 0 && leadN != find_unit(in, 2) && !n_split_ok(4))
                 leadN = -1;
         }
     }
     p->tm = order_with_lead(im, leadM);
+    if (m_split) {
+        const int unitCm = find_unit(im, 2);
+        std::vector<GettDigit> t;
+        t.push_back({leadM, 4, 1});
+        t.push_back({unitCm, im[unitCm].ext, 1});
+        if (im[leadM].ext > 4)
+            t.push_back({leadM, im[leadM].ext / 4, 4});
+        for (int i = 0; i < (int)im.size(); ++i)
+            if (i != leadM && i != unitCm)
+                t.push_back({i, im[i].ext, 1});
+        p->tm = t;
+    }
     p->tn = order_with_lead(in, leadN);
     {
         // Sec. 3.2.1: when B's stride-1 mode and C's stride-1 mode are two different
@@ -422,7 +456,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     // only A has to be gatherable in 16-byte vectors
     const bool skinny_ok = dtype == GETT_F32 &&
                            (info.loader_a == GETT_LOAD_VEC_K || info.loader_a == GETT_LOAD_VEC_FREE) &&
-                           p->N.size <= 32 &&
+                           p->N.size <= 64 &&
                            p->K.size <= (uint32_t)gett_ffma_skinny_max_k() && o.split_k <= 1 &&
                            (o.tile_m == 0 || o.tile_m == gett_ffma_skinny_rows()) && o.tile_n == 0 &&
                            o.tile_k == 0 && o.stages == 0 && o.epilogue != GETT_EPI_STAGED;
@@ -475,7 +509,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         // tensor times small matrix: B stays in shared memory, A is streamed once
         p->skinny = 1;
         info.tile_m = gett_ffma_skinny_rows();
-        info.tile_n = 32;
+        info.tile_n = p->N.size <= 32 ? 32 : 64;
         info.tile_k = (int)p->K.size;
         info.stages = 3;
         info.block = 256;

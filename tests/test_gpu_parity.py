@@ -156,6 +156,8 @@ def test_tensor_times_small_matrix_kernel(sizes):
     ("C[n0,m0,m1] = A[m0,k,m1] * B[k,n0]", dict(m0=24, m1=37, n0=8, k=20), False),     # C runs along n0
     ("C[m0,m1,n0] = A[m0,k,m1] * B[n0,k]", dict(m0=256, m1=5, n0=32, k=64), True),     # widest N and K
     ("C[m0,m1,n0] = A[m0,k,m1] * B[n0,k]", dict(m0=8, m1=300, n0=12, k=7), True),      # K not a multiple of 4
+    ("C[m1,m0,n0] = A[m0,k,m1] * B[n0,k]", dict(m0=8, m1=300, n0=12, k=7), False),     # C runs along another mode of A:
+    ("C[b,u,a,c] = A[c,k,a,b] * B[k,u]", dict(a=19, b=40, c=12, u=48, k=48), False),   # ... A's mode is split around it
 ])
 def test_tensor_times_small_matrix_kernel_a_free_major(spec, sizes, vec_rows):
     """The small-N, small-K fp32 kernel with A staged MN-major (A's stride-1 mode is free)."""

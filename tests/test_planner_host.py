@@ -169,7 +169,8 @@ def test_split_k_planning():
 
 def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
     want = {  # key, dtype -> (path, loader_a, loader_b, epilogue)
-        ("cfg1", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_K, g.GETT_EPI_DIRECT),
+        # cfg1: N = 40, K = 48 -> the small-N kernel (A staged MN-major, B read once element by element)
+        ("cfg1", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_SCALAR, g.GETT_EPI_DIRECT),
         # cfg2: plain matrices, every tile is a box of a 2-D tensor map -> TMA
         ("cfg2", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_TMA_FREE, g.GETT_LOAD_TMA_K, g.GETT_EPI_DIRECT),
         # cfg3: small N and K -> B is read once into shared memory, element by element
