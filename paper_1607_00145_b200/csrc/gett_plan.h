@@ -112,7 +112,7 @@ int gett_umma_prod_groups(int stages); // producer groups in use; must divide th
 int gett_ffma_smem_bytes(int tile_m, int tile_n, int stages);
 
 // fp32 kernel for N <= 64, K <= gett_ffma_skinny_max_k(), A K-major (kernel_ffma_skinny.cu).
-int gett_ffma_skinny_smem_bytes(int N, int K);
+int gett_ffma_skinny_smem_bytes(int N, int K, int vec_rows); // vec_rows: c_vec == 1
 int gett_ffma_skinny_mn_smem_bytes(int N, int K); // ... A staged MN-major (its stride-1 mode is free)
 int gett_ffma_skinny_rows();
 int gett_ffma_skinny_max_k();

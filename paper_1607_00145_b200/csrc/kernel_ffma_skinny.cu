@@ -28,16 +28,22 @@ struct SkinnyTables {
 // Row pitch (floats) of an A tile: a multiple of 4 whose quarter is odd, so that the
 // 128-bit reads of eight consecutive rows fall into eight different bank groups.
 __host__ __device__ constexpr uint32_t skinny_pitch(uint32_t K) { return K + (K % 8 == 0 ? 4 : 8); }
+// ... with VR (below): a power of two >= 32, the 16-byte pieces of a row XOR-swizzled by (row / 4) % 8
+__host__ __device__ constexpr uint32_t skinny_pitch_vr(uint32_t K) { return K <= 32 ? 32 : 64; }
 
 // KCT: K / 4 when known at compile time (the k loop is then fully unrolled), 0 = run time
-template <int CPT, int KCT>
+// VR : four consecutive tile rows are one aligned 16-byte vector of C.  A thread then owns rows
+//      4 q .. 4 q + 3 (instead of q, q + 64, ...) and stores 128-bit vectors along the rows.
+template <int CPT, int KCT, bool VR>
 __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_constant__ GettKernelArgs g)
 {
     constexpr int NP = 4 * CPT; // padded row of B in shared memory
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t K = g.K.size, N = g.N.size, Msz = g.M.size;
     const uint32_t KC = KCT ? (uint32_t)KCT : K / 4;
-    const uint32_t pitch = skinny_pitch(K);
+    const uint32_t pitch = VR ? skinny_pitch_vr(K) : skinny_pitch(K);
+    // byte offset of piece kc inside its row
+    auto piece = [&](uint32_t row, uint32_t kc) { return (VR ? (kc ^ ((row >> 2) & 7)) : kc) * 16; };
     const uint32_t tile_bytes = ROWS * pitch * 4;
     float* Bs = reinterpret_cast<float*>(smem);                       // [K][NP]
     uint8_t* ring = smem + K * NP * 4;
@@ -94,7 +100,8 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
                 if (!affine_rows) {
 #pragma unroll 2
                     for (uint32_t kc = 0; kc < KC; ++kc)
-                        ptx::cp_async_16(dst + kc * 16, src + (ok ? ((uint64_t)T->kA[kc] << 4) : 0), ok ? 16u : 0u);
+                        ptx::cp_async_16(dst + piece(row, kc), src + (ok ? ((uint64_t)T->kA[kc] << 4) : 0),
+                                         ok ? 16u : 0u);
                 }
             }
             if (affine_rows) {
@@ -107,7 +114,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
                     const uint32_t row = q / KC, kc = q - row * KC;
                     const uint32_t m = t * ROWS + row;
                     const bool ok = m < Msz;
-                    ptx::cp_async_16(dst0 + row * pitch * 4 + kc * 16,
+                    ptx::cp_async_16(dst0 + row * pitch * 4 + piece(row, kc),
                                      static_cast<const char*>(g.A) +
                                          (ok ? ((uint64_t)m * (uint64_t)g.M.sX[0] * 4 + ((uint64_t)T->kA[kc] << 4)) : 0),
                                      ok ? 16u : 0u);
@@ -144,8 +151,11 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
         for (uint32_t kc = 0; kc < KC && !(g.debug & 64); ++kc) { // (debug & 64: experiment, no math)
             float4 a[RPT];
 #pragma unroll
-            for (int i = 0; i < RPT; ++i)
-                a[i] = *reinterpret_cast<const float4*>(As + (q + QL * i) * pitch + kc * 4);
+            for (int i = 0; i < RPT; ++i) {
+                const uint32_t row = VR ? 4 * q + i : q + QL * i;
+                a[i] = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(As) + row * pitch * 4 +
+                                                        piece(row, kc));
+            }
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
                 float2 b[CPT / 2];
@@ -172,20 +182,45 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
             }
         }
         const int64_t* offCM = T->offCM[it % TSLOTS];
-#pragma unroll
-        for (int i = 0; i < RPT; ++i) {
-            const int64_t cm = offCM[q + QL * i];
+        if constexpr (VR) {
+            const int64_t cm = offCM[4 * q];
             if (cm < 0 || (g.debug & 2)) // (debug & 2: experiment, no stores)
                 continue;
-            float* crow = g.C + cm;
-            float old[CPT];
 #pragma unroll
-            for (int j = 0; j < CPT; ++j)
-                old[j] = (beta != 0.f && cn[j] >= 0) ? __ldcg(crow + cn[j]) : 0.f;
+            for (int j = 0; j < CPT; ++j) {
+                if (cn[j] < 0)
+                    continue;
+                float4* dst = reinterpret_cast<float4*>(g.C + cm + cn[j]);
+                float4 v;
+                v.x = alpha * ((j & 1) ? acc[0][j / 2].y : acc[0][j / 2].x);
+                v.y = alpha * ((j & 1) ? acc[1][j / 2].y : acc[1][j / 2].x);
+                v.z = alpha * ((j & 1) ? acc[2][j / 2].y : acc[2][j / 2].x);
+                v.w = alpha * ((j & 1) ? acc[3][j / 2].y : acc[3][j / 2].x);
+                if (beta != 0.f) {
+                    const float4 o = __ldcg(dst);
+                    v.x = fmaf(beta, o.x, v.x);
+                    v.y = fmaf(beta, o.y, v.y);
+                    v.z = fmaf(beta, o.z, v.z);
+                    v.w = fmaf(beta, o.w, v.w);
+                }
+                *dst = v;
+            }
+        } else {
 #pragma unroll
-            for (int j = 0; j < CPT; ++j)
-                if (cn[j] >= 0)
-                    crow[cn[j]] = fmaf(beta, old[j], alpha * ((j & 1) ? acc[i][j / 2].y : acc[i][j / 2].x));
+            for (int i = 0; i < RPT; ++i) {
+                const int64_t cm = offCM[q + QL * i];
+                if (cm < 0 || (g.debug & 2)) // (debug & 2: experiment, no stores)
+                    continue;
+                float* crow = g.C + cm;
+                float old[CPT];
+#pragma unroll
+                for (int j = 0; j < CPT; ++j)
+                    old[j] = (beta != 0.f && cn[j] >= 0) ? __ldcg(crow + cn[j]) : 0.f;
+#pragma unroll
+                for (int j = 0; j < CPT; ++j)
+                    if (cn[j] >= 0)
+                        crow[cn[j]] = fmaf(beta, old[j], alpha * ((j & 1) ? acc[i][j / 2].y : acc[i][j / 2].x));
+            }
         }
     }
     ptx::cp_async_wait_all();
@@ -370,10 +405,10 @@ int gett_ffma_skinny_mn_smem_bytes(int N, int K)
     return K * 4 * skinny_cpt((uint32_t)N) * 4 + STAGES * K * ROWS * 4 + (int)sizeof(SkinnyMnTables);
 }
 
-int gett_ffma_skinny_smem_bytes(int N, int K)
+int gett_ffma_skinny_smem_bytes(int N, int K, int vec_rows)
 {
-    return K * 4 * skinny_cpt((uint32_t)N) * 4 + STAGES * ROWS * (int)skinny_pitch((uint32_t)K) * 4 +
-           (int)sizeof(SkinnyTables);
+    const int pitch = vec_rows ? (int)skinny_pitch_vr((uint32_t)K) : (int)skinny_pitch((uint32_t)K);
+    return K * 4 * skinny_cpt((uint32_t)N) * 4 + STAGES * ROWS * pitch * 4 + (int)sizeof(SkinnyTables);
 }
 
 int gett_ffma_skinny_max_k() { return KMAX; }
@@ -406,8 +441,14 @@ cudaError_t gett_launch_ffma_skinny(const GettKernelArgs& args, int grid, int sm
         k<<<grid, NT, smem, stream>>>(args);
         return cudaGetLastError();
     }
-#define SKINNY_PICK(CPT) k = K == 24 ? gett_ffma_skinny_kernel<CPT, 6> : K == 32 ? gett_ffma_skinny_kernel<CPT, 8> \
-                             : K == 16 ? gett_ffma_skinny_kernel<CPT, 4> : gett_ffma_skinny_kernel<CPT, 0>
+#define SKINNY_PICK(CPT)                                                                                   \
+    k = vr ? (K == 24   ? gett_ffma_skinny_kernel<CPT, 6, true>                                                \
+              : K == 32 ? gett_ffma_skinny_kernel<CPT, 8, true>                                                \
+                        : gett_ffma_skinny_kernel<CPT, 0, true>)                                               \
+           : (K == 24   ? gett_ffma_skinny_kernel<CPT, 6, false>                                               \
+              : K == 32 ? gett_ffma_skinny_kernel<CPT, 8, false>                                               \
+                        : gett_ffma_skinny_kernel<CPT, 0, false>)
+    const bool vr = args.c_vec == 1; // four consecutive rows are one aligned vector of C
     switch (cpt) {
     case 2: SKINNY_PICK(2); break;
     case 4: SKINNY_PICK(4); break;

@@ -514,7 +514,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.stages = 3;
         info.block = 256;
         info.smem_bytes = info.loader_a == GETT_LOAD_VEC_K
-                              ? gett_ffma_skinny_smem_bytes((int)p->N.size, (int)p->K.size)
+                              ? gett_ffma_skinny_smem_bytes((int)p->N.size, (int)p->K.size, p->c_vec == 1)
                               : gett_ffma_skinny_mn_smem_bytes((int)p->N.size, (int)p->K.size);
         info.epilogue = GETT_EPI_DIRECT;
         info.loader_b = GETT_LOAD_SCALAR; // B is read once, element by element

@@ -150,6 +150,15 @@ def test_tensor_times_small_matrix_kernel(sizes):
         assert info.tile_m == 128
 
 
+@pytest.mark.parametrize("sizes", [dict(m0=40, m1=33, n0=24, k=24), dict(m0=36, m1=9, n0=50, k=64)])
+def test_tensor_times_small_matrix_kernel_scalar_stores(sizes):
+    """The K-major small-N kernel when C does not run along the rows (rows q, q + 64, ... per thread)."""
+    con = parse_spec("C[n0,m0,m1] = A[k,m0,m1] * B[n0,k]", sizes)
+    for alpha, beta in [(1.0, 0.0), (0.5, 2.0)]:
+        ratio, info = parity_case(con, F32, "uniform", 29, alpha, beta, repeat=2, epilogue=g.GETT_EPI_DIRECT)
+        assert info.path == g.GETT_PATH_FFMA and info.tile_m == 256 and info.loader_a == g.GETT_LOAD_VEC_K
+
+
 @pytest.mark.parametrize("spec,sizes,vec_rows", [
     ("C[m0,m1,n0] = A[m0,k,m1] * B[n0,k]", dict(m0=72, m1=11, n0=24, k=24), True),     # rows run along C
     ("C[m0,n0,m1] = A[m0,m1,k] * B[k,n0]", dict(m0=40, m1=29, n0=17, k=48), True),     # odd N
