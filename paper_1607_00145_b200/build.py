@@ -1,4 +1,8 @@
-"""Build the CUDA library in-tree: csrc/*.cu, csrc/*.cpp -> libgett_b200.so (sm_100a)."""
+"""Build the CUDA library in-tree: csrc/*.cu, csrc/*.cpp -> libgett_b200.so (sm_100a).
+
+Sources named *_mc.cu (the CTA-pair variant of the tensor-core kernel) go into a library of
+their own, libgett_b200_mc.so, which the main library loads if it is there; a tree without
+those sources builds and runs the same, without the variant."""
 from __future__ import annotations
 
 import os
@@ -10,6 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libgett_b200.so")
+LIB_MC = os.path.join(HERE, "libgett_b200_mc.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC,-fvisibility=hidden",
@@ -17,14 +22,18 @@ COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC,-fvisibility=hi
 
 
 def sources():
-    return sorted(f for f in os.listdir(CSRC) if f.endswith((".cu", ".cpp")))
+    return sorted(f for f in os.listdir(CSRC) if f.endswith((".cu", ".cpp")) and not f.endswith("_mc.cu"))
+
+
+def sources_mc():
+    return sorted(f for f in os.listdir(CSRC) if f.endswith("_mc.cu"))
 
 
 def _newest_header() -> float:
     t = 0.0
     for d in (CSRC, os.path.join(os.path.dirname(HERE), "include")):
         for f in os.listdir(d):
-            if f.endswith(".h"):
+            if f.endswith((".h", ".cuh")) or (d == CSRC and f == "kernel_umma.cu"):  # (included by *_mc.cu)
                 t = max(t, os.path.getmtime(os.path.join(d, f)))
     return t
 
@@ -55,12 +64,21 @@ def build(verbose: bool = False, force: bool = False) -> str:
     srcs = sources()
     with ThreadPoolExecutor(max_workers=min(8, len(srcs))) as ex:
         objs = list(ex.map(lambda s: _compile(s, verbose), srcs))
-    if not os.path.exists(LIB) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
-        tmp = LIB + f".tmp{os.getpid()}"
+    _link(LIB, objs)
+    mc = sources_mc()
+    if mc:
+        _link(LIB_MC, [_compile(s, verbose) for s in mc])
+    elif os.path.exists(LIB_MC):
+        os.remove(LIB_MC)
+    return LIB
+
+
+def _link(lib: str, objs) -> None:
+    if not os.path.exists(lib) or any(os.path.getmtime(o) > os.path.getmtime(lib) for o in objs):
+        tmp = lib + f".tmp{os.getpid()}"
         subprocess.check_call([NVCC, *ARCH, "-shared", "-o", tmp, *objs, "-lcudart_static",
                                "-Xlinker", "--exclude-libs=ALL"])
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
 
 
 if __name__ == "__main__":

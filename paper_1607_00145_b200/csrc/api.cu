@@ -3,9 +3,11 @@
 // workspace and the status word); gett_contract itself allocates nothing.
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <dlfcn.h>
 
 #include <cstring>
 #include <new>
+#include <string>
 #include <utility>
 
 #include "kernels.h"
@@ -74,6 +76,27 @@ bool encode_map(const GettTmaRecipe& R, int dtype, const void* base, uint64_t* o
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return rc == CUDA_SUCCESS;
+}
+
+// The CTA-pair variant of the tensor-core kernel lives in a library of its own next to this
+// one (it is left out of multi-GPU runs); null if it is not there.
+typedef int (*LaunchPairFn)(const GettKernelArgs*, const GettTmaMaps*, int, int, void*);
+
+LaunchPairFn launch_pair_fn()
+{
+    static LaunchPairFn fn = [] {
+        Dl_info me;
+        if (!dladdr(reinterpret_cast<const void*>(&gett_status_string), &me) || !me.dli_fname)
+            return (LaunchPairFn) nullptr;
+        std::string path(me.dli_fname);
+        const size_t dot = path.rfind(".so");
+        if (dot == std::string::npos)
+            return (LaunchPairFn) nullptr;
+        path.insert(dot, "_mc");
+        void* h = dlopen(path.c_str(), RTLD_NOW | RTLD_LOCAL);
+        return h ? reinterpret_cast<LaunchPairFn>(dlsym(h, "gett_launch_umma_pair")) : (LaunchPairFn) nullptr;
+    }();
+    return fn;
 }
 
 int vec_kind(int loader) // the staging layout behind a loader value
@@ -202,6 +225,29 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     case GETT_PATH_UMMA: {
         alignas(64) GettTmaMaps maps;
         memset(&maps, 0, sizeof maps);
+        if (plan->pair_ok && launch_pair_fn()) {
+            // each CTA of a pair fetches half of the A tile: a K-major A gets a half-height box
+            GettTmaRecipe ra = plan->tma_a;
+            if (args.loader_a == GETT_LOAD_VEC_K)
+                for (int i = 1; i < ra.rank; ++i)
+                    if (!ra.which[i] && ra.digit[i] == 0)
+                        ra.box[i] /= 2;
+            maps.use_a = encode_map(ra, plan->dtype, A, maps.map_a) ? 1 : 0;
+            maps.use_b = encode_map(plan->tma_b, plan->dtype, B, maps.map_b) ? 1 : 0;
+            maps.rank_a = ra.rank;
+            maps.rank_b = plan->tma_b.rank;
+            for (int i = 0; i < 5; ++i) {
+                maps.which_a[i] = ra.which[i];
+                maps.digit_a[i] = ra.digit[i];
+                maps.which_b[i] = plan->tma_b.which[i];
+                maps.digit_b[i] = plan->tma_b.digit[i];
+            }
+            if (maps.use_a && maps.use_b &&
+                launch_pair_fn()(&args, &maps, plan->info.smem_bytes, plan->sm_count, cuda_stream) == 0)
+                break;
+            cudaGetLastError(); // the variant could not run: the ordinary kernel does
+            memset(&maps, 0, sizeof maps);
+        }
         maps.use_a = encode_map(plan->tma_a, plan->dtype, A, maps.map_a) ? 1 : 0;
         maps.use_b = encode_map(plan->tma_b, plan->dtype, B, maps.map_b) ? 1 : 0;
         maps.rank_a = plan->tma_a.rank;

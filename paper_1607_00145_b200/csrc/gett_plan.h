@@ -86,6 +86,7 @@ struct gett_plan {
     int32_t c_vec;
     int32_t skinny; // fp32: B resident in shared memory, A streamed (small N and K)
     int32_t epi_lean; // see GettKernelArgs
+    int32_t pair_ok;  // the CTA-pair variant of the tensor-core kernel applies (used if its library is there)
     int32_t swapped;  // the kernels get the caller's B as their A and vice versa (im / in / ik, tm / tn / tk,
                       // M / N / K and the loaders below are the kernels' view; info is the caller's)
     GettTmaRecipe tma_a, tma_b;

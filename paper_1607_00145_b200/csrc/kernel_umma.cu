@@ -26,6 +26,20 @@
 #include "kernels.h"
 #include "ptx_sm100.cuh"
 
+// The file is compiled a second time, with GETT_UMMA_CLUSTER defined, by the source that adds
+// the CTA-pair variant (two CTAs of a cluster work on two neighbouring tile columns of one
+// tile row and share the A tile: each fetches half of it for both).  Work distribution then
+// runs over tile pairs and clusters instead of tiles and CTAs.
+#ifdef GETT_UMMA_CLUSTER
+#define GETT_WB (blockIdx.x >> 1)  // this CTA's position in the work list ...
+#define GETT_WG (gridDim.x >> 1)   // ... and the list's stride
+#define GETT_WRANK (blockIdx.x & 1u) // which tile of the pair is mine
+#else
+#define GETT_WB blockIdx.x
+#define GETT_WG gridDim.x
+#define GETT_WRANK 0u
+#endif
+
 namespace {
 
 constexpr int MMA_M = 128;            // rows of one tcgen05.mma and of one accumulator buffer
@@ -90,21 +104,30 @@ struct WorkItem {
 
 __device__ __forceinline__ WorkItem decode_work(const GettKernelArgs& g, uint32_t w, uint32_t tile_m)
 {
-    const uint32_t tiles = g.tiles_m * g.tiles_n;
+#ifdef GETT_UMMA_CLUSTER
+    const uint32_t tiles_n = g.tiles_n >> 1; // columns of tile pairs
+#else
+    const uint32_t tiles_n = g.tiles_n;
+#endif
+    const uint32_t tiles = g.tiles_m * tiles_n;
     WorkItem it;
     it.z = w / tiles;
     const uint32_t t = w - it.z * tiles;
     // Tiles are numbered panel by panel: a panel is RASTER_M tile rows high and spans all
     // tile columns, and inside it the row index runs fastest.  The ~148 tiles in flight at
     // any time then share few distinct rows of A and columns of B, which keeps them in L2.
-    const uint32_t per_panel = RASTER_M * g.tiles_n;
+    const uint32_t per_panel = RASTER_M * tiles_n;
     const uint32_t panel = t / per_panel;
     const uint32_t first_m = panel * RASTER_M;
     const uint32_t rows = min((uint32_t)RASTER_M, g.tiles_m - first_m);
     const uint32_t in_panel = t - panel * per_panel;
     const uint32_t tn = in_panel / rows;
     it.m0 = (first_m + (in_panel - tn * rows)) * tile_m;
+#ifdef GETT_UMMA_CLUSTER
+    it.n0 = (2 * tn + GETT_WRANK) * (uint32_t)g.tile_n;
+#else
     it.n0 = tn * (uint32_t)g.tile_n;
+#endif
     it.kbeg = it.z * g.k_per_split;
     it.kend = min(g.K.size, it.kbeg + g.k_per_split);
     it.nslab = (it.kend - it.kbeg + TILE_K - 1) / TILE_K;
@@ -262,7 +285,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
     const bool rmw = beta != 0.f && !(g.debug & 128); // (debug & 128: experiment, old C not read)
     // this warp's set handles the CTA's tiles with local number es, es + 2, ...; `j` counts them
     const uint32_t es = warp >> 2, eq = warp & 3;
-    const uint32_t ncta = total_work > blockIdx.x ? (total_work - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const uint32_t ncta = total_work > GETT_WB ? (total_work - GETT_WB + GETT_WG - 1) / GETT_WG : 0;
     const uint32_t ntile = ncta > es ? (ncta - es + 1) / 2 : 0;
     const uint32_t nchunk = ntile * NCH;
     static_assert(EPI_DEPTH == 2, "row offsets are kept in two scalars");
@@ -273,7 +296,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
         if (cj < nchunk) {
             const uint32_t j = cj / NCH, ch = cj - j * NCH;
             if (ch == 0) {
-                const WorkItem wi = decode_work(g, blockIdx.x + (es + 2 * j) * gridDim.x, MMA_M);
+                const WorkItem wi = decode_work(g, GETT_WB + (es + 2 * j) * GETT_WG, MMA_M);
                 int64_t rc = -1;
                 const uint32_t m = wi.m0 + eq * 32 + lane;
                 if (m < g.M.size)
@@ -472,7 +495,7 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
     int32_t fa[5] = {0, 0, 0, 0, 0}, fb[5] = {0, 0, 0, 0, 0}; // digit indices of the tile origin
     uint32_t first = 0; // slab number of the current work item's first slab
     bool alive = true;
-    for (uint32_t w = blockIdx.x; w < total_work && pg < ng; w += gridDim.x) {
+    for (uint32_t w = GETT_WB; w < total_work && pg < ng; w += GETT_WG) {
         const WorkItem wi = decode_work(g, w, TILE_M);
         // my group's first slab in this item: smallest j with (first + j) % ng == pg
         uint32_t j = (pg + ng - first % ng) % ng;
@@ -525,6 +548,26 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
 #pragma unroll
                     for (int i = 0; i < 5; ++i)
                         c[i] = tm.which_a[i] ? kd[tm.digit_a[i]] : fa[tm.digit_a[i]];
+#ifdef GETT_UMMA_CLUSTER
+                    // my half of the A tile, delivered to both CTAs of the pair (the partner
+                    // fetches the other half); each CTA's barrier counts the whole stage
+                    const uint32_t half = GETT_WRANK;
+                    if (A_VEC_K) { // the map's box is TILE_M / 2 rows high
+#pragma unroll
+                        for (int i = 1; i < 5; ++i)
+                            if (!tm.which_a[i] && tm.digit_a[i] == 0)
+                                c[i] += (int32_t)(half * (TILE_M / 2));
+                        ptx_mc::tma_load_pair(sa + half * (A_STAGE_BYTES / 2), tm.map_a, fullbar, tm.rank_a, c);
+                    } else {
+                        c[0] += (int32_t)(half * (TILE_M / 2));
+#pragma unroll
+                        for (int b = 0; b < TILE_M / 128; ++b) {
+                            ptx_mc::tma_load_pair(sa + (half * (TILE_M / 128) + b) * MN_BLOCK_BYTES, tm.map_a, fullbar,
+                                                  tm.rank_a, c);
+                            c[0] += 64;
+                        }
+                    }
+#else
                     if (A_VEC_K) {
                         ptx::tma_load(sa, tm.map_a, fullbar, tm.rank_a, c);
                     } else {
@@ -534,6 +577,7 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
                             c[0] += 64;
                         }
                     }
+#endif
                 }
                 if (tmaB) {
 #pragma unroll
@@ -589,13 +633,21 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
     const uint32_t stage0 = ptx::smem_u32(smem);
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef GETT_UMMA_CLUSTER
+    const uint32_t total_work = g.tiles_m * (g.tiles_n >> 1) * g.split_k; // tile pairs
+#else
     const uint32_t total_work = g.tiles_m * g.tiles_n * g.split_k;
+#endif
     volatile int* abort_flag = &T->abort_flag;
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < stages; ++s) {
             ptx::mbar_init(ptx::smem_u32(&T->full[s]), g.prod_groups == 1 ? PROD_THREADS : GROUP_LANES); // the slab's producers
+#ifdef GETT_UMMA_CLUSTER
+            ptx::mbar_init(ptx::smem_u32(&T->empty[s]), 2); // both CTAs of the pair are done with the stage
+#else
             ptx::mbar_init(ptx::smem_u32(&T->empty[s]), 1);
+#endif
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(ptx::smem_u32(&T->acc_full[b]), 1);
@@ -612,6 +664,9 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = T->tmem_base;
+#ifdef GETT_UMMA_CLUSTER
+    ptx_mc::cluster_sync(); // the partner's barriers exist before anything is sent to them
+#endif
 
     if (warp >= PROD_WARP0) {
         // Producers.  With a ring of one stage (tiles of a single slab) all producer warps
@@ -640,7 +695,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
             const uint32_t sbo = (g.debug & 1) ? MN_BLOCK_BYTES : ATOM_BYTES;
             uint32_t it = 0, local = 0;
             bool alive = true;
-            for (uint32_t w = blockIdx.x; w < total_work && alive; w += gridDim.x, ++local) {
+            for (uint32_t w = GETT_WB; w < total_work && alive; w += GETT_WG, ++local) {
                 const WorkItem wi = decode_work(g, w, TILE_M);
                 // 128-row tiles alternate between the two accumulator buffers; a 256-row tile
                 // uses both (rows 0-127 in buffer 0, rows 128-255 in buffer 1)
@@ -677,7 +732,12 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                             ptx::umma_f16(d_tmem + h * 256, ad, bd, idesc, (j | kk) ? 1u : 0u);
                         }
                     }
+#ifdef GETT_UMMA_CLUSTER
+                    // ... in both CTAs: the partner's copies land in this stage too
+                    ptx_mc::umma_commit_pair(ptx::smem_u32(&T->empty[s]));
+#else
                     ptx::umma_commit(ptx::smem_u32(&T->empty[s])); // stage reusable once these MMAs retire
+#endif
                 }
                 if (alive) {
                     ptx::umma_commit(ptx::smem_u32(&T->acc_full[buf]));
@@ -711,8 +771,8 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
         uint32_t j = 0; // counts this set's tiles
         // 128-row tiles: set es takes every other tile.  256-row tiles: both sets work on
         // every tile, set es on its rows 128 es .. 128 es + 127.
-        const uint32_t w_first = blockIdx.x + (TWO_HALVES ? 0u : es * gridDim.x);
-        const uint32_t w_step = (TWO_HALVES ? 1u : 2u) * gridDim.x;
+        const uint32_t w_first = GETT_WB + (TWO_HALVES ? 0u : es * GETT_WG);
+        const uint32_t w_step = (TWO_HALVES ? 1u : 2u) * GETT_WG;
         for (uint32_t w = w_first; w < total_work && !staged; w += w_step, ++j) {
             WorkItem wi = decode_work(g, w, TILE_M);
             if (TWO_HALVES)
@@ -781,6 +841,9 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
 
     ptx::tc_fence_before();
     __syncthreads();
+#ifdef GETT_UMMA_CLUSTER
+    ptx_mc::cluster_sync(); // the partner no longer writes to this CTA's shared memory or barriers
+#endif
     if (threadIdx.x == 0 && T->abort_flag && g.status)
         *g.status = GETT_ERR_TIMEOUT;
     if (warp == MMA_WARP) {
@@ -791,6 +854,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
 
 } // namespace
 
+#ifndef GETT_UMMA_CLUSTER
 int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged_cv, int lean)
 {
     return 1024 + stages * (int)stage_bytes((uint32_t)tile_m, (uint32_t)tile_n) + (int)sizeof(SmemTables) +
@@ -847,3 +911,4 @@ cudaError_t gett_launch_umma(const GettKernelArgs& args, const GettTmaMaps& maps
         return launch_tn<false, true>(args, maps, grid, smem, stream);
     return launch_tn<false, false>(args, maps, grid, smem, stream);
 }
+#endif // !GETT_UMMA_CLUSTER

@@ -680,6 +680,10 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.grid = (int32_t)std::min<uint64_t>(tiles * split, (uint64_t)sms);
     if (p->skinny) // persistent: two CTAs per SM stream the row tiles
         info.grid = (int32_t)std::min<uint64_t>(p->tiles_m, 2ull * sms);
+    // two neighbouring 256 x 256 tiles per CTA pair, A shared between the two CTAs
+    p->pair_ok = path == GETT_PATH_UMMA && p->tma_a.enabled && p->tma_b.enabled && info.tile_m == 256 &&
+                 info.tile_n == 256 && info.epilogue == GETT_EPI_DIRECT && split == 1 && p->tiles_n % 2 == 0 &&
+                 !(p->debug & 16384); // (experiment switch: never)
     info.swapped = p->swapped;
     if (p->swapped) { // report the caller's view
         std::swap(info.M, info.N);

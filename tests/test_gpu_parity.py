@@ -136,6 +136,33 @@ def test_fp32_64_row_tiles(spec, sizes):
     parity_case(con, F32, "uniform", 17, 1.0, 0.5, tile_m=64, split_k=2)
 
 
+@pytest.mark.parametrize("spec,sizes", [
+    ("C[m,n] = A[m,k] * B[k,n]", dict(m=648, n=1000, k=200)),    # A in boxes of 64 rows, ragged M, N and K
+    ("C[m,n] = A[k,m] * B[n,k]", dict(m=520, n=520, k=136)),     # K-major A: half-height boxes
+])
+def test_cta_pair_variant_equals_the_single_cta_kernel(spec, sizes):
+    """Two CTAs per pair of 256 x 256 tiles sharing the A tile (used when its library is there and
+    the number of tile columns is even) against the oracle and, bit for bit, against the ordinary
+    kernel (same arithmetic, same order)."""
+    import torch
+    from workloads import make_inputs
+    con = parse_spec(spec, sizes)
+    for dtype in (BF16_F32, F16_F32):
+        parity_case(con, dtype, "normal", 41, 1.0, 0.5, repeat=2, tile_m=256, tile_n=256)
+        a, b, c = make_inputs(con, dtype, "normal", 41, 0.5)
+        outs = []
+        for switch in (0, 16384):  # 16384: never use the pair variant
+            da = torch.from_numpy(a.view(np.int16)).cuda()
+            db = torch.from_numpy(b.view(np.int16)).cuda()
+            dc = torch.from_numpy(c).cuda()
+            p = g.Plan(con, dtype, tile_m=256, tile_n=256, reserved0=switch)
+            p(1.0, da, db, 0.5, dc)
+            torch.cuda.synchronize()
+            assert p.device_status() == 0
+            outs.append(dc.cpu())
+        assert torch.equal(outs[0], outs[1])
+
+
 @pytest.mark.parametrize("sizes", [dict(m0=40, m1=33, n0=24, k=24), dict(m0=300, m1=7, n0=5, k=12),
                                    dict(m0=64, m1=9, n0=32, k=64), dict(m0=17, m1=3, n0=1, k=4)])
 def test_tensor_times_small_matrix_kernel(sizes):
