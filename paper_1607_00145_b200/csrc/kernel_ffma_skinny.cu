@@ -52,18 +52,20 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
     const int tid = threadIdx.x;
     const uint32_t ntiles = g.tiles_m;
 
-    // ---- B and the tile-independent tables, once ----
-    for (uint32_t i = tid; i < K * NP; i += NT) {
-        const uint32_t k = i / NP, n = i - k * NP;
-        float v = 0.f;
-        if (n < N) {
-            int64_t bn, cn, ak, bk;
-            gett_decompose(g.N, n, bn, cn);
-            gett_decompose(g.K, k, ak, bk);
-            v = __ldg(static_cast<const float*>(g.B) + bn + bk);
+    // ---- the tile-independent tables, once (B follows the first copies of A, below) ----
+    auto fill_b = [&]() {
+        for (uint32_t i = tid; i < K * NP; i += NT) {
+            const uint32_t k = i / NP, n = i - k * NP;
+            float v = 0.f;
+            if (n < N) {
+                int64_t bn, cn, ak, bk;
+                gett_decompose(g.N, n, bn, cn);
+                gett_decompose(g.K, k, ak, bk);
+                v = __ldg(static_cast<const float*>(g.B) + bn + bk);
+            }
+            Bs[i] = v;
         }
-        Bs[i] = v;
-    }
+    };
     if (tid < 64) {
         int64_t bn, cn = -1;
         if ((uint32_t)tid < N)
@@ -124,9 +126,10 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
         ptx::cp_async_commit();
     };
 
-    __syncthreads(); // kA ready
+    __syncthreads(); // kA, offCN ready
     for (uint32_t s = 0; s < STAGES - 1; ++s)
         issue(s);
+    fill_b(); // while the first tiles are on their way; visible after the loop's first barrier
 
     const uint32_t q = tid % QL, cg = tid / QL; // rows q + QL i; a warp shares one column group
     const float alpha = g.alpha, beta = g.beta;
@@ -253,17 +256,19 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_mn_kernel(const __grid
     const int tid = threadIdx.x;
     const uint32_t ntiles = g.tiles_m;
 
-    for (uint32_t i = tid; i < K * NP; i += NT) {
-        const uint32_t k = i / NP, n = i - k * NP;
-        float v = 0.f;
-        if (n < N) {
-            int64_t bn, cn, ak, bk;
-            gett_decompose(g.N, n, bn, cn);
-            gett_decompose(g.K, k, ak, bk);
-            v = __ldg(static_cast<const float*>(g.B) + bn + bk);
+    auto fill_b = [&]() {
+        for (uint32_t i = tid; i < K * NP; i += NT) {
+            const uint32_t k = i / NP, n = i - k * NP;
+            float v = 0.f;
+            if (n < N) {
+                int64_t bn, cn, ak, bk;
+                gett_decompose(g.N, n, bn, cn);
+                gett_decompose(g.K, k, ak, bk);
+                v = __ldg(static_cast<const float*>(g.B) + bn + bk);
+            }
+            Bs[i] = v;
         }
-        Bs[i] = v;
-    }
+    };
     if (tid < 64) {
         int64_t bn, cn = -1;
         if ((uint32_t)tid < N)
@@ -305,9 +310,10 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_mn_kernel(const __grid
         ptx::cp_async_commit();
     };
 
-    __syncthreads(); // kA ready
+    __syncthreads(); // kA, offCN ready
     for (uint32_t s = 0; s < STAGES - 1; ++s)
         issue(s);
+    fill_b(); // while the first tiles are on their way; visible after the loop's first barrier
 
     const uint32_t q = tid % QL, cg = tid / QL; // rows 4 q ..; a warp shares one column group
     const float alpha = g.alpha, beta = g.beta;
