@@ -31,3 +31,21 @@ def test_status_strings():
     assert g.gett_status_string(0) == "ok"
     assert len({g.gett_status_string(i) for i in range(9)}) == 9
     assert g.gett_status_string(99) == "unknown status"
+
+
+def test_optional_pair_library_is_self_contained():
+    """The CTA-pair variant lives in a library of its own next to the main one: when its sources
+    are in the tree it is built, loads without a GPU and exports its one entry point; without
+    them the main library is complete by itself (checked by every other test)."""
+    from paper_1607_00145_b200 import library_path
+    src = os.path.join(ROOT, "paper_1607_00145_b200", "csrc", "kernel_umma_mc.cu")
+    pair = library_path().replace(".so", "_mc.so")
+    if not os.path.exists(src):
+        assert not os.path.exists(pair)
+        return
+    assert os.path.exists(pair), "run python -m paper_1607_00145_b200.build"
+    assert hasattr(ctypes.CDLL(pair), "gett_launch_umma_pair")
+    # the files that name copies delivered to a whole cluster are listed for multi-GPU runs
+    listed = open(os.path.join(ROOT, ".gpurunignore.multi")).read()
+    for f in ("csrc/kernel_umma_mc.cu", "csrc/ptx_sm100_mc.cuh", "libgett_b200_mc.so"):
+        assert f in listed
