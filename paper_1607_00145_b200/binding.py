@@ -101,7 +101,19 @@ def _load() -> ctypes.CDLL:
     return lib
 
 
-_lib = _load()
+class _LazyLibrary:
+    """The shared library, loaded at the first call (so that importing the package -- and its
+    `build` submodule on a fresh checkout -- does not need it).  A missing library raises
+    ImportError at that first call: there is no fallback implementation."""
+    _cdll = None
+
+    def __getattr__(self, name):
+        if _LazyLibrary._cdll is None:
+            _LazyLibrary._cdll = _load()
+        return getattr(_LazyLibrary._cdll, name)
+
+
+_lib = _LazyLibrary()
 
 
 class GettError(RuntimeError):

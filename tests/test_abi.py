@@ -49,3 +49,24 @@ def test_optional_pair_library_is_self_contained():
     listed = open(os.path.join(ROOT, ".gpurunignore.multi")).read()
     for f in ("csrc/kernel_umma_mc.cu", "csrc/ptx_sm100_mc.cuh", "libgett_b200_mc.so"):
         assert f in listed
+
+
+def test_package_and_build_module_import_without_the_library(tmp_path):
+    """A fresh checkout has no shared library yet: importing the package and its build module
+    must still work (the library is loaded at the first call), and a call without the library
+    must fail loudly instead of falling back to anything."""
+    import subprocess
+    import sys
+    code = ("import os, sys\n"
+            f"sys.path.insert(0, {ROOT!r})\n"
+            f"os.environ['GETT_LIBRARY'] = {str(tmp_path / 'absent.so')!r}\n"
+            "import paper_1607_00145_b200 as g\n"
+            "from paper_1607_00145_b200 import build\n"
+            "assert callable(build.build)\n"
+            "try:\n"
+            "    g.gett_status_string(0)\n"
+            "except ImportError as e:\n"
+            "    print('loud:', 'no fallback' in str(e))\n")
+    r = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    assert "loud: True" in r.stdout
