@@ -7,8 +7,11 @@
 One step = one gett_contract call (pack A/B tiles, macro-kernel, alpha/beta
 update of C; plus the slice reduction when the plan splits K) over one seeded
 synthetic input set.  The headline line is the 8192^3 GEMM control through the
-tensor path; `--all` appends the other workloads and the equal-GEMM ratios under
-"workloads".  Prints exactly one JSON line on rank 0.
+tensor path; the same line carries, under "workloads", one row per workload / dtype /
+split-K variant (time, TFLOP/s, GB/s, roofline fraction, plan, clocks, ratio to the
+equal-sized GEMM, sampled parity against the CPU oracle) and, under "targets", which of the
+seven workload/dtype pairs reach 0.70 of their roofline (`--no-workloads` leaves both out).
+Prints exactly one JSON line on rank 0.
 """
 from __future__ import annotations
 
@@ -48,6 +51,48 @@ def _peaks():
 # figure exists for it; the clock is the one seen during the timed region).
 def _fp32_peak_tflops(sm_mhz: float) -> float:
     return 148 * 128 * 2 * sm_mhz * 1e6 / 1e12
+
+
+def measure_ffma_peak(torch, index: int):
+    """fp32 FMA rate of a register-only loop (plain and two-wide packed FMAs), timed with CUDA
+    events: the measured denominator of the strict-fp32 roofline fractions."""
+    import ctypes
+    path = os.path.join(ROOT, "paper_1607_00145_b200", "libgett_b200_bench.so")
+    if not os.path.exists(path):
+        return None
+    lib = ctypes.CDLL(path)
+    fn = lib.gett_bench_ffma_peak
+    fn.restype = ctypes.c_longlong
+    fn.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
+    out = torch.zeros(4, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+    sms = torch.cuda.get_device_properties(index).multi_processor_count
+    res = {}
+    with clock_sampler(index) as clk:
+        for name, packed in (("plain", 0), ("packed", 1)):
+            best = 0.0
+            for rep in range(6):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fmas = fn(packed, 4096, 2 * sms, out.data_ptr(), stream.cuda_stream)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if fmas < 0:
+                    return None
+                if rep:  # the first launch is a warm-up
+                    best = max(best, 2.0 * fmas / (e0.elapsed_time(e1) / 1e3) / 1e12)
+            res[name] = best
+        t0 = time.perf_counter()  # long enough for a few clock samples
+        while time.perf_counter() - t0 < 0.3:
+            fn(1, 4096, 2 * sms, out.data_ptr(), stream.cuda_stream)
+            torch.cuda.synchronize()
+    c = clk.summary()
+    res["tflops"] = max(res["plain"], res["packed"])
+    res["sm_mhz"] = c["sm_mhz"]
+    res["reasons"] = c["reasons"]
+    res["derived_at_sampled_clock"] = _fp32_peak_tflops(c["sm_mhz"]) if c["sm_mhz"] else None
+    res["how"] = "register-only FMA loop, 32 chains/thread, 2 x 1024 threads per SM, best of 5, CUDA events"
+    return res
 
 
 class NvmlSampler:
@@ -358,7 +403,8 @@ def run_ours(args):
     value = replicas_value(flops, world, sec_per_step)
     clocks = clk.summary()
     sm_mhz = clocks["sm_mhz"] or 1965.0
-    fp32_peak = _fp32_peak_tflops(sm_mhz)
+    ffma = measure_ffma_peak(torch, local) if rank == 0 else None
+    fp32_peak = ffma["tflops"] if ffma else _fp32_peak_tflops(sm_mhz)
 
     # ---- roofline of the contraction kernel ----
     avg = float(per.mean())
@@ -376,14 +422,20 @@ def run_ours(args):
     else:
         achieved = flops / avg / 1e12
         peak, runit = fp32_peak, "TFLOP/s"
-        peak_note = f"derived: 148 SM x 128 FMA lanes x 2 x {sm_mhz:.0f} MHz sampled"
-    traffic = None
+        peak_note = ("measured in this run: register-only FMA loop" if ffma else
+                     f"derived: 148 SM x 128 FMA lanes x 2 x {sm_mhz:.0f} MHz sampled")
+    # DRAM bytes of one launch: not measured by this run (it needs a profiler pass); the figure
+    # is the one-pass ncu capture of this same workload that the named summary records
+    traffic, traffic_source = None, None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
+    if os.path.exists(tpath) and not scale:
         with open(tpath) as f:
-            traffic = json.load(f).get(f"{w.key}:{DTYPE_NAMES[dtype]}:{info['path']}")
+            ent = json.load(f).get(f"{w.key}:{DTYPE_NAMES[dtype]}:{info['path']}")
+        if isinstance(ent, dict):
+            traffic, traffic_source = ent.get("bytes"), ent.get("source")
     roofline = {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit,
-                "frac": achieved / peak, "traffic": traffic, "peak_note": peak_note,
+                "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_source,
+                "peak_note": peak_note,
                 "kernel_ms_avg": avg * 1e3, "kernel_ms_min": float(per.min()) * 1e3,
                 "roofline_time_ms": t_roof * 1e3}
 
@@ -392,8 +444,11 @@ def run_ours(args):
         out = {"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": sec_per_step * 1e3,
                "config": {"workload": f"{w.key} {DTYPE_NAMES[dtype]} {M}x{N}x{K}", "info": info},
                "roofline": roofline, "clocks": clocks}
+        if ffma:
+            out["ffma_peak"] = ffma
         if args.all:
             out["workloads"] = run_all(torch, g, peaks, fp32_peak, args)
+            out["targets"] = targets_summary(out["workloads"])
         if args.pool:
             out.update(run_pool(torch, g, peaks, args))
     elif rank == 0:
@@ -471,7 +526,7 @@ def run_ours(args):
 
         # ---- equal-sized GEMM through the same kernels (Sec. 7) ----
         extra = {}
-        if con.A.labels != [0, 2] or len(con.C.labels) != 2:
+        if not con.is_plain_gemm():
             eg = equal_gemm(con)
             ga, gb, gc = make_inputs(eg, dtype, w.dist, w.seed, w.beta)
             gdev = (_to_dev(ga, torch), _to_dev(gb, torch), _to_dev(gc, torch))
@@ -495,8 +550,12 @@ def run_ours(args):
             "roofline": roofline, "cpu_baseline": base, "e2e": e2e,
             "gpu_launches": args.steps * launches_per_step, "clocks": clocks, **extra,
         }
-        if args.all:
+        if ffma:
+            out["ffma_peak"] = ffma
+        if not args.no_workloads and world == 1:
+            del dev
             out["workloads"] = run_all(torch, g, peaks, fp32_peak, args)
+            out["targets"] = targets_summary(out["workloads"])
     plan.close()
     if rank == 0:
         print(json.dumps(out))
@@ -504,16 +563,74 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def run_all(torch, g, peaks, fp32_peak, args):
-    """Every workload/dtype pair: TFLOP/s, roofline fraction, equal-GEMM ratio."""
+def time_plan(torch, plan, alpha, beta, dev, steps, warmup, flush):
+    """Per-launch device times (seconds, one CUDA-event pair per launch on the launching
+    stream) of a plan on resident inputs, the L2 flushed between launches when `flush` is
+    given; returns (times, clock summary)."""
+    a, b, c = dev
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        plan(alpha, a, b, beta, c, stream)
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    with clock_sampler(torch.cuda.current_device()) as clk:
+        t0 = time.perf_counter()
+        for e0, e1 in evs:
+            if flush is not None:
+                flush.zero_()
+            e0.record(stream)
+            plan(alpha, a, b, beta, c, stream)
+            e1.record(stream)
+        torch.cuda.synchronize()
+        while time.perf_counter() - t0 < 0.05:  # at least a few clock samples under load
+            plan(alpha, a, b, beta, c, stream)
+            torch.cuda.synchronize()
+    if plan.device_status() != 0:
+        raise RuntimeError(f"device status {plan.device_status()}")
+    return np.array([e0.elapsed_time(e1) for e0, e1 in evs]) / 1e3, clk.summary()
+
+
+def equal_gemm_seconds(torch, g, con, dtype, alpha, beta, steps, flush):
+    """Median launch time of the plain GEMM with the same M, N, K through the same library
+    (Sec. 7: the equal-sized GEMM line); its operands are seeded uniform[-1, 1) device draws."""
+    eg = equal_gemm(con)
+    gen = torch.Generator(device="cuda").manual_seed(1234)
+    def draw(n, as16):
+        x = torch.empty(n, dtype=torch.float32, device="cuda").uniform_(-1.0, 1.0, generator=gen)
+        return x.to(torch.bfloat16).view(torch.int16) if as16 else x
+    dev = (draw(eg.A.span, dtype != F32), draw(eg.B.span, dtype != F32), draw(eg.C.span, False))
+    plan = g.Plan(eg, dtype)
+    try:
+        t, _ = time_plan(torch, plan, alpha, beta, dev, steps, 3, flush)
+        info = plan.info.as_dict()
+    finally:
+        plan.close()
+    return float(np.median(t)), info
+
+
+TARGET_PAIRS = [("cfg2", "bf16"), ("cfg2", "f32"), ("cfg3", "f32"), ("cfg4", "bf16"), ("cfg4", "f32"),
+                ("cfg5", "bf16"), ("cfg5", "f32")]
+
+
+def run_all(torch, g, peaks, fp32_peak, args, keys=None):
+    """One row per workload / dtype / variant: launch time (median and min of per-launch CUDA
+    events), TFLOP/s, GB/s, roofline fraction and bound, the plan, the SM clock and throttle
+    reasons sampled during the row, the ratio to the equal-sized GEMM through the same library,
+    and -- the row's CPU-baseline leg -- the oracle timed on a bounded sample of the row's
+    outputs, whose values also give the row's acceptance ratio.  fp32 fractions use the FMA
+    peak measured in this run (`fp32_peak`)."""
+    import oracle
     rows = []
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    for key in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "splitk", "splitk_vec"):
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for key in keys or ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "splitk", "splitk_vec"):
         w = workload(key)
+        con = w.contraction
+        M, N, K = con.mnk()
         for dtype in w.dtypes:
-            con = w.contraction
             a, b, c = make_inputs(con, dtype, w.dist, w.seed, w.beta)
             dev = (_to_dev(a, torch), _to_dev(b, torch), _to_dev(c, torch))
+            small = a.nbytes + b.nbytes + c.nbytes * (2 if w.beta != 0.0 else 1) <= 2 * 126e6
+            flush = flush_buf if small else None
             variants = [("auto", {})]
             if key == "cfg3":
                 # K = 24 is one slab of the vector kernels; only the scalar path can slice it
@@ -522,34 +639,83 @@ def run_all(torch, g, peaks, fp32_peak, args):
             if key in ("splitk", "splitk_vec"):
                 variants += [("split_k=1", {"split_k": 1}), ("split_k=4", {"split_k": 4}),
                              ("split_k=16", {"split_k": 16})]
+            # sampled outputs for the parity / CPU-baseline leg (the same for every variant)
+            rng = np.random.default_rng(7)
+            npts = int(max(64, min(4096, args.row_macs // max(K, 1))))
+            ext = np.array(con.C.extents, dtype=np.int64)
+            pts = np.concatenate([np.zeros((1, len(ext)), np.int64), (ext - 1)[None, :],
+                                  np.stack([rng.integers(0, e, npts) for e in ext], axis=1)], axis=0)
+            off = (pts * np.array(con.C.strides, dtype=np.int64)).sum(axis=1)
+            cores = oracle.default_threads()
+            t0 = time.perf_counter()
+            ref, absacc = oracle.points(con, dtype, w.alpha, a, b, w.beta, c, pts, threads=cores)
+            t_cpu = time.perf_counter() - t0
+            scale = abs(w.alpha) * absacc
+            if w.beta != 0.0:
+                scale = scale + abs(w.beta) * np.abs(c[off].astype(np.float64))
+            off_dev = torch.from_numpy(off).cuda()
             for name, opts in variants:
+                row = {"workload": key, "dtype": DTYPE_NAMES[dtype], "variant": name, "mnk": [M, N, K]}
                 try:
-                    t, info = time_contraction(torch, g, con, dtype, w.alpha, w.beta, dev,
-                                               args.all_steps, 3, opts)
+                    plan = g.Plan(con, dtype, **opts)
                 except Exception as e:  # an unsupported forced option is reported, not fatal
-                    rows.append({"workload": key, "dtype": DTYPE_NAMES[dtype], "variant": name,
-                                 "error": str(e)})
+                    row["error"] = str(e)
+                    rows.append(row)
                     continue
-                flush.zero_()
-                mhz = info["clocks"]["sm_mhz"] or 1965.0
-                t_roof, bound = roofline_time_s(con, dtype, w.beta, peaks, _fp32_peak_tflops(mhz))
-                row = {"workload": key, "dtype": DTYPE_NAMES[dtype], "variant": name,
-                       "ms": t * 1e3, "tflops": con.flops() / t / 1e12,
-                       "gbs": con.compulsory_bytes(dtype, w.beta) / t / 1e9, "bound": bound,
-                       "roofline_frac": t_roof / t, "path": info["path"],
-                       "tile": [info["tile_m"], info["tile_n"], info["tile_k"]],
-                       "split_k": info["split_k"], "sm_mhz": mhz}
-                if name == "auto" and key != "cfg2" and not args.kernel_only:
-                    eg = equal_gemm(con)
-                    ga, gb, gc = make_inputs(eg, dtype, w.dist, w.seed, w.beta)
-                    gdev = (_to_dev(ga, torch), _to_dev(gb, torch), _to_dev(gc, torch))
-                    t_eq, _ = time_contraction(torch, g, eg, dtype, w.alpha, w.beta, gdev,
-                                               args.all_steps, 3)
-                    row["speedup_vs_equal_gemm"] = t_eq / t
-                    del gdev
+                try:
+                    # parity on a fresh C (NaN where beta == 0: C must not be read)
+                    if w.beta == 0.0:
+                        dev[2].fill_(float("nan"))
+                    else:
+                        dev[2].copy_(torch.from_numpy(c))
+                    plan(w.alpha, dev[0], dev[1], w.beta, dev[2], torch.cuda.current_stream())
+                    torch.cuda.synchronize()
+                    got = dev[2][off_dev].cpu().numpy().astype(np.float64)
+                    parity = float(np.max(np.abs(got - ref)) / np.max(scale)) if np.all(np.isfinite(got)) \
+                        else float("inf")
+                    if w.beta != 0.0:
+                        dev[2].copy_(torch.from_numpy(c))
+                    steps = args.all_steps if M * N * K < 4e12 else max(3, args.all_steps // 2)
+                    t, clocks = time_plan(torch, plan, w.alpha, w.beta, dev, steps, 3, flush)
+                    info = plan.info.as_dict()
+                finally:
+                    plan.close()
+                med, tmin = float(np.median(t)), float(t.min())
+                t_roof, bound = roofline_time_s(con, dtype, w.beta, peaks, fp32_peak)
+                row.update({
+                    "ms": med * 1e3, "ms_min": tmin * 1e3, "tflops": con.flops() / med / 1e12,
+                    "gbs": con.compulsory_bytes(dtype, w.beta) / med / 1e9, "bound": bound,
+                    "roofline_ms": t_roof * 1e3, "roofline_frac": t_roof / med,
+                    "roofline_frac_best": t_roof / tmin,
+                    "path": info["path"], "tile": [info["tile_m"], info["tile_n"], info["tile_k"]],
+                    "stages": info["stages"], "loaders": [info["loader_a"], info["loader_b"]],
+                    "epilogue": info["epilogue"], "split_k": info["split_k"], "grid": info["grid"],
+                    "swapped": info["swapped"], "l2": "flushed" if small else "inputs_larger_than_l2",
+                    "sm_mhz": clocks["sm_mhz"], "clock_reasons": clocks["reasons"],
+                    "parity_ratio": parity, "parity_points": int(len(off)), "parity_ok": bool(parity <= 1e-5),
+                    "cpu_baseline": {"value": 2.0 * len(off) * K / t_cpu / 1e12, "unit": UNIT, "cores": cores,
+                                     "kind": "oracle", "sample": f"{len(off)} outputs, {t_cpu:.2f} s"},
+                })
+                if name == "auto" and not con.is_plain_gemm():
+                    t_eq, ginfo = equal_gemm_seconds(torch, g, con, dtype, w.alpha, w.beta, steps, flush)
+                    row["equal_gemm_ms"] = t_eq * 1e3
+                    row["speedup_vs_equal_gemm"] = t_eq / med
                 rows.append(row)
-            del dev
+            del dev, off_dev
     return rows
+
+
+def targets_summary(rows):
+    """The seven workload/dtype pairs of the stated target: roofline fraction of the automatic
+    plan and whether it reaches 0.70."""
+    out = []
+    for key, dt in TARGET_PAIRS:
+        r = [x for x in rows if x.get("workload") == key and x.get("dtype") == dt and x.get("variant") == "auto"
+             and "roofline_frac" in x]
+        if r:
+            out.append({"workload": key, "dtype": dt, "bound": r[0]["bound"], "roofline_frac": r[0]["roofline_frac"],
+                        "met": bool(r[0]["roofline_frac"] >= 0.70), "parity_ok": r[0]["parity_ok"]})
+    return {"threshold": 0.70, "pairs": out, "met": sum(1 for x in out if x["met"]), "of": len(out)}
 
 
 def run_pool(torch, g, peaks, args):
@@ -604,8 +770,12 @@ def main():
                     help="with --kernel-only: also time the seeded pool of synthetic contractions")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end, equal-GEMM and CPU legs (profiling runs)")
-    ap.add_argument("--all", action="store_true", help="also time every workload")
+    ap.add_argument("--all", action="store_true", help="with --kernel-only: also time every workload")
+    ap.add_argument("--no-workloads", action="store_true",
+                    help="leave the per-workload rows and the targets summary out of the line")
     ap.add_argument("--all-steps", type=int, default=10)
+    ap.add_argument("--row-macs", type=float, default=1.0e8,
+                    help="multiply-adds in the oracle's sample of each per-workload row")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--ref-macs", type=float, default=5.0e8,
                     help="multiply-adds in the oracle's bounded sample")

@@ -15,6 +15,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libgett_b200.so")
 LIB_MC = os.path.join(HERE, "libgett_b200_mc.so")
+LIB_BENCH = os.path.join(HERE, "libgett_b200_bench.so")  # measurement helpers (*_bench.cu), not the product
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC,-fvisibility=hidden",
@@ -22,7 +23,8 @@ COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC,-fvisibility=hi
 
 
 def sources():
-    return sorted(f for f in os.listdir(CSRC) if f.endswith((".cu", ".cpp")) and not f.endswith("_mc.cu"))
+    return sorted(f for f in os.listdir(CSRC)
+                  if f.endswith((".cu", ".cpp")) and not f.endswith(("_mc.cu", "_bench.cu")))
 
 
 def sources_mc():
@@ -70,6 +72,9 @@ def build(verbose: bool = False, force: bool = False) -> str:
         _link(LIB_MC, [_compile(s, verbose) for s in mc])
     elif os.path.exists(LIB_MC):
         os.remove(LIB_MC)
+    bench = sorted(f for f in os.listdir(CSRC) if f.endswith("_bench.cu"))
+    if bench:
+        _link(LIB_BENCH, [_compile(s, verbose) for s in bench])
     return LIB
 
 

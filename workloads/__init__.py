@@ -189,6 +189,13 @@ class Contraction:
         m, n, k = self.mnk()
         return 2 * m * n * k
 
+    def is_plain_gemm(self) -> bool:
+        """Packed A[m,k], B[k,n], C[m,n]: already the equal-sized GEMM of its own comparison."""
+        a, b, c = self.A, self.B, self.C
+        return (len(a.labels) == 2 and len(b.labels) == 2 and len(c.labels) == 2
+                and c.labels == [a.labels[0], b.labels[1]] and a.labels[1] == b.labels[0]
+                and all(t.strides == packed_strides(t.extents) for t in (a, b, c)))
+
     def compulsory_bytes(self, dtype: int, beta: float) -> int:
         """|A| + |B| + |C| * (1 + [beta != 0]) with fp32 C."""
         ab = 4 if dtype == F32 else 2
