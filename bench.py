@@ -362,6 +362,8 @@ def run_ours(args):
         opts["path"] = args.path
     if args.split_k:
         opts["split_k"] = args.split_k
+    if world > 1:  # the CTA-pair variant is for single-GPU processes only
+        opts["flags"] = g.GETT_OPT_NO_PAIR
     plan = g.Plan(con, dtype, **opts)
     info = plan.info.as_dict()
     stream = torch.cuda.current_stream()

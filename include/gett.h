@@ -96,6 +96,16 @@ typedef enum {
                             switches that split off.                                        */
 } gett_epilogue_t;
 
+/* Bits of gett_plan_opts_t.flags: each switches one automatic choice of the planner off.
+ * Results are the same with or without them; they exist so that every loader / launch
+ * variant can be run on the same problem (tests, comparisons). */
+typedef enum {
+    GETT_OPT_NO_TMA = 1,      /* gather with 16-byte copies even where tensor-map (TMA) boxes apply  */
+    GETT_OPT_NO_PAIR = 2,     /* never launch the CTA-pair variant of the tensor-core kernel         */
+    GETT_OPT_NO_EXCHANGE = 4, /* never exchange the roles of A and B                                 */
+    GETT_OPT_NO_ATOMS = 8     /* no re-ordering of I_m, I_n, I_k into 64 x 64 atoms that are boxes   */
+} gett_opt_flags_t;
+
 /* Planner overrides; zero-initialise for "auto".  Unsupported combinations make
  * gett_plan_create return GETT_ERR_UNSUPPORTED rather than being silently changed. */
 typedef struct {
@@ -106,7 +116,13 @@ typedef struct {
     int32_t stages;   /* 0 = auto                                        */
     int32_t split_k;  /* 0 = auto, 1 = never, s > 1 = exactly s slices   */
     int32_t epilogue; /* gett_epilogue_t                                 */
-    int32_t reserved[9];
+    int32_t flags;    /* gett_opt_flags_t bits                           */
+    int32_t wait_limit_us; /* 0 = default (2 s): how long a device-side wait on a barrier may last
+                              before the kernel gives up and records GETT_ERR_TIMEOUT.  Honoured by
+                              the tensor-core kernel when both operands are gathered (its TMA
+                              loaders keep the default); meant for tests of the give-up path.   */
+    int32_t experiment; /* ignored, except by builds made with -DGETT_EXPERIMENT (timing probes) */
+    int32_t reserved[6];
 } gett_plan_opts_t;
 
 /* What the planner decided (Sec. 3.2.1: index sets, fused sizes, blocking). */
@@ -170,6 +186,11 @@ GETT_API gett_status_t gett_plan_create(gett_plan_t** out, const gett_tensor_des
  *             vectorised kernels, otherwise the scalar path is used.
  *   alpha, beta : host scalars.  beta == 0 means C is not read (NaN/Inf in the
  *             old C do not propagate).  alpha == 0 takes no shortcut.
+ * The device current at the call must be the one the plan was created on
+ * (info.device), otherwise GETT_ERR_INVALID_ARG.  (Where the optional CTA-pair variant
+ * of the tensor-core kernel is installed, it is used only when A and B are ordinary
+ * device memory of that same GPU: its copies are delivered to two CTAs at once and its
+ * tensor maps must cover this GPU's memory alone; only single-GPU processes use it.)
  * Asynchronous; allocates nothing; returns launch-time errors only.  C must not
  * alias A or B.  A plan may be reused; calls that use the same plan concurrently
  * on different streams race on its workspace when info.split_k > 1.

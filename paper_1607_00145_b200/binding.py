@@ -13,6 +13,7 @@ GETT_PATH_AUTO, GETT_PATH_SIMT, GETT_PATH_FFMA, GETT_PATH_UMMA = 0, 1, 2, 3
 GETT_LOAD_SCALAR, GETT_LOAD_VEC_FREE, GETT_LOAD_VEC_K = 0, 1, 2
 GETT_LOAD_TMA_FREE, GETT_LOAD_TMA_K = 3, 4
 GETT_EPI_AUTO, GETT_EPI_DIRECT, GETT_EPI_STAGED = 0, 1, 2
+GETT_OPT_NO_TMA, GETT_OPT_NO_PAIR, GETT_OPT_NO_EXCHANGE, GETT_OPT_NO_ATOMS = 1, 2, 4, 8
 TABLE_NAMES = ("A_M", "A_K", "B_N", "B_K", "C_M", "C_N")
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -33,7 +34,9 @@ class _Desc(ctypes.Structure):
 class PlanOpts(ctypes.Structure):
     _fields_ = [("path", ctypes.c_int32), ("tile_m", ctypes.c_int32), ("tile_n", ctypes.c_int32),
                 ("tile_k", ctypes.c_int32), ("stages", ctypes.c_int32), ("split_k", ctypes.c_int32),
-                ("epilogue", ctypes.c_int32), ("reserved", ctypes.c_int32 * 9)]
+                ("epilogue", ctypes.c_int32), ("flags", ctypes.c_int32),
+                ("wait_limit_us", ctypes.c_int32), ("experiment", ctypes.c_int32),
+                ("reserved", ctypes.c_int32 * 6)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -225,10 +228,9 @@ class Plan:
         if opts:
             o = PlanOpts()
             for k, v in opts.items():
-                if k == "reserved0":  # experiment switches (0 in normal use)
-                    o.reserved[0] = int(v)
-                else:
-                    setattr(o, k, int(v))
+                if k not in dict(PlanOpts._fields_) or k == "reserved":
+                    raise TypeError(f"unknown plan option {k!r}")
+                setattr(o, k, int(v))
         self.handle = gett_plan_create(con.A, con.B, con.C, dtype, o)
         self.info = gett_plan_get_info(self.handle)
 

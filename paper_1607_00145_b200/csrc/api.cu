@@ -12,6 +12,8 @@
 
 #include "kernels.h"
 
+extern "C" GETT_API int gett_internal_pointer_is_local(int memory_type, int pointer_device, int plan_device);
+
 namespace {
 
 int current_device_sm_count(int* device_out)
@@ -55,14 +57,16 @@ EncodeTiledFn encode_tiled_fn()
 }
 
 // Tensor map of one operand for this call's base pointer.  False = use the gather loader.
-bool encode_map(const GettTmaRecipe& R, int dtype, const void* base, uint64_t* out_map)
+bool encode_side(const GettTmaRecipe& R, int dtype, const void* base, GettTmaSide& out)
 {
+    memset(&out, 0, sizeof out);
     EncodeTiledFn fn = encode_tiled_fn();
     if (!R.enabled || !fn)
         return false;
+    const int rank = R.co.rank;
     cuuint64_t dims[5], strides_bytes[4];
     cuuint32_t box[5], estr[5];
-    for (int i = 0; i < R.rank; ++i) {
+    for (int i = 0; i < rank; ++i) {
         dims[i] = R.dims[i];
         box[i] = R.box[i];
         estr[i] = 1;
@@ -71,16 +75,21 @@ bool encode_map(const GettTmaRecipe& R, int dtype, const void* base, uint64_t* o
     }
     const CUtensorMapDataType dt = dtype == GETT_BF16_F32 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
                                                           : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
-    CUresult rc = fn(reinterpret_cast<CUtensorMap*>(out_map), dt, (cuuint32_t)R.rank, const_cast<void*>(base),
+    CUresult rc = fn(reinterpret_cast<CUtensorMap*>(out.map), dt, (cuuint32_t)rank, const_cast<void*>(base),
                      dims, strides_bytes, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return rc == CUDA_SUCCESS;
+    if (rc != CUDA_SUCCESS)
+        return false;
+    out.co = R.co;
+    out.hybrid = R.hybrid;
+    out.use = 1;
+    return true;
 }
 
 // The CTA-pair variant of the tensor-core kernel lives in a library of its own next to this
 // one (it is left out of multi-GPU runs); null if it is not there.
-typedef int (*LaunchPairFn)(const GettKernelArgs*, const GettTmaMaps*, int, int, void*);
+typedef int (*LaunchPairFn)(const GettKernelArgs*, const GettTmaMaps*, int, int, void*, size_t, size_t);
 
 LaunchPairFn launch_pair_fn()
 {
@@ -99,6 +108,18 @@ LaunchPairFn launch_pair_fn()
     return fn;
 }
 
+// The CTA-pair variant delivers copies to both CTAs of a cluster; its tensor maps must cover
+// this GPU's own memory alone.  True if `p` is ordinary device memory of device `device`.
+bool on_this_device(const void* p, int device)
+{
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return gett_internal_pointer_is_local((int)attr.type, attr.device, device) != 0;
+}
+
 int vec_kind(int loader) // the staging layout behind a loader value
 {
     return loader == GETT_LOAD_TMA_FREE ? GETT_LOAD_VEC_FREE : loader == GETT_LOAD_TMA_K ? GETT_LOAD_VEC_K : loader;
@@ -107,6 +128,13 @@ int vec_kind(int loader) // the staging layout behind a loader value
 } // namespace
 
 extern "C" {
+
+// (internal, exported for the host tests) the rule behind on_this_device(): memory type 2 is
+// cudaMemoryTypeDevice; host, managed and unregistered memory, and another GPU's memory, are not local.
+GETT_API int gett_internal_pointer_is_local(int memory_type, int pointer_device, int plan_device)
+{
+    return memory_type == (int)cudaMemoryTypeDevice && pointer_device == plan_device && plan_device >= 0;
+}
 
 gett_status_t gett_plan_create(gett_plan_t** out, const gett_tensor_desc_t* A,
                                const gett_tensor_desc_t* B, const gett_tensor_desc_t* C,
@@ -167,6 +195,16 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
         std::swap(A, B);
     if (plan->info.device < 0)
         return GETT_ERR_CUDA;
+    {
+        // the plan's workspace, status word and SM count belong to the device it was created on
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) {
+            cudaGetLastError();
+            return GETT_ERR_CUDA;
+        }
+        if (dev != plan->info.device)
+            return GETT_ERR_INVALID_ARG;
+    }
     const uintptr_t es = plan->dtype == GETT_F32 ? 4 : 2;
     if (((uintptr_t)A % es) || ((uintptr_t)B % es) || ((uintptr_t)C % 4))
         return GETT_ERR_ALIGNMENT;
@@ -198,9 +236,17 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     args.stages = plan->info.stages;
     args.epilogue = plan->info.epilogue;
     args.debug = plan->debug;
+    // a shortened wait limit applies only where a CTA that gives up has nothing in flight that
+    // it cannot wait for: plans whose operands are both gathered (cp.async is drained on exit)
+    const bool any_tma = plan->tma_a.enabled || plan->tma_b.enabled;
+    args.wait_limit_us = (plan->wait_limit_us > 0 && !any_tma) ? (uint32_t)plan->wait_limit_us : 2000000u;
     args.c_vec = plan->c_vec;
     args.prod_groups = plan->info.path == GETT_PATH_UMMA ? gett_umma_prod_groups(plan->info.stages) : 0;
     args.epi_lean = plan->epi_lean;
+#ifdef GETT_EXPERIMENT
+    if (plan->debug & 2048) // probe: all producer warps as one wide group
+        args.prod_groups = 1;
+#endif
 
     int path = plan->info.path;
     // the vectorised kernels need 16-byte aligned operand bases; otherwise gather scalars
@@ -224,40 +270,22 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
         break;
     case GETT_PATH_UMMA: {
         alignas(64) GettTmaMaps maps;
-        memset(&maps, 0, sizeof maps);
-        if (plan->pair_ok && launch_pair_fn()) {
+        if (plan->pair_ok && launch_pair_fn() && on_this_device(A, plan->info.device) &&
+            on_this_device(B, plan->info.device)) {
             // each CTA of a pair fetches half of the A tile: a K-major A gets a half-height box
             GettTmaRecipe ra = plan->tma_a;
-            if (args.loader_a == GETT_LOAD_VEC_K)
-                for (int i = 1; i < ra.rank; ++i)
-                    if (!ra.which[i] && ra.digit[i] == 0)
-                        ra.box[i] /= 2;
-            maps.use_a = encode_map(ra, plan->dtype, A, maps.map_a) ? 1 : 0;
-            maps.use_b = encode_map(plan->tma_b, plan->dtype, B, maps.map_b) ? 1 : 0;
-            maps.rank_a = ra.rank;
-            maps.rank_b = plan->tma_b.rank;
-            for (int i = 0; i < 5; ++i) {
-                maps.which_a[i] = ra.which[i];
-                maps.digit_a[i] = ra.digit[i];
-                maps.which_b[i] = plan->tma_b.which[i];
-                maps.digit_b[i] = plan->tma_b.digit[i];
-            }
-            if (maps.use_a && maps.use_b &&
-                launch_pair_fn()(&args, &maps, plan->info.smem_bytes, plan->sm_count, cuda_stream) == 0)
+            if (args.loader_a == GETT_LOAD_VEC_K && ra.co.fdim[0] >= 0)
+                ra.box[ra.co.fdim[0]] /= 2;
+            const bool ua = encode_side(ra, plan->dtype, A, maps.a);
+            const bool ub = encode_side(plan->tma_b, plan->dtype, B, maps.b);
+            if (ua && ub &&
+                launch_pair_fn()(&args, &maps, plan->info.smem_bytes, plan->sm_count, cuda_stream,
+                                 sizeof(GettKernelArgs), sizeof(GettTmaMaps)) == 0)
                 break;
             cudaGetLastError(); // the variant could not run: the ordinary kernel does
-            memset(&maps, 0, sizeof maps);
         }
-        maps.use_a = encode_map(plan->tma_a, plan->dtype, A, maps.map_a) ? 1 : 0;
-        maps.use_b = encode_map(plan->tma_b, plan->dtype, B, maps.map_b) ? 1 : 0;
-        maps.rank_a = plan->tma_a.rank;
-        maps.rank_b = plan->tma_b.rank;
-        for (int i = 0; i < 5; ++i) {
-            maps.which_a[i] = plan->tma_a.which[i];
-            maps.digit_a[i] = plan->tma_a.digit[i];
-            maps.which_b[i] = plan->tma_b.which[i];
-            maps.digit_b[i] = plan->tma_b.digit[i];
-        }
+        encode_side(plan->tma_a, plan->dtype, A, maps.a);
+        encode_side(plan->tma_b, plan->dtype, B, maps.b);
         err = gett_launch_umma(args, maps, plan->info.grid, plan->info.smem_bytes, stream);
         break;
     }

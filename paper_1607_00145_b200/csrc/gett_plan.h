@@ -15,14 +15,26 @@ struct GettMode {
     int64_t sA, sB, sC; // element strides; 0 where the tensor does not carry the mode
 };
 
-// One digit of a tile-order fused index: indices (i / mult) % ext of mode `mode`
-// (an index into the canonical list of that set).  mult > 1 or ext < mode extent
-// means the mode was split by factors of its extent (Sec. 3.2.1, Examples 1-2).
+// One digit of a tile-order fused index: value v of the digit stands for index
+// off + v * mult of mode `mode` (an index into the canonical list of that set).
+// mult > 1 or ext < mode extent means the mode was split by factors of its extent
+// (Sec. 3.2.1, Examples 1-2); off > 0 (or a range shorter than the extent) means the
+// digit covers a sub-range of the mode, which happens only in two-segment dimensions.
 struct GettDigit {
     int32_t mode;
     int64_t ext;
     int64_t mult;
+    int64_t off;
 };
+
+// Timing probes ("skip the stores", "skip the math", ...) that give wrong results on purpose
+// exist only in builds made with -DGETT_EXPERIMENT; in the library as shipped GETT_DBG()
+// is the constant 0 and the code behind it is compiled out.
+#ifdef GETT_EXPERIMENT
+#define GETT_DBG(g, bits) (((g).debug & (bits)) != 0)
+#else
+#define GETT_DBG(g, bits) false
+#endif
 
 // Arguments common to every contraction kernel (passed by value).
 struct GettKernelArgs {
@@ -47,37 +59,54 @@ struct GettKernelArgs {
     int32_t c_vec;        // four consecutive tile rows (1) or columns (2) are one aligned 16-byte
                           // vector of C; column-to-slot pattern of the staged epilogues: 1 or 8
                           // (tensor-core kernel), 4 (fp32 kernel: column = a + 4 p, p along C)
-    int32_t debug;        // opts.reserved[0]: experiment switches, 0 in normal use
+    int32_t debug;        // opts.experiment: timing probes, read only by GETT_EXPERIMENT builds
+    uint32_t wait_limit_us; // bound of every device-side wait on a barrier
     int32_t prod_groups;  // producer groups the tensor-core kernel uses (divides stages)
     int32_t epi_lean;     // staged epilogue of the tensor-core kernel with one narrow staging buffer per warp
 };
 
-// Recipe for one operand's TMA tensor map: dimension i of the map follows digit
-// digit[i] of the operand's free dimension (which[i] == 0) or of K (which[i] == 1).
-// Dimension 0 is the operand's stride-1 digit.  A tile is one box (K-major staging)
-// or rows/64 boxes of 64 free indices (MN-major staging).
+// How the coordinates of a TMA box follow from fused indices: digit d of the operand's free
+// dimension adds (digit value) * fmul[d] to coordinate fdim[d], digit d of K adds
+// (digit value) * kmul[d] to coordinate kdim[d] (a negative dimension: none).
+struct GettTmaCoords {
+    int32_t rank;
+    int8_t fdim[GETT_MAX_DIGITS], kdim[GETT_MAX_DIGITS];
+    int32_t fmul[GETT_MAX_DIGITS], kmul[GETT_MAX_DIGITS];
+};
+
+// Recipe for one operand's TMA tensor map (the map itself is encoded per call, since it
+// embeds the operand's base address).  Dimension 0 is the operand's stride-1 mode.
+// K-major staging: the whole tile (rows x 64 k) is one box.  MN-major staging: the tile is
+// fetched in "atoms" of 64 free indices x 64 k, one box each; when the free dimension has
+// two segments (gett_dims.h), only the atoms of segment 0 are boxes and those of segment 1
+// are gathered (`hybrid`).
 struct GettTmaRecipe {
     int32_t enabled;
-    int32_t rank;
+    int32_t hybrid;
     uint64_t dims[5];
     uint64_t strides[5]; // elements; strides[0] == 1
     uint32_t box[5];
-    int8_t which[5], digit[5];
+    GettTmaCoords co;
 };
 
 // What the tensor-core kernel receives besides GettKernelArgs when an operand is
 // loaded through TMA.  `map` is an opaque CUtensorMap (128 bytes, 64-byte aligned).
+struct alignas(64) GettTmaSide {
+    uint64_t map[16];
+    int32_t use;    // 0: the operand is gathered
+    int32_t hybrid; // 1: atoms of segment 1 of the free dimension are gathered, the others come by TMA
+    GettTmaCoords co;
+};
 struct alignas(64) GettTmaMaps {
-    uint64_t map_a[16];
-    uint64_t map_b[16];
-    int32_t use_a, use_b, rank_a, rank_b;
-    int8_t which_a[5], digit_a[5], which_b[5], digit_b[5];
+    GettTmaSide a, b;
 };
 
 struct gett_plan {
     int32_t dtype;
     std::vector<GettMode> im, in, ik; // canonical order (what get_info reports)
     std::vector<GettDigit> tm, tn, tk; // tile order, before merging
+    int32_t tm_seg1, tn_seg1;          // position in tm / tn where segment 1 starts, -1: a plain order
+    int32_t tm_hi, tn_hi;              // ... and where the high part starts (see gett_dims.h)
     GettDim M, N, K;                   // tile order, merged: what the kernels get
     gett_plan_info_t info;
     // geometry
@@ -94,7 +123,9 @@ struct gett_plan {
     float* ws;
     int32_t* status;
     int32_t sm_count;
-    int32_t debug;
+    int32_t debug;     // opts.experiment
+    int32_t flags;     // opts.flags
+    int32_t wait_limit_us;
 };
 
 // Host planner (planner.cpp): everything except device allocation.

@@ -247,7 +247,7 @@ __global__ void __launch_bounds__(2 * TM, 256 / TM) gett_ffma_kernel(const __gri
         const char* As = reinterpret_cast<const char*>(smem) + (slab % stages) * STAGE;
         const char* Bs = As + TM * TK * 4;
 #pragma unroll
-        for (int k4 = 0; k4 < TK / 4 && !(g.debug & 64); ++k4) { // (debug & 64: experiment, no math)
+        for (int k4 = 0; k4 < TK / 4 && !GETT_DBG(g, 64); ++k4) { // (debug & 64: experiment, no math)
             float a[8][4], b[FN][4];
             if (A_K) {
                 frag_kmajor<8>(As, rows, swA, k4, a);
@@ -324,7 +324,7 @@ __global__ void __launch_bounds__(2 * TM, 256 / TM) gett_ffma_kernel(const __gri
     // ---- unpack: C <- alpha * acc + beta * C (or the raw slice sums under split-K) ----
     const float alpha = g.alpha, beta = g.beta;
     const bool vec_m = g.c_vec == 1;
-    if (g.debug & 2) // experiment: no stores
+    if (GETT_DBG(g, 2)) // experiment: no stores
         return;
     if (FN == 8 && (g.c_vec == 2 || g.c_vec == 4) && g.split_k == 1) {
         // C's stride-1 mode runs along the tile's columns.  The scaled accumulators pass

@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
             for (int j = 0; j < CPT / 2; ++j)
                 acc[i][j] = make_float2(0.f, 0.f);
 #pragma unroll(KCT ? KCT : 2)
-        for (uint32_t kc = 0; kc < KC && !(g.debug & 64); ++kc) { // (debug & 64: experiment, no math)
+        for (uint32_t kc = 0; kc < KC && !GETT_DBG(g, 64); ++kc) { // (debug & 64: experiment, no math)
             float4 a[RPT];
 #pragma unroll
             for (int i = 0; i < RPT; ++i) {
@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
         const int64_t* offCM = T->offCM[it % TSLOTS];
         if constexpr (VR) {
             const int64_t cm = offCM[4 * q];
-            if (cm < 0 || (g.debug & 2)) // (debug & 2: experiment, no stores)
+            if (cm < 0 || GETT_DBG(g, 2)) // (debug & 2: experiment, no stores)
                 continue;
 #pragma unroll
             for (int j = 0; j < CPT; ++j) {
@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_kernel(const __grid_co
 #pragma unroll
             for (int i = 0; i < RPT; ++i) {
                 const int64_t cm = offCM[q + QL * i];
-                if (cm < 0 || (g.debug & 2)) // (debug & 2: experiment, no stores)
+                if (cm < 0 || GETT_DBG(g, 2)) // (debug & 2: experiment, no stores)
                     continue;
                 float* crow = g.C + cm;
                 float old[CPT];
@@ -334,7 +334,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_mn_kernel(const __grid
             for (int j = 0; j < CPT / 2; ++j)
                 acc[i][j] = make_float2(0.f, 0.f);
 #pragma unroll(KT ? KT : 4)
-        for (uint32_t k = 0; k < K && !(g.debug & 64); ++k) { // (debug & 64: experiment, no math)
+        for (uint32_t k = 0; k < K && !GETT_DBG(g, 64); ++k) { // (debug & 64: experiment, no math)
             const float4 a = *reinterpret_cast<const float4*>(As + k * ROWS);
             float2 b[CPT / 2];
             const float* brow = Bs + k * NP + cg * CPT;
@@ -357,7 +357,7 @@ __global__ void __launch_bounds__(NT, 2) gett_ffma_skinny_mn_kernel(const __grid
                     acc[i][j] = __ffma2_rn(a2, b[j], acc[i][j]);
             }
         }
-        if (g.debug & 2) // (experiment: no stores)
+        if (GETT_DBG(g, 2)) // (experiment: no stores)
             continue;
         const int64_t* offCM = T->offCM[it % TSLOTS] + 4 * q;
         if (vec_rows) {

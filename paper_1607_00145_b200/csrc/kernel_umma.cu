@@ -79,6 +79,7 @@ __host__ __device__ constexpr int epi_warp_bytes(int tile_n, int cv, int lean)
 }
 
 constexpr uint32_t INVALID16 = 0xFFFFFFFFu; // "outside the tensor" in the 16-byte-unit offset tables
+constexpr uint32_t SKIP16 = 0xFFFFFFFEu;    // "not mine": the piece belongs to an atom that arrives by TMA
 
 // Offsets in the producer tables are in units of 16 bytes (every vector a producer
 // copies starts on a 16-byte boundary), which keeps them in 32 bits.
@@ -86,7 +87,10 @@ struct alignas(16) SmemTables { // the staging rows that follow it hold 128-bit 
     int64_t colC[2][256];                     // per epilogue set: C offset of each tile column
     uint32_t kTab[PROD_GROUPS][2][TILE_K];    // per producer group: A / B offsets of the slab's k
     uint32_t rowTab[PROD_GROUPS][256 + 256];  // per producer group: row offsets (K-major operands)
+    int32_t atomc[PROD_GROUPS][2][4][8];      // per producer group and operand: TMA coordinates (5) and
+                                              // segment of each 64-wide atom of the current tile
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
+    uint64_t drain; // after a give-up: the tensor core has finished what had been issued
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -155,6 +159,52 @@ struct OperandLoader {
 
     uint32_t row16;    // VEC_FREE: this thread's row offset (16-byte units), INVALID16 if outside
     uint32_t dst_lane; // byte offset of this thread's piece 0 inside the operand's stage buffer
+
+    // Hybrid tiles (VEC_FREE only): the 64-wide atoms that lie in segment 0 of the dimension
+    // arrive by TMA; only the atoms of segment 1 are gathered, eight 16-byte pieces per k row.
+    // Thread gl owns piece gl % 8 of the k rows gl / 8 + (LANES / 8) p of every such atom.
+    static constexpr int HY_ATOMS = R / 64 > 0 ? R / 64 : 1;
+    static constexpr int HY_KROWS = LANES / 8;
+    uint32_t hy_row16[HY_ATOMS]; // offset of my piece of atom b, SKIP16 if the atom is not gathered
+
+    __device__ __forceinline__ void setup_hybrid(const GettDim& D, uint32_t origin, uint32_t gl)
+    {
+#pragma unroll
+        for (int b = 0; b < HY_ATOMS; ++b) {
+            const uint32_t f = origin + 64u * b + 8u * (gl & 7);
+            hy_row16[b] = SKIP16;
+            if (f < D.size) {
+                int64_t x, y;
+                if (gett_decompose(D, f, x, y) == 1)
+                    hy_row16[b] = (uint32_t)(x >> 3);
+            }
+        }
+    }
+
+    // The slab is a box of I_k (that is how plans with such tiles order I_k): k row number k of the
+    // slab lies k % 2^kshift steps of K's first digit and k >> kshift steps of its second digit
+    // from the slab's first row, so its offset needs no table.  k16_0: offset of the slab's first
+    // row, s0_16 / s1_16: the two digit strides (all in 16-byte units); nvalid: rows inside K.
+    __device__ __forceinline__ void load_hybrid(const char* __restrict__ base, uint32_t stage_dst, uint32_t gl,
+                                                uint32_t k16_0, uint32_t s0_16, uint32_t s1_16, uint32_t kshift,
+                                                uint32_t nvalid) const
+    {
+        const uint32_t pc = gl & 7, krow = gl >> 3;
+#pragma unroll
+        for (int b = 0; b < HY_ATOMS; ++b) {
+            if (hy_row16[b] == SKIP16)
+                continue;
+            const char* src = base + ((uint64_t)(hy_row16[b] + k16_0) << 4);
+#pragma unroll
+            for (int p = 0; p < TILE_K / HY_KROWS; ++p) {
+                const uint32_t k = krow + HY_KROWS * p;
+                const uint32_t off16 = (k & ((1u << kshift) - 1u)) * s0_16 + (k >> kshift) * s1_16;
+                const bool ok = k < nvalid;
+                ptx::cp_async_16(stage_dst + b * MN_BLOCK_BYTES + k * 128 + ((pc ^ (k & 7)) << 4),
+                                 ok ? src + ((uint64_t)off16 << 4) : base, ok ? 16u : 0u);
+            }
+        }
+    }
 
     // rowTab: the group's table for this operand (used by VEC_K only; the caller
     // synchronises the group before and after).
@@ -276,13 +326,14 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
                                                 uint32_t total_work, volatile int* abort_flag)
 {
     using Sh = StagedShape<TILE_N, CV, LEAN>;
+    const uint64_t wait_ns = (uint64_t)g.wait_limit_us * 1000ull;
     constexpr uint32_t NCH = Sh::NCH, PITCH = Sh::PITCH, GPR = Sh::GPR, NP = Sh::NP, DEPTH = Sh::DEPTH;
     constexpr uint32_t FULL = 0xFFFFFFFFu;
     float* S = reinterpret_cast<float*>(epi_smem + warp * epi_warp_bytes(TILE_N, CV, LEAN));
     int64_t* grp = reinterpret_cast<int64_t*>(S + DEPTH * 32 * PITCH);
     const uint32_t s_u32 = ptx::smem_u32(S);
     const float alpha = g.alpha, beta = g.beta;
-    const bool rmw = beta != 0.f && !(g.debug & 128); // (debug & 128: experiment, old C not read)
+    const bool rmw = beta != 0.f && !GETT_DBG(g, 128); // (debug & 128: experiment, old C not read)
     // this warp's set handles the CTA's tiles with local number es, es + 2, ...; `j` counts them
     const uint32_t es = warp >> 2, eq = warp & 3;
     const uint32_t ncta = total_work > GETT_WB ? (total_work - GETT_WB + GETT_WG - 1) / GETT_WG : 0;
@@ -360,7 +411,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
                 q[k].z = fmaf(beta, o[k].z, q[k].z);
                 q[k].w = fmaf(beta, o[k].w, q[k].w);
             }
-            if (!(g.debug & 512)) // (debug & 512: experiment, no staging writes)
+            if (!GETT_DBG(g, 512)) // (debug & 512: experiment, no staging writes)
                 *reinterpret_cast<float4*>(p[k]) = q[k];
         }
     };
@@ -378,7 +429,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
         __syncwarp(); // ... and everybody else's
         const uint32_t j = ci / NCH, ch = ci - j * NCH, buf = es; // tile es + 2j uses accumulator es
         if (ch == 0) {
-            if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag))
+            if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag, wait_ns))
                 break;
             ptx::tc_fence_after();
         }
@@ -444,7 +495,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
         const int64_t* gch = grp + (j & 1) * EPI_GROUPS + ch * GPR;
         // four groups at a time: staging reads first, then the global stores
 #pragma unroll
-        for (uint32_t t0 = 0; t0 < GPR && !(g.debug & 256); t0 += 4) { // (debug & 256: experiment, no store phase)
+        for (uint32_t t0 = 0; t0 < GPR && !GETT_DBG(g, 256); t0 += 4) { // (debug & 256: experiment, no store phase)
             float4 val[4];
             float* dstp[4];
 #pragma unroll
@@ -452,7 +503,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
                 const uint32_t q = lane + 32 * (t0 + k), row = q / GPR, gi = q - row * GPR;
                 const long long rc = __shfl_sync(FULL, myrow, row);
                 const int64_t cn = gch[gi];
-                dstp[k] = (rc >= 0 && cn >= 0 && !(g.debug & 2)) ? g.C + rc + cn : nullptr; // (debug & 2: no stores)
+                dstp[k] = (rc >= 0 && cn >= 0 && !GETT_DBG(g, 2)) ? g.C + rc + cn : nullptr; // (debug & 2: no stores)
                 val[k] = *reinterpret_cast<const float4*>(Sb + row * PITCH + 4 * gi);
             }
 #pragma unroll
@@ -475,6 +526,7 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
 {
     constexpr uint32_t sbytes = stage_bytes(TILE_M, TILE_N);
     constexpr uint32_t A_STAGE_BYTES = TILE_M * TILE_K * 2;
+    const uint64_t wait_ns = (uint64_t)g.wait_limit_us * 1000ull;
     // ------------------------------ producers ------------------------------
     // Slab number `it` (counted over the CTA's whole work list) belongs to producer
     // group it % PROD_GROUPS, so PROD_GROUPS slabs are gathered concurrently.  The
@@ -488,11 +540,40 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
     OperandLoader<B_VEC_K, TILE_N, LANES> lb;
     const char* baseA = static_cast<const char*>(g.A);
     const char* baseB = static_cast<const char*>(g.B);
-    // An operand whose tile is a box of a <= 5-D tensor map is fetched by TMA: thread 0
-    // of the group issues the copies and the stage's barrier counts their bytes.
-    const bool tmaA = tm.use_a != 0, tmaB = tm.use_b != 0, all_tma = tmaA && tmaB;
-    const uint32_t tma_bytes = (tmaA ? A_STAGE_BYTES : 0) + (tmaB ? TILE_N * TILE_K * 2 : 0);
-    int32_t fa[5] = {0, 0, 0, 0, 0}, fb[5] = {0, 0, 0, 0, 0}; // digit indices of the tile origin
+    // An operand whose tile is a box -- or a list of 64-wide atoms that are boxes -- of a
+    // <= 5-D tensor map is fetched by TMA: thread 0 of the group issues the copies and the
+    // stage's barrier counts their bytes.
+    const bool tmaA = tm.a.use != 0, tmaB = tm.b.use != 0;
+    // hybrid: the atoms of segment 1 of the operand's free dimension are gathered
+    const bool hybridA = tmaA && !A_VEC_K && tm.a.hybrid, hybridB = tmaB && !B_VEC_K && tm.b.hybrid;
+    const bool all_tma = tmaA && tmaB; // no offset tables (and no barriers of the group) are needed
+    constexpr uint32_t ATOM_STAGE_BYTES = 64 * TILE_K * 2; // one atom: 64 free indices x 64 k
+    constexpr int NATOM_A = A_VEC_K ? 1 : TILE_M / 64, NATOM_B = B_VEC_K ? 1 : TILE_N / 64;
+    int32_t (*atomA)[8] = T->atomc[pg][0];
+    int32_t (*atomB)[8] = T->atomc[pg][1];
+    uint32_t tma_bytes = 0; // what the current tile's TMA copies deliver per stage
+    int natomA = 0, natomB = 0;
+    // coordinates of the atoms of a tile (the free-dimension part, kept for all slabs of the
+    // tile) and their segment; returns the bytes per stage of those that come by TMA
+    auto atom_coords = [&](const GettDim& D, const GettTmaCoords& co, uint32_t origin, int natom_max,
+                           int32_t (*out)[8], int& natom) {
+        uint32_t bytes = 0;
+        natom = 0;
+        for (int b = 0; b < natom_max; ++b) {
+            const uint32_t f = origin + 64u * (uint32_t)b;
+            if (b > 0 && f >= D.size)
+                break; // atoms past the end of the dimension are not fetched (their rows are never stored)
+            int32_t c[5] = {0, 0, 0, 0, 0};
+            const int seg = gett_add_coords(D, f, co.fdim, co.fmul, c);
+#pragma unroll
+            for (int i = 0; i < 5; ++i)
+                out[b][i] = c[i];
+            out[b][5] = seg;
+            bytes += seg == 0 ? ATOM_STAGE_BYTES : 0u;
+            ++natom;
+        }
+        return bytes;
+    };
     uint32_t first = 0; // slab number of the current work item's first slab
     bool alive = true;
     for (uint32_t w = GETT_WB; w < total_work && pg < ng; w += GETT_WG) {
@@ -502,14 +583,23 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
         if (j < wi.nslab) {
             if (!all_tma)
                 ptx::named_barrier(gbar, LANES); // the group is done with the previous tables
+            tma_bytes = 0;
             if (!tmaA)
                 la.setup_tile(g.M, wi.m0, gl, rowA);
-            else if (gl == 0)
-                gett_digit_indices(g.M, wi.m0, fa, 5);
+            else if (hybridA)
+                la.setup_hybrid(g.M, wi.m0, gl);
+            if (tmaA && gl == 0) {
+                const uint32_t bytes = atom_coords(g.M, tm.a.co, wi.m0, NATOM_A, atomA, natomA);
+                tma_bytes += A_VEC_K ? A_STAGE_BYTES : bytes;
+            }
             if (!tmaB)
                 lb.setup_tile(g.N, wi.n0, gl, rowB);
-            else if (gl == 0)
-                gett_digit_indices(g.N, wi.n0, fb, 5);
+            else if (hybridB)
+                lb.setup_hybrid(g.N, wi.n0, gl);
+            if (tmaB && gl == 0) {
+                const uint32_t bytes = atom_coords(g.N, tm.b.co, wi.n0, NATOM_B, atomB, natomB);
+                tma_bytes += B_VEC_K ? TILE_N * TILE_K * 2 : bytes;
+            }
         }
         const bool tile_full = wi.m0 + TILE_M <= g.M.size && wi.n0 + TILE_N <= g.N.size;
         for (; j < wi.nslab; j += ng) {
@@ -532,70 +622,70 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
                 ptx::named_barrier(gbar, LANES); // tables (rows and k) complete
             }
             const uint32_t s = it % stages;
+            // the slab's part of the TMA coordinates, before the wait for the stage
+            int32_t ckA[5] = {0, 0, 0, 0, 0}, ckB[5] = {0, 0, 0, 0, 0};
+            if (gl == 0 && alive) {
+                if (tmaA)
+                    gett_add_coords(g.K, k0, tm.a.co.kdim, tm.a.co.kmul, ckA);
+                if (tmaB)
+                    gett_add_coords(g.K, k0, tm.b.co.kdim, tm.b.co.kmul, ckB);
+            }
             // After a timeout a thread keeps walking the loop (so its group's named
             // barriers stay matched) but neither waits nor copies any more.
-            if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->empty[s]), ((it / stages) & 1) ^ 1, abort_flag))
+            if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->empty[s]), ((it / stages) & 1) ^ 1, abort_flag, wait_ns))
                 alive = false;
             if (!alive)
                 continue;
             const uint32_t sa = stage0 + s * sbytes;
             const uint32_t fullbar = ptx::smem_u32(&T->full[s]);
-            if (gl == 0 && tma_bytes && !(g.debug & 4)) {
-                int32_t kd[5] = {0, 0, 0, 0, 0}, c[5];
-                gett_digit_indices(g.K, k0, kd, 5);
+            if (gl == 0 && tma_bytes && !GETT_DBG(g, 4)) {
                 ptx::mbar_expect_tx(fullbar, tma_bytes);
                 if (tmaA) {
-#pragma unroll
-                    for (int i = 0; i < 5; ++i)
-                        c[i] = tm.which_a[i] ? kd[tm.digit_a[i]] : fa[tm.digit_a[i]];
+                    const int32_t(&ck)[5] = ckA;
+                    int32_t c[5];
 #ifdef GETT_UMMA_CLUSTER
                     // my half of the A tile, delivered to both CTAs of the pair (the partner
                     // fetches the other half); each CTA's barrier counts the whole stage
                     const uint32_t half = GETT_WRANK;
                     if (A_VEC_K) { // the map's box is TILE_M / 2 rows high
 #pragma unroll
-                        for (int i = 1; i < 5; ++i)
-                            if (!tm.which_a[i] && tm.digit_a[i] == 0)
-                                c[i] += (int32_t)(half * (TILE_M / 2));
-                        ptx_mc::tma_load_pair(sa + half * (A_STAGE_BYTES / 2), tm.map_a, fullbar, tm.rank_a, c);
+                        for (int i = 0; i < 5; ++i)
+                            c[i] = atomA[0][i] + ck[i];
+                        c[tm.a.co.fdim[0]] += (int32_t)(half * (TILE_M / 2));
+                        ptx_mc::tma_load_pair(sa + half * (A_STAGE_BYTES / 2), tm.a.map, fullbar, tm.a.co.rank, c);
                     } else {
-                        c[0] += (int32_t)(half * (TILE_M / 2));
+                        for (int b = (int)half * (NATOM_A / 2); b < (int)(half + 1) * (NATOM_A / 2) && b < natomA; ++b) {
 #pragma unroll
-                        for (int b = 0; b < TILE_M / 128; ++b) {
-                            ptx_mc::tma_load_pair(sa + (half * (TILE_M / 128) + b) * MN_BLOCK_BYTES, tm.map_a, fullbar,
-                                                  tm.rank_a, c);
-                            c[0] += 64;
+                            for (int i = 0; i < 5; ++i)
+                                c[i] = atomA[b][i] + ck[i];
+                            ptx_mc::tma_load_pair(sa + b * MN_BLOCK_BYTES, tm.a.map, fullbar, tm.a.co.rank, c);
                         }
                     }
 #else
-                    if (A_VEC_K) {
-                        ptx::tma_load(sa, tm.map_a, fullbar, tm.rank_a, c);
-                    } else {
+                    for (int b = 0; b < natomA; ++b) {
+                        if (atomA[b][5])
+                            continue; // an atom of segment 1: gathered below
 #pragma unroll
-                        for (int b = 0; b < TILE_M / 64; ++b) {
-                            ptx::tma_load(sa + b * MN_BLOCK_BYTES, tm.map_a, fullbar, tm.rank_a, c);
-                            c[0] += 64;
-                        }
+                        for (int i = 0; i < 5; ++i)
+                            c[i] = atomA[b][i] + ck[i];
+                        ptx::tma_load(sa + b * MN_BLOCK_BYTES, tm.a.map, fullbar, tm.a.co.rank, c);
                     }
 #endif
                 }
                 if (tmaB) {
+                    const int32_t(&ck)[5] = ckB;
+                    int32_t c[5];
+                    for (int b = 0; b < natomB; ++b) {
+                        if (atomB[b][5])
+                            continue;
 #pragma unroll
-                    for (int i = 0; i < 5; ++i)
-                        c[i] = tm.which_b[i] ? kd[tm.digit_b[i]] : fb[tm.digit_b[i]];
-                    if (B_VEC_K) {
-                        ptx::tma_load(sa + A_STAGE_BYTES, tm.map_b, fullbar, tm.rank_b, c);
-                    } else {
-#pragma unroll
-                        for (int b = 0; b < TILE_N / 64; ++b) {
-                            ptx::tma_load(sa + A_STAGE_BYTES + b * MN_BLOCK_BYTES, tm.map_b, fullbar,
-                                          tm.rank_b, c);
-                            c[0] += 64;
-                        }
+                        for (int i = 0; i < 5; ++i)
+                            c[i] = atomB[b][i] + ck[i];
+                        ptx::tma_load(sa + A_STAGE_BYTES + b * MN_BLOCK_BYTES, tm.b.map, fullbar, tm.b.co.rank, c);
                     }
                 }
             }
-            if (g.debug & 4) {
+            if (GETT_DBG(g, 4)) {
                 // experiment switch: no copies at all (measures the rest of the pipeline)
             } else if (tile_full && k0 + TILE_K <= wi.kend) {
                 if (!tmaA)
@@ -607,6 +697,19 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
                     la.template load_slab<false>(baseA, sa, kA, rowA, gl);
                 if (!tmaB)
                     lb.template load_slab<false>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+            }
+            if ((hybridA || hybridB) && !GETT_DBG(g, 4 | 1024)) { // (probe 1024: the gathered atoms are skipped)
+                int64_t xa, xb;
+                gett_decompose(g.K, k0, xa, xb);
+                // (a slab spans the first digit -- a power of two -- and part of the second, or lies in the first)
+                const uint32_t e0 = (g.K.ndig <= 1 || g.K.ext[0] >= (uint32_t)TILE_K) ? (uint32_t)TILE_K : g.K.ext[0];
+                const uint32_t kbox0 = 31u - (uint32_t)__clz((int)e0), nvalid = wi.kend - k0;
+                if (hybridA)
+                    la.load_hybrid(baseA, sa, gl, (uint32_t)(xa >> 3), (uint32_t)(g.K.sX[0] >> 3),
+                                   (uint32_t)(g.K.sX[1] >> 3), kbox0, nvalid);
+                if (hybridB)
+                    lb.load_hybrid(baseB, sa + A_STAGE_BYTES, gl, (uint32_t)(xb >> 3), (uint32_t)(g.K.sY[0] >> 3),
+                                   (uint32_t)(g.K.sY[1] >> 3), kbox0, nvalid);
             }
             // full[s] hears from this thread when its copies for the slab have landed
             ptx::cp_async_mbar_arrive_noinc(fullbar);
@@ -639,6 +742,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
     const uint32_t total_work = g.tiles_m * g.tiles_n * g.split_k;
 #endif
     volatile int* abort_flag = &T->abort_flag;
+    const uint64_t wait_ns = (uint64_t)g.wait_limit_us * 1000ull; // bound of every wait on a barrier
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < stages; ++s) {
@@ -653,6 +757,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
             ptx::mbar_init(ptx::smem_u32(&T->acc_full[b]), 1);
             ptx::mbar_init(ptx::smem_u32(&T->acc_empty[b]), EPI_SET_THREADS);
         }
+        ptx::mbar_init(ptx::smem_u32(&T->drain), 1);
         T->abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -691,8 +796,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
             // bytes the descriptor start address advances per 16-wide k step
             const uint32_t a_step = A_VEC_K ? 32u : 2u * ATOM_BYTES;
             const uint32_t b_step = B_VEC_K ? 32u : 2u * ATOM_BYTES;
-            const uint32_t lbo = (g.debug & 1) ? ATOM_BYTES : MN_BLOCK_BYTES;
-            const uint32_t sbo = (g.debug & 1) ? MN_BLOCK_BYTES : ATOM_BYTES;
+            const uint32_t lbo = MN_BLOCK_BYTES, sbo = ATOM_BYTES;
             uint32_t it = 0, local = 0;
             bool alive = true;
             for (uint32_t w = GETT_WB; w < total_work && alive; w += GETT_WG, ++local) {
@@ -701,22 +805,21 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                 // uses both (rows 0-127 in buffer 0, rows 128-255 in buffer 1)
                 const uint32_t buf = TWO_HALVES ? 0u : (local & 1);
                 const uint32_t par = TWO_HALVES ? (local & 1) : ((local >> 1) & 1);
-                if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[buf]), par ^ 1, abort_flag))
+                if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[buf]), par ^ 1, abort_flag, wait_ns))
                     break;
-                if (TWO_HALVES && !ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[1]), par ^ 1, abort_flag))
+                if (TWO_HALVES && !ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[1]), par ^ 1, abort_flag, wait_ns))
                     break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * 256;
                 for (uint32_t j = 0; j < wi.nslab; ++j, ++it) {
                     const uint32_t s = it % stages;
-                    if (!ptx::mbar_wait(ptx::smem_u32(&T->full[s]), (it / stages) & 1, abort_flag)) {
+                    if (!ptx::mbar_wait(ptx::smem_u32(&T->full[s]), (it / stages) & 1, abort_flag, wait_ns)) {
                         alive = false;
                         break;
                     }
                     // the copies were generic-proxy writes; the tensor core reads through the
                     // async proxy, so order the two before issuing
-                    if (!(g.debug & 8))
-                        ptx::fence_proxy_async_smem();
+                    ptx::fence_proxy_async_smem();
                     ptx::tc_fence_after();
                     const uint32_t sa = stage0 + s * sbytes, sb = sa + A_STAGE_BYTES;
 #pragma unroll
@@ -744,6 +847,13 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                     if (TWO_HALVES)
                         ptx::umma_commit(ptx::smem_u32(&T->acc_full[1]));
                 }
+            }
+            if (*abort_flag) {
+                // somebody gave up: let the tensor core finish what was issued (it still reads the
+                // stages and writes tensor memory) before the CTA frees both; bounded like every wait
+                int never = 0;
+                ptx::umma_commit(ptx::smem_u32(&T->drain));
+                ptx::mbar_wait(ptx::smem_u32(&T->drain), 0, &never, 2000000000ull);
             }
         }
         __syncwarp();
@@ -790,7 +900,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                 colC[c] = y;
             }
             ptx::named_barrier(1 + es, EPI_SET_THREADS);
-            if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag))
+            if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag, wait_ns))
                 alive = false;
             if (!alive)
                 continue; // keep the named barriers above matched, do nothing else
@@ -802,7 +912,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                 uint32_t v[16];
                 ptx::tmem_ld_32x16(taddr + c0, v);
                 ptx::tmem_wait_ld();
-                if (!row_ok || (g.debug & 2)) // (debug & 2: experiment switch, no stores)
+                if (!row_ok || GETT_DBG(g, 2)) // (debug & 2: experiment switch, no stores)
                     continue;
                 if (g.split_k > 1) {
                     float* dst = g.ws + ((size_t)wi.z * g.N.size + wi.n0 + c0) * g.M.size + wi.m0 + et;

@@ -46,11 +46,16 @@ cudaError_t launch_pair(const GettKernelArgs& args, const GettTmaMaps& maps, int
 } // namespace
 
 // args.tiles_n must be even, args.tile_m == args.tile_n == 256, both maps in use, split_k == 1.
+// args_bytes / maps_bytes: sizeof the two structures as the caller was compiled with; a library
+// built from other headers refuses to run (the ordinary kernel then does).
 extern "C" __attribute__((visibility("default"))) int
-gett_launch_umma_pair(const GettKernelArgs* args, const GettTmaMaps* maps, int smem, int sm_count, void* stream)
+gett_launch_umma_pair(const GettKernelArgs* args, const GettTmaMaps* maps, int smem, int sm_count, void* stream,
+                      size_t args_bytes, size_t maps_bytes)
 {
+    if (args_bytes != sizeof(GettKernelArgs) || maps_bytes != sizeof(GettTmaMaps))
+        return (int)cudaErrorInvalidValue;
     if (!args || !maps || args->tile_m != 256 || args->tile_n != 256 || (args->tiles_n & 1) || args->split_k != 1 ||
-        !maps->use_a || !maps->use_b || args->epilogue != GETT_EPI_DIRECT)
+        !maps->a.use || !maps->b.use || args->epilogue != GETT_EPI_DIRECT)
         return (int)cudaErrorInvalidValue;
     const bool ak = args->loader_a == GETT_LOAD_VEC_K, bk = args->loader_b == GETT_LOAD_VEC_K;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -85,9 +85,14 @@ std::vector<GettDigit> order_with_lead(const std::vector<GettMode>& modes, int l
 }
 
 // Build the kernel-side dimension: one entry per digit, merging a digit into its
-// predecessor when it continues it contiguously in both carrier tensors.
+// predecessor when it continues it contiguously in both carrier tensors (unless `merge`
+// is off).  With seg1 >= 0 the digit list is [segment 0 | segment 1 | high part]: `seg1`
+// and `hi` are the positions in `digits` where segment 1 and the high part start (see
+// gett_dims.h); digits never merge across these positions.  `src`, if given, receives for
+// every kernel-side digit the position in `digits` it came from (meaningful without merging).
 gett_status_t make_dim(const std::vector<GettMode>& modes, const std::vector<GettDigit>& digits,
-                       int carrierX, int carrierY, GettDim& D)
+                       int carrierX, int carrierY, GettDim& D, int seg1 = -1, int hi = -1, bool merge = true,
+                       std::vector<int>* src = nullptr)
 {
     auto stride_of = [](const GettMode& m, int which) {
         return which == 0 ? m.sA : which == 1 ? m.sB : m.sC;
@@ -95,33 +100,73 @@ gett_status_t make_dim(const std::vector<GettMode>& modes, const std::vector<Get
     memset(&D, 0, sizeof D);
     struct E {
         int64_t ext, sx, sy;
+        int from;
     };
+    const int n = (int)digits.size();
+    const bool two = seg1 >= 0;
+    if (two && !(0 < seg1 && seg1 < hi && hi <= n))
+        return GETT_ERR_INVALID_ARG;
     std::vector<E> e;
-    for (const GettDigit& g : digits) {
+    int64_t part_size[3] = {1, 1, 1}; // segment 0, segment 1, high part (plain dimension: all in [0])
+    int part_first_dig[3] = {0, 0, 0};
+    int64_t bx = 0, by = 0;
+    size_t first = 0; // entries of `e` that belong to the part being built
+    for (int i = 0; i < n; ++i) {
+        const int part = !two ? 0 : i < seg1 ? 0 : i < hi ? 1 : 2;
+        if (two && (i == seg1 || i == hi)) {
+            part_first_dig[part] = (int)e.size();
+            first = e.size();
+        }
+        const GettDigit& g = digits[i];
         const GettMode& m = modes[g.mode];
-        E cur{g.ext, stride_of(m, carrierX) * g.mult, stride_of(m, carrierY) * g.mult};
+        E cur{g.ext, stride_of(m, carrierX) * g.mult, stride_of(m, carrierY) * g.mult, i};
+        if (g.off != 0) {
+            if (part != 1)
+                return GETT_ERR_INVALID_ARG; // only segment 1 starts inside a mode
+            bx += stride_of(m, carrierX) * g.off;
+            by += stride_of(m, carrierY) * g.off;
+        }
         if (cur.ext == 1)
             continue;
-        if (!e.empty() && cur.sx == e.back().sx * e.back().ext && cur.sy == e.back().sy * e.back().ext &&
-            e.back().ext * cur.ext < (1ll << 31))
+        part_size[part] *= cur.ext;
+        if (part_size[part] >= (1ll << 31))
+            return GETT_ERR_UNSUPPORTED;
+        if (merge && e.size() > first && cur.sx == e.back().sx * e.back().ext &&
+            cur.sy == e.back().sy * e.back().ext && e.back().ext * cur.ext < (1ll << 31))
             e.back().ext *= cur.ext;
         else
             e.push_back(cur);
     }
-    if ((int)e.size() > GETT_MAX_DIGITS)
+    if (two && hi == n)
+        part_first_dig[2] = (int)e.size();
+    const int64_t total = two ? (part_size[0] + part_size[1]) * part_size[2] : part_size[0];
+    if ((int)e.size() > GETT_MAX_DIGITS || total >= (1ll << 31))
         return GETT_ERR_UNSUPPORTED;
-    int64_t size = 1;
     D.ndig = (int)e.size();
+    if (src)
+        src->clear();
     for (int d = 0; d < D.ndig; ++d) {
         D.ext[d] = (uint32_t)e[d].ext;
         gett_magic(D.ext[d], D.mul[d], D.sh[d]);
         D.sX[d] = e[d].sx;
         D.sY[d] = e[d].sy;
-        size *= e[d].ext;
-        if (size >= (1ll << 31))
-            return GETT_ERR_UNSUPPORTED;
+        if (src)
+            src->push_back(e[d].from);
     }
-    D.size = (uint32_t)size;
+    D.size = (uint32_t)total;
+    D.seg1_dig = D.hi_dig = D.ndig;
+    D.seg1_start = D.period = D.size;
+    if (two) {
+        if (part_first_dig[1] == 0 || part_first_dig[1] >= part_first_dig[2])
+            return GETT_ERR_UNSUPPORTED; // both segments must have digits
+        D.seg1_dig = part_first_dig[1];
+        D.hi_dig = part_first_dig[2];
+        D.seg1_start = (uint32_t)part_size[0];
+        D.period = (uint32_t)(part_size[0] + part_size[1]);
+        gett_magic(D.period, D.period_mul, D.period_sh);
+        D.seg1_bX = bx;
+        D.seg1_bY = by;
+    }
     return GETT_OK;
 }
 
@@ -170,19 +215,23 @@ void make_tma_recipe(const GettDim& F, bool fX, const GettDim& Kd, bool kX, int 
         return;
     if (F.ndig < 1 || Kd.ndig < 1 || F.ndig + Kd.ndig > 5)
         return;
+    if (F.seg1_dig < F.hi_dig || Kd.seg1_dig < Kd.hi_dig)
+        return;
     if (F.ndig > 1 && F.ext[0] % rows != 0)
         return;
     if (Kd.ndig > 1 && Kd.ext[0] % 64 != 0)
         return;
     const int64_t* fs = fX ? F.sX : F.sY;
     const int64_t* ks = kX ? Kd.sX : Kd.sY;
+    for (int d = 0; d < GETT_MAX_DIGITS; ++d)
+        R.co.fdim[d] = R.co.kdim[d] = -1;
     int n = 0;
     auto push = [&](int which, int d) {
         const GettDim& D = which ? Kd : F;
         R.dims[n] = D.ext[d];
         R.strides[n] = (uint64_t)(which ? ks[d] : fs[d]);
-        R.which[n] = (int8_t)which;
-        R.digit[n] = (int8_t)d;
+        (which ? R.co.kdim : R.co.fdim)[d] = (int8_t)n;
+        (which ? R.co.kmul : R.co.fmul)[d] = 1;
         R.box[n] = 1;
         ++n;
     };
@@ -193,7 +242,7 @@ void make_tma_recipe(const GettDim& F, bool fX, const GettDim& Kd, bool kX, int 
         push(0, d);
     for (int d = 1; d < Kd.ndig; ++d)
         push(1, d);
-    R.rank = n;
+    R.co.rank = n;
     R.box[0] = 64;                      // 128 bytes = the swizzle span
     R.box[1] = free_inner ? 64 : rows;  // MN-major: 64 k rows per box; K-major: all rows in one box
     if (R.strides[0] != 1)
@@ -202,6 +251,202 @@ void make_tma_recipe(const GettDim& F, bool fX, const GettDim& Kd, bool kX, int 
         if (R.strides[i] % 8 != 0 || R.strides[i] >= (1ull << 38))
             return;
     R.enabled = 1;
+}
+
+// ---- tiles of 64-wide atoms for operands whose stride-1 mode is a free mode (Sec. 3.2.1) ----
+//
+// Such an operand is staged as rows of 64 consecutive free indices per k.  A TMA box can fill
+// one "atom" (64 free indices x 64 k) when its 64 indices are consecutive indices of the
+// lead (stride-1) mode.  With that mode's extent e = 64 q + r:
+//   r == 0            every atom is such a run;
+//   r in {16, 32}     the first 64 q indices of every run of the lead mode form such atoms
+//                     (segment 0), the remaining r are combined with 64 / r consecutive
+//                     indices of a second free mode (the partner) into atoms of r x 64/r
+//                     (segment 1) -- the paper's sub-tensor made of pieces of two modes, used
+//                     for the remainder only, so that most of the data still moves in 128-byte
+//                     rows.  Those atoms are not boxes with a 128-byte inner extent and are
+//                     gathered with 16-byte copies.
+// The two kinds alternate with period e * 64/r (64/r runs of the lead mode), so every tile
+// holds both in the same proportion.
+struct SideOrder {
+    bool ok = false;
+    std::vector<GettDigit> digits; // [segment 0 | segment 1 | high part] or a plain order
+    int seg1 = -1, hi = -1;
+    int lead = -1;
+};
+
+SideOrder atom_order(const std::vector<GettMode>& modes, const std::vector<GettDigit>& cur, int carrier)
+{
+    SideOrder S;
+    if (cur.empty())
+        return S;
+    for (const GettDigit& g : cur)
+        if (g.mult != 1 || g.off != 0 || g.ext != modes[g.mode].ext)
+            return S; // already split for another purpose
+    auto stride_of = [&](int m) { return carrier == 0 ? modes[m].sA : modes[m].sB; };
+    S.lead = cur[0].mode;
+    const int64_t e = modes[S.lead].ext;
+    if (stride_of(S.lead) != 1 || e % 8 != 0)
+        return S;
+    if (e % 64 == 0) {
+        S.digits = cur;
+        S.ok = true;
+        return S;
+    }
+    const int64_t q = e / 64, r = e % 64;
+    // (r == 8: the remainder would be gathered in isolated 16-byte pieces, one memory request
+    //  each -- measured slower than gathering the whole operand, whose copies follow the runs)
+    if (q == 0 || 64 % r != 0 || r < 16)
+        return S;
+    const int64_t need = 64 / r;
+    int partner = -1;
+    for (size_t i = 1; i < cur.size() && partner < 0; ++i)
+        if (modes[cur[i].mode].ext % need == 0)
+            partner = cur[i].mode;
+    if (partner < 0)
+        return S;
+    S.digits.push_back({S.lead, 64 * q, 1, 0});
+    S.digits.push_back({partner, need, 1, 0});
+    S.seg1 = (int)S.digits.size();
+    S.digits.push_back({S.lead, r, 1, 64 * q});
+    S.digits.push_back({partner, need, 1, 0});
+    S.hi = (int)S.digits.size();
+    S.digits.push_back({partner, modes[partner].ext / need, need, 0});
+    for (size_t i = 1; i < cur.size(); ++i)
+        if (cur[i].mode != partner)
+            S.digits.push_back(cur[i]);
+    S.ok = true;
+    return S;
+}
+
+// Order of I_k in which every slab of 64 contracted indices is a box of the modes: a mode
+// whose extent is a multiple of 64 first, or a p-wide piece (p a power of two) of one mode
+// times 64 / p consecutive indices of a second one (Sec. 3.2.1, the sub-tensor k_C = 64 made
+// of pieces of two modes).  box_u x box_v is the slab's shape on the first two modes of the
+// order (box_v == 0: the slab lies in the first mode alone).
+struct KOrder {
+    bool ok = false;
+    std::vector<GettDigit> digits;
+    int u = -1, v = -1;
+    int64_t box_u = 64, box_v = 0;
+};
+
+KOrder slab_order(const std::vector<GettMode>& modes, const std::vector<GettDigit>& cur)
+{
+    KOrder K;
+    if (cur.empty())
+        return K;
+    for (const GettDigit& g : cur)
+        if (g.mult != 1 || g.off != 0 || g.ext != modes[g.mode].ext)
+            return K;
+    auto rest = [&](int skip1, int skip2) {
+        for (const GettDigit& g : cur)
+            if (g.mode != skip1 && g.mode != skip2)
+                K.digits.push_back(g);
+    };
+    if (cur.size() == 1) {
+        K.digits = cur;
+        K.u = cur[0].mode;
+        K.ok = true;
+        return K;
+    }
+    for (const GettDigit& g : cur)
+        if (g.ext % 64 == 0) {
+            K.u = g.mode;
+            K.digits.push_back(g);
+            rest(g.mode, -1);
+            K.ok = true;
+            return K;
+        }
+    int64_t best_p = 0;
+    for (const GettDigit& gu : cur) {
+        int64_t p = 1;
+        while (p < 32 && gu.ext % (2 * p) == 0)
+            p *= 2;
+        if (p < 2 || p <= best_p)
+            continue;
+        for (const GettDigit& gv : cur)
+            if (gv.mode != gu.mode && gv.ext % (64 / p) == 0) {
+                best_p = p;
+                K.u = gu.mode;
+                K.v = gv.mode;
+                break;
+            }
+    }
+    if (best_p == 0)
+        return K;
+    K.box_u = best_p;
+    K.box_v = 64 / best_p;
+    K.digits.push_back({K.u, best_p, 1, 0});
+    K.digits.push_back({K.v, modes[K.v].ext, 1, 0});
+    K.digits.push_back({K.u, modes[K.u].ext / best_p, best_p, 0});
+    rest(K.u, K.v);
+    K.ok = true;
+    return K;
+}
+
+// Tensor map of an operand fetched atom by atom (the atoms of segment 0; segment 1, if there
+// is one, is gathered).  Map dimensions: the lead mode, the other free modes, then the modes
+// of I_k in slab order.  `fsrc` / `ksrc` give, for each digit of the kernel-side dimensions,
+// its position in S.digits / K.digits.
+bool make_atom_recipe(const std::vector<GettMode>& fmodes, const SideOrder& S, const std::vector<int>& fsrc,
+                      const GettDim& F, const std::vector<GettMode>& kmodes, const KOrder& K,
+                      const std::vector<int>& ksrc, int carrier, GettTmaRecipe& R)
+{
+    memset(&R, 0, sizeof R);
+    for (int d = 0; d < GETT_MAX_DIGITS; ++d)
+        R.co.fdim[d] = R.co.kdim[d] = -1;
+    auto stride_of = [&](const GettMode& m) { return carrier == 0 ? m.sA : m.sB; };
+    std::vector<int> fdim_of(fmodes.size(), -1), kdim_of(kmodes.size(), -1);
+    int n = 0;
+    auto add = [&](const GettMode& m, int& slot) {
+        if (slot >= 0)
+            return true;
+        if (n >= 5)
+            return false;
+        slot = n;
+        R.dims[n] = (uint64_t)m.ext;
+        R.strides[n] = (uint64_t)stride_of(m);
+        R.box[n] = 1;
+        ++n;
+        return true;
+    };
+    if (!add(fmodes[S.lead], fdim_of[S.lead]))
+        return false;
+    for (const GettDigit& g : S.digits)
+        if (!add(fmodes[g.mode], fdim_of[g.mode]))
+            return false;
+    for (const GettDigit& g : K.digits)
+        if (!add(kmodes[g.mode], kdim_of[g.mode]))
+            return false;
+    R.co.rank = n;
+    if (n < 2) // (a tensor map needs a second dimension; such a case keeps the gather)
+        return false;
+    if (R.strides[0] != 1)
+        return false;
+    for (int i = 1; i < n; ++i)
+        if (R.strides[i] % 8 != 0 || R.strides[i] >= (1ull << 38))
+            return false;
+    R.box[fdim_of[S.lead]] = 64;
+    R.box[kdim_of[K.u]] = (uint32_t)K.box_u;
+    if (K.box_v)
+        R.box[kdim_of[K.v]] = (uint32_t)K.box_v;
+    // coordinates: the digits of segment 0 and of the high part (segment 1 is not fetched by TMA)
+    for (size_t d = 0; d < fsrc.size(); ++d) {
+        if ((int)d >= F.seg1_dig && (int)d < F.hi_dig)
+            continue;
+        const GettDigit& g = S.digits[fsrc[d]];
+        R.co.fdim[d] = (int8_t)fdim_of[g.mode];
+        R.co.fmul[d] = (int32_t)g.mult;
+    }
+    for (size_t d = 0; d < ksrc.size(); ++d) {
+        const GettDigit& g = K.digits[ksrc[d]];
+        R.co.kdim[d] = (int8_t)kdim_of[g.mode];
+        R.co.kmul[d] = (int32_t)g.mult;
+    }
+    R.hybrid = S.seg1 >= 0 ? 1 : 0;
+    R.enabled = 1;
+    return true;
 }
 
 // 16-byte vectors of `vec` elements along the first digit of `lead` are legal for
@@ -301,7 +546,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         const bool small_nk = dtype == GETT_F32 && nsz <= 64 && ksz <= gett_ffma_skinny_max_k();
         bool want = !small_nk && unitCm >= 0 && unitAm >= 0 && unitCm != unitAm && im[unitAm].ext % vec == 0 &&
                     im[unitAm].ext > vec && im[unitCm].ext % 4 == 0 && o.epilogue != GETT_EPI_DIRECT &&
-                    !(o.reserved[0] & 8192); // (experiment switch: never exchange)
+                    !(o.flags & GETT_OPT_NO_EXCHANGE);
         if (want && dtype == GETT_F32) { // the same alignment the fp32 split asks for
             for (const GettMode& m : in)
                 want = want && m.sC % 4 == 0;
@@ -409,6 +654,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         }
     }
     p->tk = order_with_lead(ik, leadK);
+    p->tm_seg1 = p->tn_seg1 = p->tm_hi = p->tn_hi = -1;
     if ((rc = make_dim(im, p->tm, 0, 2, p->M)) || (rc = make_dim(in, p->tn, 1, 2, p->N)) ||
         (rc = make_dim(ik, p->tk, 0, 1, p->K)))
         return rc;
@@ -451,7 +697,24 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     if (path < GETT_PATH_AUTO || path > GETT_PATH_UMMA)
         return GETT_ERR_INVALID_ARG;
     const bool both_vec = info.loader_a != GETT_LOAD_SCALAR && info.loader_b != GETT_LOAD_SCALAR;
-    const bool umma_ok = dtype != GETT_F32 && both_vec;
+    // The vectorised kernels keep operand offsets in 32 bits (elements for fp32, 16-byte units
+    // for the 16-bit types, two top values reserved as markers).  An operand whose largest
+    // offset does not fit goes to the scalar-gather kernel, whose offsets are 64-bit.
+    bool offsets_fit = true;
+    {
+        int64_t maxA = 0, maxB = 0;
+        for (const GettMode& m : im)
+            maxA += (m.ext - 1) * m.sA;
+        for (const GettMode& m : in)
+            maxB += (m.ext - 1) * m.sB;
+        for (const GettMode& m : ik) {
+            maxA += (m.ext - 1) * m.sA;
+            maxB += (m.ext - 1) * m.sB;
+        }
+        const int64_t worst = std::max(maxA, maxB);
+        offsets_fit = dtype == GETT_F32 ? worst < (int64_t)0xFFFFFFF0ll : (worst >> 3) < (int64_t)0xFFFFFFF0ll;
+    }
+    const bool umma_ok = dtype != GETT_F32 && both_vec && offsets_fit;
     // fp32 with small N and K and a K-major A: B is read once element by element, so
     // only A has to be gatherable in 16-byte vectors
     const bool skinny_ok = dtype == GETT_F32 &&
@@ -460,7 +723,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
                            p->K.size <= (uint32_t)gett_ffma_skinny_max_k() && o.split_k <= 1 &&
                            (o.tile_m == 0 || o.tile_m == gett_ffma_skinny_rows()) && o.tile_n == 0 &&
                            o.tile_k == 0 && o.stages == 0 && o.epilogue != GETT_EPI_STAGED;
-    const bool ffma_ok = dtype == GETT_F32; // any layout: operands without usable vectors go scalar
+    const bool ffma_ok = dtype == GETT_F32 && offsets_fit; // any layout: operands without usable vectors go scalar
     if (path == GETT_PATH_AUTO)
         path = umma_ok ? GETT_PATH_UMMA : ffma_ok ? GETT_PATH_FFMA : GETT_PATH_SIMT;
     if ((path == GETT_PATH_UMMA && !umma_ok) || (path == GETT_PATH_FFMA && !ffma_ok))
@@ -482,7 +745,11 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     const bool split4 = dtype == GETT_F32 && p->c_vec == 0 && p->N.ndig >= 2 && p->N.ext[0] == 4 &&
                         p->N.sY[1] == 1 && p->N.ext[1] % 4 == 0 && others_mult4(1);
     info.path = path;
-    p->debug = o.reserved[0];
+    p->debug = o.experiment;
+    p->flags = o.flags;
+    if (o.wait_limit_us < 0)
+        return GETT_ERR_INVALID_ARG;
+    p->wait_limit_us = o.wait_limit_us;
     p->skinny = 0;
     p->epi_lean = 0;
     memset(&p->tma_a, 0, sizeof p->tma_a);
@@ -633,9 +900,54 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         info.stages = st;
         info.block = gett_umma_block();
         info.smem_bytes = gett_umma_smem_bytes(tmh, tn, st, staged_cv, lean);
-        if (!(p->debug & 32)) { // (debug & 32: experiment switch, gather even where TMA applies)
+        if (!(p->flags & GETT_OPT_NO_TMA)) {
             make_tma_recipe(p->M, true, p->K, true, info.loader_a, (uint32_t)tmh, p->tma_a);
             make_tma_recipe(p->N, true, p->K, false, info.loader_b, (uint32_t)tn, p->tma_b);
+            // Both operands staged as rows of 64 free indices and not both tiles boxes: order
+            // I_m, I_n and I_k so that the tiles consist of 64 x 64 atoms that are boxes
+            // (Sec. 3.2.1: sub-tensors made of pieces of one or two modes), and fetch those by TMA.
+            if (!(p->tma_a.enabled && p->tma_b.enabled) && info.loader_a == GETT_LOAD_VEC_FREE &&
+                info.loader_b == GETT_LOAD_VEC_FREE && !staged_cv && !ik.empty() && !(p->flags & GETT_OPT_NO_ATOMS)) {
+                const KOrder ko = slab_order(ik, p->tk);
+                const SideOrder sa = atom_order(im, p->tm, 0), sb = atom_order(in, p->tn, 1);
+                GettDim M2, N2, K2;
+                std::vector<int> srcm, srcn, srck;
+                if (ko.ok && (sa.ok || sb.ok) &&
+                    make_dim(im, sa.ok ? sa.digits : p->tm, 0, 2, M2, sa.ok ? sa.seg1 : -1, sa.hi, false, &srcm) == GETT_OK &&
+                    make_dim(in, sb.ok ? sb.digits : p->tn, 1, 2, N2, sb.ok ? sb.seg1 : -1, sb.hi, false, &srcn) == GETT_OK &&
+                    make_dim(ik, ko.digits, 0, 1, K2, -1, -1, false, &srck) == GETT_OK) {
+                    GettTmaRecipe ra, rb;
+                    const bool oka = sa.ok && make_atom_recipe(im, sa, srcm, M2, ik, ko, srck, 0, ra);
+                    const bool okb = sb.ok && make_atom_recipe(in, sb, srcn, N2, ik, ko, srck, 1, rb);
+                    if ((int)oka + (int)okb > p->tma_a.enabled + p->tma_b.enabled) {
+                        if (oka) {
+                            p->tm = sa.digits;
+                            p->tm_seg1 = sa.seg1;
+                            p->tm_hi = sa.hi;
+                            p->tma_a = ra;
+                        } else {
+                            memset(&p->tma_a, 0, sizeof p->tma_a);
+                        }
+                        if (okb) {
+                            p->tn = sb.digits;
+                            p->tn_seg1 = sb.seg1;
+                            p->tn_hi = sb.hi;
+                            p->tma_b = rb;
+                        } else {
+                            memset(&p->tma_b, 0, sizeof p->tma_b);
+                        }
+                        p->tk = ko.digits;
+                        // (a side that keeps the gather keeps its order; its digits are only no longer merged)
+                        if ((rc = make_dim(im, p->tm, 0, 2, p->M, p->tm_seg1, p->tm_hi, false)) ||
+                            (rc = make_dim(in, p->tn, 1, 2, p->N, p->tn_seg1, p->tn_hi, false)))
+                            return rc;
+                        p->K = K2;
+                        info.digits_m = p->M.ndig;
+                        info.digits_n = p->N.ndig;
+                        info.digits_k = p->K.ndig;
+                    }
+                }
+            }
             if (p->tma_a.enabled)
                 info.loader_a = info.loader_a == GETT_LOAD_VEC_FREE ? GETT_LOAD_TMA_FREE : GETT_LOAD_TMA_K;
             if (p->tma_b.enabled)
@@ -681,9 +993,10 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     if (p->skinny) // persistent: two CTAs per SM stream the row tiles
         info.grid = (int32_t)std::min<uint64_t>(p->tiles_m, 2ull * sms);
     // two neighbouring 256 x 256 tiles per CTA pair, A shared between the two CTAs
-    p->pair_ok = path == GETT_PATH_UMMA && p->tma_a.enabled && p->tma_b.enabled && info.tile_m == 256 &&
+    p->pair_ok = path == GETT_PATH_UMMA && p->tma_a.enabled && p->tma_b.enabled && !p->tma_a.hybrid &&
+                 !p->tma_b.hybrid && info.tile_m == 256 &&
                  info.tile_n == 256 && info.epilogue == GETT_EPI_DIRECT && split == 1 && p->tiles_n % 2 == 0 &&
-                 !(p->debug & 16384); // (experiment switch: never)
+                 !(p->flags & GETT_OPT_NO_PAIR);
     info.swapped = p->swapped;
     if (p->swapped) { // report the caller's view
         std::swap(info.M, info.N);
@@ -697,14 +1010,16 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     return GETT_OK;
 }
 
-// Canonical table `which`: fused canonical index -> per-mode indices -> tile-order
-// fused index -> gett_decompose() on the digits the kernels receive.
+// Canonical table `which`: every tile-order fused index t is taken apart into its digits
+// (the digits the kernels receive), which give both the per-mode indices -- hence the
+// canonical fused index the entry belongs to -- and, through gett_decompose(), the offset.
 gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, size_t capacity)
 {
     const std::vector<GettMode>* modes;
     const std::vector<GettDigit>* digits;
     const GettDim* D;
     bool wantX;
+    int seg1 = -1, hi = -1;
     if (p->swapped) { // the caller's A is the kernels' B: rows <-> columns, X <-> Y for K
         switch (which) {
         case GETT_TABLE_A_M: which = GETT_TABLE_B_N; break;
@@ -717,10 +1032,10 @@ gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, si
         }
     }
     switch (which) {
-    case GETT_TABLE_A_M: modes = &p->im; digits = &p->tm; D = &p->M; wantX = true; break;
-    case GETT_TABLE_C_M: modes = &p->im; digits = &p->tm; D = &p->M; wantX = false; break;
-    case GETT_TABLE_B_N: modes = &p->in; digits = &p->tn; D = &p->N; wantX = true; break;
-    case GETT_TABLE_C_N: modes = &p->in; digits = &p->tn; D = &p->N; wantX = false; break;
+    case GETT_TABLE_A_M: modes = &p->im; digits = &p->tm; D = &p->M; wantX = true; seg1 = p->tm_seg1; hi = p->tm_hi; break;
+    case GETT_TABLE_C_M: modes = &p->im; digits = &p->tm; D = &p->M; wantX = false; seg1 = p->tm_seg1; hi = p->tm_hi; break;
+    case GETT_TABLE_B_N: modes = &p->in; digits = &p->tn; D = &p->N; wantX = true; seg1 = p->tn_seg1; hi = p->tn_hi; break;
+    case GETT_TABLE_C_N: modes = &p->in; digits = &p->tn; D = &p->N; wantX = false; seg1 = p->tn_seg1; hi = p->tn_hi; break;
     case GETT_TABLE_A_K: modes = &p->ik; digits = &p->tk; D = &p->K; wantX = true; break;
     case GETT_TABLE_B_K: modes = &p->ik; digits = &p->tk; D = &p->K; wantX = false; break;
     default: return GETT_ERR_INVALID_ARG;
@@ -728,22 +1043,49 @@ gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, si
     if (!dst || capacity < D->size)
         return GETT_ERR_INVALID_ARG;
     const int nm = (int)modes->size();
-    std::vector<int64_t> idx(nm, 0);
-    for (uint32_t c = 0; c < D->size; ++c) {
-        // tile-order fused index of the tuple idx[]
-        uint64_t t = 0, weight = 1;
-        for (const GettDigit& g : *digits) {
-            t += (uint64_t)((idx[g.mode] / g.mult) % g.ext) * weight;
-            weight *= (uint64_t)g.ext;
+    const int nd = (int)digits->size();
+    std::vector<int64_t> idx(nm);
+    std::vector<uint64_t> weight(nm); // of a mode in the canonical fused index, first mode fastest
+    uint64_t w = 1;
+    for (int j = 0; j < nm; ++j) {
+        weight[j] = w;
+        w *= (uint64_t)(*modes)[j].ext;
+    }
+    // sizes of the two segments of the low part (a plain order is one "segment" with no high part)
+    const bool two = seg1 > 0;
+    const int s1 = two ? seg1 : nd, h = two ? hi : nd;
+    uint64_t size0 = 1, size1 = 1;
+    for (int i = 0; i < s1; ++i)
+        size0 *= (uint64_t)(*digits)[i].ext;
+    for (int i = s1; i < h; ++i)
+        size1 *= (uint64_t)(*digits)[i].ext;
+    const uint64_t period = two ? size0 + size1 : size0;
+    auto take = [&](int from, int to, uint64_t rem) {
+        for (int i = from; i < to; ++i) {
+            const GettDigit& g = (*digits)[i];
+            idx[g.mode] += g.off + (int64_t)(rem % (uint64_t)g.ext) * g.mult;
+            rem /= (uint64_t)g.ext;
         }
+    };
+    std::vector<bool> seen(D->size, false);
+    for (uint32_t t = 0; t < D->size; ++t) {
+        std::fill(idx.begin(), idx.end(), 0);
+        const uint64_t lo = two ? t % period : t;
+        if (two && lo >= size0)
+            take(s1, h, lo - size0);
+        else
+            take(0, s1, lo);
+        if (two)
+            take(h, nd, t / period);
+        uint64_t c = 0;
+        for (int j = 0; j < nm; ++j)
+            c += (uint64_t)idx[j] * weight[j];
+        if (c >= D->size || seen[c])
+            return GETT_ERR_INVALID_ARG; // the tile order is not a permutation of the canonical one
+        seen[c] = true;
         int64_t ox, oy;
-        gett_decompose(*D, (uint32_t)t, ox, oy);
+        gett_decompose(*D, t, ox, oy);
         dst[c] = wantX ? ox : oy;
-        for (int j = 0; j < nm; ++j) { // advance the canonical odometer, first mode fastest
-            if (++idx[j] < (*modes)[j].ext)
-                break;
-            idx[j] = 0;
-        }
     }
     return GETT_OK;
 }

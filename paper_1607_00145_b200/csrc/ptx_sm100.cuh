@@ -47,7 +47,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait: gives up after `limit_ns`, or as soon as another thread of the CTA
 // has raised *abort_flag.  Returns false on give-up (and raises the flag itself).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          uint64_t limit_ns = 2000000000ull)
+                                          uint64_t limit_ns)
 {
     if (mbar_try_wait(bar, parity))
         return true;
@@ -55,7 +55,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity))
             return true;
-        if ((spin & 255u) == 0) {
+        if ((spin & 63u) == 0) {
             if (*abort_flag)
                 return false;
             if (globaltimer() - t0 > limit_ns) {

@@ -91,14 +91,14 @@ def test_staged_epilogue_when_columns_already_run_along_c():
 ])
 def test_tma_loader_against_gather_loader_and_oracle(spec, sizes):
     """Tiles that are boxes of a tensor map go through TMA; the same plan with the
-    gather loader (experiment switch 32) must give the same C, and both the oracle's."""
+    gather loader (GETT_OPT_NO_TMA) must give the same C, and both the oracle's."""
     con = parse_spec(spec, sizes)
     for dtype in (BF16_F32, F16_F32):
         ratio, info = parity_case(con, dtype, "normal", 21, 1.0, 0.5, repeat=2)
         assert info.path == g.GETT_PATH_UMMA
         assert info.loader_a in (g.GETT_LOAD_TMA_FREE, g.GETT_LOAD_TMA_K)
         assert info.loader_b in (g.GETT_LOAD_TMA_FREE, g.GETT_LOAD_TMA_K)
-        ratio2, info2 = parity_case(con, dtype, "normal", 21, 1.0, 0.5, reserved0=32)
+        ratio2, info2 = parity_case(con, dtype, "normal", 21, 1.0, 0.5, flags=g.GETT_OPT_NO_TMA)
         assert info2.loader_a in (g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_K)
         parity_case(con, dtype, "normal", 21, 1.0, 0.0, split_k=2)
 
@@ -113,7 +113,7 @@ def test_256_row_tiles(spec, sizes):
     """One tile in both accumulator buffers (tile_m = 256), forced, against the oracle."""
     con = parse_spec(spec, sizes)
     for dtype in (BF16_F32, F16_F32):
-        for extra in ({}, {"reserved0": 32}, {"split_k": 2}):
+        for extra in ({}, {"flags": g.GETT_OPT_NO_TMA}, {"split_k": 2}):
             ratio, info = parity_case(con, dtype, "normal", 33, 1.0, 0.5, repeat=2, tile_m=256,
                                       tile_n=256, **extra)
             assert info.tile_m == 256 and info.path == g.GETT_PATH_UMMA
@@ -136,6 +136,39 @@ def test_fp32_64_row_tiles(spec, sizes):
     parity_case(con, F32, "uniform", 17, 1.0, 0.5, tile_m=64, split_k=2)
 
 
+ATOM_SPEC = "C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]"
+
+
+@pytest.mark.parametrize("spec,sizes", [
+    # 80 = 64 + 16: atoms of 64 (TMA) and atoms of 16 x 4 (gathered) on both sides, slabs of 8 x 8 contracted indices
+    (ATOM_SPEC, dict(m0=80, m1=8, n0=16, n1=80, k0=72, k1=8)),
+    # 96 = 64 + 32 (atoms of 32 x 2) against 16 = 0 * 64 + 16 (no atoms: gathered); slab = 16 x 4
+    (ATOM_SPEC, dict(m0=96, m1=6, n0=12, n1=16, k0=48, k1=12)),
+    # 128-wide and 192-wide lead modes (64-wide atoms only), a contracted mode that is a multiple of 64 goes first
+    (ATOM_SPEC, dict(m0=128, m1=3, n0=3, n1=192, k0=24, k1=64)),
+    # one side keeps the gather (40 = 0 * 64 + 40 does not divide into atoms), the other uses atoms
+    (ATOM_SPEC, dict(m0=40, m1=8, n0=8, n1=96, k0=72, k1=8)),
+    # a single contracted mode that is not a multiple of 64: the last slab is zero-filled (TMA and gathered atoms alike)
+    ("C[m0,n0,m1,n1] = A[m0,k,m1] * B[n1,k,n0]", dict(m0=80, m1=8, n0=8, n1=24, k=200)),
+    # three free modes on one side (five map dimensions), the partner is the second mode of the order
+    ("C[m0,n0,m1,m2] = A[m0,k0,m2,m1,k1] * B[n0,k1,k0]", dict(m0=96, m1=8, m2=3, n0=136, k0=8, k1=24)),
+])
+def test_atom_tma_loader_against_gather_loader_and_oracle(spec, sizes):
+    """Operands whose tiles are not boxes but lists of 64 x 64 atoms that are (the 72-wide family):
+    TMA atom by atom, against the oracle, against the gather loader, with split-K, with 256-row
+    tiles, and with a ragged last tile in both directions."""
+    con = parse_spec(spec, sizes)
+    for dtype in (BF16_F32, F16_F32):
+        ratio, info = parity_case(con, dtype, "normal", 51, 1.0, 0.5, repeat=2)
+        assert info.path == g.GETT_PATH_UMMA
+        assert g.GETT_LOAD_TMA_FREE in (info.loader_a, info.loader_b)
+        ratio2, info2 = parity_case(con, dtype, "normal", 51, 1.0, 0.5, flags=g.GETT_OPT_NO_TMA)
+        assert info2.loader_a == g.GETT_LOAD_VEC_FREE and info2.loader_b == g.GETT_LOAD_VEC_FREE
+    parity_case(con, BF16_F32, "normal", 51, -0.5, 0.0, repeat=2, split_k=2)
+    parity_case(con, BF16_F32, "normal", 51, 1.0, 1.0, repeat=2, tile_m=256, tile_n=256)
+    parity_case(con, BF16_F32, "normal", 51, 1.0, 0.0, tile_n=64)
+
+
 @pytest.mark.parametrize("spec,sizes", [
     ("C[m,n] = A[m,k] * B[k,n]", dict(m=648, n=1000, k=200)),    # A in boxes of 64 rows, ragged M, N and K
     ("C[m,n] = A[k,m] * B[n,k]", dict(m=520, n=520, k=136)),     # K-major A: half-height boxes
@@ -151,11 +184,11 @@ def test_cta_pair_variant_equals_the_single_cta_kernel(spec, sizes):
         parity_case(con, dtype, "normal", 41, 1.0, 0.5, repeat=2, tile_m=256, tile_n=256)
         a, b, c = make_inputs(con, dtype, "normal", 41, 0.5)
         outs = []
-        for switch in (0, 16384):  # 16384: never use the pair variant
+        for switch in (0, g.GETT_OPT_NO_PAIR):
             da = torch.from_numpy(a.view(np.int16)).cuda()
             db = torch.from_numpy(b.view(np.int16)).cuda()
             dc = torch.from_numpy(c).cuda()
-            p = g.Plan(con, dtype, tile_m=256, tile_n=256, reserved0=switch)
+            p = g.Plan(con, dtype, tile_m=256, tile_n=256, flags=switch)
             p(1.0, da, db, 0.5, dc)
             torch.cuda.synchronize()
             assert p.device_status() == 0

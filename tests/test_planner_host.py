@@ -175,6 +175,7 @@ def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
         ("cfg2", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_TMA_FREE, g.GETT_LOAD_TMA_K, g.GETT_EPI_DIRECT),
         # cfg3: small N and K -> B is read once into shared memory, element by element
         ("cfg3", g.GETT_F32): (g.GETT_PATH_FFMA, g.GETT_LOAD_VEC_K, g.GETT_LOAD_SCALAR, g.GETT_EPI_DIRECT),
+        # cfg4: tiles straddle the 72-wide modes (72 = 64 + 8: the remainder is too narrow for atoms) -> gathers
         ("cfg4", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_DIRECT),
         ("cfg5", g.GETT_BF16_F32): (g.GETT_PATH_UMMA, g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_FREE, g.GETT_EPI_STAGED),
     }
@@ -200,7 +201,22 @@ def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
                          w5.label_names)
     i = g.Plan(padded, g.GETT_F32).info
     assert (i.loader_b, i.epilogue) == (g.GETT_LOAD_SCALAR, g.GETT_EPI_DIRECT)
-    # cfg4's 128-row tiles straddle the 72-wide modes: not boxes, so the gather loader stays
+    # 80-wide lead modes (80 = 64 + 16): tiles of 64 x 64 atoms -- 64 lead indices, or the last 16
+    # x 4 indices of the next mode, alternating with period 80 * 4 -- and slabs of 8 x 8 contracted
+    # indices (I_k ordered 8 x 72 x 9): the 64-wide atoms come by TMA, the others are gathered
+    at = parse_spec("C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]",
+                    dict(m0=80, m1=64, n0=64, n1=80, k0=72, k1=72))
+    i = g.Plan(at, g.GETT_BF16_F32).info
+    assert (i.loader_a, i.loader_b) == (g.GETT_LOAD_TMA_FREE, g.GETT_LOAD_TMA_FREE)
+    assert (i.digits_m, i.digits_n, i.digits_k) == (5, 5, 3) and (i.M, i.N, i.K) == (5120, 5120, 5184)
+    _tables_match(at, g.GETT_BF16_F32)
+    i = g.Plan(at, g.GETT_BF16_F32, flags=g.GETT_OPT_NO_ATOMS).info
+    assert (i.loader_a, i.loader_b) == (g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_VEC_FREE)
+    # ... a lead extent whose remainder does not divide 64 (40 = 0 * 64 + 40) keeps the gather
+    nob = parse_spec("C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]",
+                     dict(m0=40, m1=8, n0=8, n1=96, k0=72, k1=8))
+    i = g.Plan(nob, g.GETT_BF16_F32).info
+    assert (i.loader_a, i.loader_b) == (g.GETT_LOAD_VEC_FREE, g.GETT_LOAD_TMA_FREE)
     # a 4-D operand whose leading extents are multiples of the tile is a box of a 4-D tensor map
     boxy = parse_spec("C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]",
                       dict(m0=128, m1=3, n0=5, n1=256, k0=64, k1=3))
@@ -212,3 +228,36 @@ def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
     with pytest.raises(g.GettError) as e:
         g.Plan(odd, g.GETT_BF16_F32, path=g.GETT_PATH_UMMA)
     assert e.value.status == 4
+
+
+def test_operands_beyond_32_bit_offsets_go_to_the_scalar_kernel():
+    """The vector kernels keep operand offsets in 32 bits; a (padded) operand that spans more is
+    planned for the scalar-gather kernel, and forcing a vector path is refused.  No memory is
+    allocated: only the plan is made."""
+    huge = 1 << 33  # elements between consecutive columns of A: 32 GiB of fp32
+    for dtype, vec_path in ((g.GETT_F32, g.GETT_PATH_FFMA), (g.GETT_BF16_F32, g.GETT_PATH_UMMA)):
+        stride = huge if dtype == g.GETT_F32 else huge * 8
+        con = Contraction("wide", TensorSpec([0, 2], [128, 64], [1, stride]), TensorSpec([2, 1], [64, 128], [1, 64]),
+                          TensorSpec([0, 1], [128, 128], [1, 128]))
+        i = g.Plan(con, dtype).info
+        assert i.path == g.GETT_PATH_SIMT
+        with pytest.raises(g.GettError) as e:
+            g.Plan(con, dtype, path=vec_path)
+        assert e.value.status == 4
+        # just below the limit the vector path is still taken
+        small = Contraction("ok", TensorSpec([0, 2], [128, 64], [1, 1 << 20]), con.B, con.C)
+        assert g.Plan(small, dtype).info.path == vec_path
+
+
+def test_pair_variant_guard_rule():
+    """The CTA-pair variant may only see operands that are ordinary device memory of the plan's own GPU."""
+    import ctypes
+    lib = ctypes.CDLL(g.library_path())
+    f = lib.gett_internal_pointer_is_local
+    f.restype = ctypes.c_int
+    f.argtypes = [ctypes.c_int] * 3
+    DEVICE, HOST, MANAGED, UNREGISTERED = 2, 1, 3, 0
+    assert f(DEVICE, 0, 0) == 1 and f(DEVICE, 3, 3) == 1
+    assert f(DEVICE, 1, 0) == 0          # a peer GPU's memory
+    assert f(HOST, 0, 0) == 0 and f(MANAGED, 0, 0) == 0 and f(UNREGISTERED, 0, 0) == 0
+    assert f(DEVICE, -1, -1) == 0        # a plan without a device
