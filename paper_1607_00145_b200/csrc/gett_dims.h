@@ -104,10 +104,29 @@ struct GettWalk {
 };
 
 // Offsets of fused index `idx` in the two carrier tensors; returns the segment (0 or 1).
+// (A plain dimension takes the first loop, which is all the arithmetic it needs.)
 GETT_HD int gett_decompose(const GettDim& D, uint32_t idx, int64_t& oX, int64_t& oY)
 {
+    int64_t x = 0, y = 0;
+    if (D.seg1_dig == D.hi_dig) {
+        uint32_t rem = idx;
+#pragma unroll 1
+        for (int d = 0; d < D.ndig; ++d) {
+            uint32_t q = gett_fastdiv(rem, D.mul[d], D.sh[d]);
+            uint32_t r = rem - q * D.ext[d];
+            x += (int64_t)r * D.sX[d];
+            y += (int64_t)r * D.sY[d];
+            rem = q;
+        }
+        oX = x;
+        oY = y;
+        return 0;
+    }
     GettWalk w(D, idx);
-    int64_t x = w.seg ? D.seg1_bX : 0, y = w.seg ? D.seg1_bY : 0;
+    if (w.seg) {
+        x = D.seg1_bX;
+        y = D.seg1_bY;
+    }
     do {
 #pragma unroll 1
         for (int d = w.d; d < w.dend; ++d) {
@@ -126,8 +145,20 @@ GETT_HD int gett_decompose(const GettDim& D, uint32_t idx, int64_t& oX, int64_t&
 // The offset in the second carrier alone (M, N: the offset in C), for the unpacking code.
 GETT_HD int64_t gett_offset_y(const GettDim& D, uint32_t idx)
 {
+    int64_t y = 0;
+    if (D.seg1_dig == D.hi_dig) {
+        uint32_t rem = idx;
+#pragma unroll 1
+        for (int d = 0; d < D.ndig; ++d) {
+            uint32_t q = gett_fastdiv(rem, D.mul[d], D.sh[d]);
+            y += (int64_t)(rem - q * D.ext[d]) * D.sY[d];
+            rem = q;
+        }
+        return y;
+    }
     GettWalk w(D, idx);
-    int64_t y = w.seg ? D.seg1_bY : 0;
+    if (w.seg)
+        y = D.seg1_bY;
     do {
 #pragma unroll 1
         for (int d = w.d; d < w.dend; ++d) {

@@ -89,6 +89,7 @@ struct alignas(16) SmemTables { // the staging rows that follow it hold 128-bit 
     uint32_t rowTab[PROD_GROUPS][256 + 256];  // per producer group: row offsets (K-major operands)
     int32_t atomc[PROD_GROUPS][2][4][8];      // per producer group and operand: TMA coordinates (5) and
                                               // segment of each 64-wide atom of the current tile
+    int32_t slabc[PROD_GROUPS][2][8];         // ... and the current slab's part of the coordinates
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
     uint64_t drain; // after a give-up: the tensor core has finished what had been issued
     uint32_t tmem_base;
@@ -518,7 +519,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
 
 // The producer role.  A group of LANES threads (index gl inside the group, named barrier
 // gbar) owns the slabs with number it % ng == pg and fills their ring stage.
-template <bool A_VEC_K, bool B_VEC_K, int TILE_N, int TILE_M, int LANES>
+template <bool A_VEC_K, bool B_VEC_K, int TILE_N, int TILE_M, int LANES, bool HYBRID>
 __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const GettTmaMaps& tm, SmemTables* T,
                                               uint32_t stage0, uint32_t stages, uint32_t total_work,
                                               volatile int* abort_flag, uint32_t pg, uint32_t ng, uint32_t gl,
@@ -545,7 +546,8 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
     // stage's barrier counts their bytes.
     const bool tmaA = tm.a.use != 0, tmaB = tm.b.use != 0;
     // hybrid: the atoms of segment 1 of the operand's free dimension are gathered
-    const bool hybridA = tmaA && !A_VEC_K && tm.a.hybrid, hybridB = tmaB && !B_VEC_K && tm.b.hybrid;
+    // (HYBRID is the compile-time form of "some operand is hybrid": the common case carries no state for it)
+    const bool hybridA = HYBRID && tmaA && !A_VEC_K && tm.a.hybrid, hybridB = HYBRID && tmaB && !B_VEC_K && tm.b.hybrid;
     const bool all_tma = tmaA && tmaB; // no offset tables (and no barriers of the group) are needed
     constexpr uint32_t ATOM_STAGE_BYTES = 64 * TILE_K * 2; // one atom: 64 free indices x 64 k
     constexpr int NATOM_A = A_VEC_K ? 1 : TILE_M / 64, NATOM_B = B_VEC_K ? 1 : TILE_N / 64;
@@ -563,11 +565,10 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
             const uint32_t f = origin + 64u * (uint32_t)b;
             if (b > 0 && f >= D.size)
                 break; // atoms past the end of the dimension are not fetched (their rows are never stored)
-            int32_t c[5] = {0, 0, 0, 0, 0};
-            const int seg = gett_add_coords(D, f, co.fdim, co.fmul, c);
 #pragma unroll
             for (int i = 0; i < 5; ++i)
-                out[b][i] = c[i];
+                out[b][i] = 0;
+            const int seg = gett_add_coords(D, f, co.fdim, co.fmul, out[b]);
             out[b][5] = seg;
             bytes += seg == 0 ? ATOM_STAGE_BYTES : 0u;
             ++natom;
@@ -623,8 +624,12 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
             }
             const uint32_t s = it % stages;
             // the slab's part of the TMA coordinates, before the wait for the stage
-            int32_t ckA[5] = {0, 0, 0, 0, 0}, ckB[5] = {0, 0, 0, 0, 0};
-            if (gl == 0 && alive) {
+            int32_t* ckA = T->slabc[pg][0]; // (written and read by thread 0 of the group only)
+            int32_t* ckB = T->slabc[pg][1];
+            if (gl == 0 && alive && (tmaA || tmaB)) {
+#pragma unroll
+                for (int i = 0; i < 5; ++i)
+                    ckA[i] = ckB[i] = 0;
                 if (tmaA)
                     gett_add_coords(g.K, k0, tm.a.co.kdim, tm.a.co.kmul, ckA);
                 if (tmaB)
@@ -641,7 +646,7 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
             if (gl == 0 && tma_bytes && !GETT_DBG(g, 4)) {
                 ptx::mbar_expect_tx(fullbar, tma_bytes);
                 if (tmaA) {
-                    const int32_t(&ck)[5] = ckA;
+                    const int32_t* ck = ckA;
                     int32_t c[5];
 #ifdef GETT_UMMA_CLUSTER
                     // my half of the A tile, delivered to both CTAs of the pair (the partner
@@ -651,7 +656,10 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
 #pragma unroll
                         for (int i = 0; i < 5; ++i)
                             c[i] = atomA[0][i] + ck[i];
-                        c[tm.a.co.fdim[0]] += (int32_t)(half * (TILE_M / 2));
+                        const int fd0 = tm.a.co.fdim[0];
+#pragma unroll
+                        for (int i = 0; i < 5; ++i)
+                            c[i] += i == fd0 ? (int32_t)(half * (TILE_M / 2)) : 0;
                         ptx_mc::tma_load_pair(sa + half * (A_STAGE_BYTES / 2), tm.a.map, fullbar, tm.a.co.rank, c);
                     } else {
                         for (int b = (int)half * (NATOM_A / 2); b < (int)(half + 1) * (NATOM_A / 2) && b < natomA; ++b) {
@@ -673,7 +681,7 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
 #endif
                 }
                 if (tmaB) {
-                    const int32_t(&ck)[5] = ckB;
+                    const int32_t* ck = ckB;
                     int32_t c[5];
                     for (int b = 0; b < natomB; ++b) {
                         if (atomB[b][5])
@@ -779,14 +787,23 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
         // warps own whole slabs round-robin.  The ring depth is a multiple of the group
         // count, so a stage's barriers are always used by the same group.
         const uint32_t ng = (uint32_t)g.prod_groups;
+        const bool hybrid = (tm.a.use && tm.a.hybrid) || (tm.b.use && tm.b.hybrid);
         if (ng == 1) {
-            producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, PROD_THREADS>(
-                g, tm, T, stage0, stages, total_work, abort_flag, 0, 1, threadIdx.x - PROD_WARP0 * 32, 3);
+            if (hybrid)
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, PROD_THREADS, true>(
+                    g, tm, T, stage0, stages, total_work, abort_flag, 0, 1, threadIdx.x - PROD_WARP0 * 32, 3);
+            else
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, PROD_THREADS, false>(
+                    g, tm, T, stage0, stages, total_work, abort_flag, 0, 1, threadIdx.x - PROD_WARP0 * 32, 3);
         } else {
             const uint32_t pg = (warp - PROD_WARP0) / WARPS_PER_GROUP;
-            producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, GROUP_LANES>(
-                g, tm, T, stage0, stages, total_work, abort_flag, pg, ng,
-                threadIdx.x - (PROD_WARP0 + pg * WARPS_PER_GROUP) * 32, 3 + pg);
+            const uint32_t gl = threadIdx.x - (PROD_WARP0 + pg * WARPS_PER_GROUP) * 32;
+            if (hybrid)
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, GROUP_LANES, true>(
+                    g, tm, T, stage0, stages, total_work, abort_flag, pg, ng, gl, 3 + pg);
+            else
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, GROUP_LANES, false>(
+                    g, tm, T, stage0, stages, total_work, abort_flag, pg, ng, gl, 3 + pg);
         }
     } else if (warp == MMA_WARP) {
         // ------------------------------ MMA issuer -----------------------------
