@@ -453,6 +453,13 @@ def run_ours(args):
             out["targets"] = targets_summary(out["workloads"])
         if args.pool:
             out.update(run_pool(torch, g, peaks, args))
+        if args.paper_pool:
+            from workloads.paper_benchmark import fig11_sweep, paper_pool
+            out.update(run_pool(torch, g, peaks, args, paper_pool("sp"), "paper_pool"))
+            out.update(run_pool(torch, g, peaks, args, fig11_sweep(), "fig11"))
+            # the paper's own figures for the same statistic (one Haswell core, MKL GEMM): context only
+            out["paper_pool_context"] = {"gett_vs_equal_gemm_percent_sp": {"min": 72.4, "mean": 98.1, "max": 141.4},
+                                         "source": "Sec. 7.2, Fig. 9"}
     elif rank == 0:
         # ---- end to end through the C ABI with host buffers ----
         pin = [torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
@@ -720,17 +727,18 @@ def targets_summary(rows):
     return {"threshold": 0.70, "pairs": out, "met": sum(1 for x in out if x["met"]), "of": len(out)}
 
 
-def run_pool(torch, g, peaks, args):
-    """The seeded pool of synthetic contractions (workloads.pool): per item and dtype the plan,
+def run_pool(torch, g, peaks, args, items=None, label="pool"):
+    """A pool of contractions -- the seeded synthetic pool (workloads.pool) or the paper's own 48
+    shapes and its Fig. 11 sweep (workloads.paper_benchmark): per item and dtype the plan,
     TFLOP/s, roofline fraction and the ratio to the equal-sized GEMM through the same library
     (the paper's Sec. 7 statistic), plus the distribution of that ratio."""
     from workloads import pool
     rows = []
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    for w in pool():
+    for w in (items if items is not None else pool()):
         con = w.contraction
         for dtype in w.dtypes:
-            a, b, c = make_inputs(con, dtype, w.dist, w.seed, w.beta)
+            a, b, c = make_inputs(con, dtype, w.dist, w.seed, w.beta, cache=True)
             dev = (_to_dev(a, torch), _to_dev(b, torch), _to_dev(c, torch))
             t, info = time_contraction(torch, g, con, dtype, w.alpha, w.beta, dev, args.all_steps, 3)
             flush.zero_()
@@ -748,12 +756,17 @@ def run_pool(torch, g, peaks, args):
                          "tile": [info["tile_m"], info["tile_n"], info["tile_k"]],
                          "split_k": info["split_k"], "speedup_vs_equal_gemm": t_eq / t})
             del dev, gdev
-    out = {"pool": rows}
+    out = {label: rows}
     for name in sorted(DTYPE_BY_NAME):
         r = np.array([x["speedup_vs_equal_gemm"] for x in rows if x["dtype"] == name])
+        f = np.array([x["roofline_frac"] for x in rows if x["dtype"] == name])
         if r.size:
-            out[f"ratio_to_equal_gemm_{name}"] = {"min": float(r.min()), "median": float(np.median(r)),
-                                                  "max": float(r.max()), "n": int(r.size)}
+            out[f"{label}_ratio_to_equal_gemm_{name}"] = {
+                "min": float(r.min()), "mean": float(r.mean()), "median": float(np.median(r)),
+                "max": float(r.max()), "n": int(r.size)}
+            out[f"{label}_roofline_frac_{name}"] = {
+                "min": float(f.min()), "median": float(np.median(f)), "max": float(f.max()),
+                "at_least_0.7": int((f >= 0.7).sum()), "n": int(f.size)}
     return out
 
 
@@ -770,6 +783,8 @@ def main():
     ap.add_argument("--scale", default="", help="override extents, e.g. m=4096,n=4096 (profiling)")
     ap.add_argument("--pool", action="store_true",
                     help="with --kernel-only: also time the seeded pool of synthetic contractions")
+    ap.add_argument("--paper-pool", action="store_true",
+                    help="with --kernel-only: the paper's 48 contractions (Table III extents) and its Fig. 11 sweep")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end, equal-GEMM and CPU legs (profiling runs)")
     ap.add_argument("--all", action="store_true", help="with --kernel-only: also time every workload")

@@ -81,7 +81,11 @@ typedef enum {
     GETT_LOAD_VEC_FREE = 1, /* 16-byte vectors along the operand's free (M or N) dimension */
     GETT_LOAD_VEC_K = 2,    /* 16-byte vectors along the contracted dimension              */
     GETT_LOAD_TMA_FREE = 3, /* tensor-map (TMA) boxes, operand's stride-1 mode is free      */
-    GETT_LOAD_TMA_K = 4     /* tensor-map (TMA) boxes, operand's stride-1 mode is contracted */
+    GETT_LOAD_TMA_K = 4,    /* tensor-map (TMA) boxes, operand's stride-1 mode is contracted */
+    GETT_LOAD_VEC_KT = 5    /* 16-bit operand whose stride-1 mode is a contracted mode other than the one
+                               the other operand runs along: 16-byte pieces are read along its own
+                               stride-1 mode and 8 x 8 blocks are transposed in registers on their way
+                               to shared memory (Sec. 3.2.2: packing is a transposition)             */
 } gett_loader_t;
 
 typedef enum {

@@ -9,6 +9,6 @@ from .binding import (GettError, Plan, gett_contract, gett_plan_create, gett_pla
 from .binding import (GETT_F32, GETT_BF16_F32, GETT_F16_F32, GETT_PATH_AUTO, GETT_PATH_SIMT,  # noqa: F401
                       GETT_PATH_FFMA, GETT_PATH_UMMA, GETT_EPI_AUTO, GETT_EPI_DIRECT,
                       GETT_EPI_STAGED, GETT_LOAD_SCALAR, GETT_LOAD_VEC_FREE, GETT_LOAD_VEC_K,
-                      GETT_LOAD_TMA_FREE, GETT_LOAD_TMA_K,
+                      GETT_LOAD_TMA_FREE, GETT_LOAD_TMA_K, GETT_LOAD_VEC_KT,
                       GETT_OPT_NO_TMA, GETT_OPT_NO_PAIR, GETT_OPT_NO_EXCHANGE, GETT_OPT_NO_ATOMS,
                       TABLE_NAMES)

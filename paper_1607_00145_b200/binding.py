@@ -11,7 +11,7 @@ GETT_MAX_MODES = 12
 GETT_F32, GETT_BF16_F32, GETT_F16_F32 = 0, 1, 2
 GETT_PATH_AUTO, GETT_PATH_SIMT, GETT_PATH_FFMA, GETT_PATH_UMMA = 0, 1, 2, 3
 GETT_LOAD_SCALAR, GETT_LOAD_VEC_FREE, GETT_LOAD_VEC_K = 0, 1, 2
-GETT_LOAD_TMA_FREE, GETT_LOAD_TMA_K = 3, 4
+GETT_LOAD_TMA_FREE, GETT_LOAD_TMA_K, GETT_LOAD_VEC_KT = 3, 4, 5
 GETT_EPI_AUTO, GETT_EPI_DIRECT, GETT_EPI_STAGED = 0, 1, 2
 GETT_OPT_NO_TMA, GETT_OPT_NO_PAIR, GETT_OPT_NO_EXCHANGE, GETT_OPT_NO_ATOMS = 1, 2, 4, 8
 TABLE_NAMES = ("A_M", "A_K", "B_N", "B_K", "C_M", "C_N")

@@ -237,13 +237,18 @@ struct OperandLoader {
         }
     }
 
-    template <bool FAST>
+    // KT (K-major staging only): the operand's 16-byte pieces run along K's SECOND digit while the
+    // slab's k order is first digit (extent 8) fastest.  Piece number i of a row is then read
+    // from first-digit index i (table entry i, not 8 i) and holds eight consecutive indices of
+    // the second digit: the row arrives as the transpose of what the tensor core needs, and
+    // transpose_rows() below puts it right.
+    template <bool FAST, bool KT = false>
     __device__ __forceinline__ void load_slab(const char* __restrict__ base, uint32_t stage_dst,
                                               const uint32_t* kTab, const uint32_t* rowTab,
                                               uint32_t gl) const
     {
         if (VEC_K) {
-            const uint32_t k16 = kTab[(gl & 7) * 8];
+            const uint32_t k16 = kTab[KT ? (gl & 7) : (gl & 7) * 8];
             const uint32_t dst = stage_dst + dst_lane;
             const uint32_t* rows = rowTab + (gl >> 3);
 #pragma unroll 8
@@ -279,6 +284,33 @@ struct OperandLoader {
         }
     }
 };
+
+// In-place transposition of the rows a warp has just copied with load_slab<.., KT = true>
+// (packing as a transposition, Sec. 3.2.2 / Eq. 10, at the granularity of 8 x 8 blocks).
+// A row of the K-major stage (one free index, 128 bytes, pieces XOR-swizzled by row % 8) holds
+// an 8 x 8 block of 16-bit elements: piece i = first-digit index i, eight second-digit indices.
+// The tensor core needs piece j = second-digit index j, eight first-digit indices.  A warp
+// owns rows r0 .. r0 + 3 of every pass (the rows its own lanes copied), reads four blocks
+// transposed (ldmatrix.trans: lanes 8 q .. 8 q + 7 give the piece addresses of block q) and
+// writes them back to the same rows (stmatrix).
+template <int R, int LANES>
+__device__ __forceinline__ void transpose_rows(uint32_t stage_dst, uint32_t gl)
+{
+    constexpr int RP = LANES / 8; // rows per pass of the K-major gather
+    const uint32_t lane = gl & 31;
+    const uint32_t row0 = ((gl >> 5) << 2) + (lane >> 3); // my block's row in pass 0
+    const uint32_t i = lane & 7;                          // the piece whose address I supply
+#pragma unroll 4
+    for (uint32_t r = row0; r < (uint32_t)R; r += RP) {
+        // (rows of a pass beyond R do not exist; R and RP are multiples of 4, so a warp's four
+        //  blocks are either all inside or all outside)
+        const uint32_t addr = stage_dst + r * 128 + ((i ^ (r & 7)) << 4);
+        uint32_t v0, v1, v2, v3;
+        ptx::ldmatrix_x4_trans(addr, v0, v1, v2, v3);
+        __syncwarp(); // all four blocks are in registers before any of them is overwritten
+        ptx::stmatrix_x4(addr, v0, v1, v2, v3);
+    }
+}
 
 // ---- staged epilogue (Eq. 11 as a transposition through shared memory) ----
 // The accumulator is walked in chunks of up to 64 columns, and inside a chunk the columns
@@ -519,7 +551,7 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
 
 // The producer role.  A group of LANES threads (index gl inside the group, named barrier
 // gbar) owns the slabs with number it % ng == pg and fills their ring stage.
-template <bool A_VEC_K, bool B_VEC_K, int TILE_N, int TILE_M, int LANES, bool HYBRID>
+template <bool A_VEC_K, bool B_VEC_K, int TILE_N, int TILE_M, int LANES, bool HYBRID, bool B_TRANS>
 __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const GettTmaMaps& tm, SmemTables* T,
                                               uint32_t stage0, uint32_t stages, uint32_t total_work,
                                               volatile int* abort_flag, uint32_t pg, uint32_t ng, uint32_t gl,
@@ -698,13 +730,30 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
             } else if (tile_full && k0 + TILE_K <= wi.kend) {
                 if (!tmaA)
                     la.template load_slab<true>(baseA, sa, kA, rowA, gl);
-                if (!tmaB)
+                if (!tmaB && !B_TRANS)
                     lb.template load_slab<true>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+                if (B_TRANS) { // B first, as a copy group of its own (waited for below)
+                    lb.template load_slab<true, true>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+                    ptx::cp_async_commit();
+                }
             } else {
                 if (!tmaA)
                     la.template load_slab<false>(baseA, sa, kA, rowA, gl);
-                if (!tmaB)
+                if (!tmaB && !B_TRANS)
                     lb.template load_slab<false>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+                if (B_TRANS) {
+                    lb.template load_slab<false, true>(baseB, sa + A_STAGE_BYTES, kB, rowB, gl);
+                    ptx::cp_async_commit();
+                }
+            }
+            if (B_TRANS) {
+                // B's rows have arrived transposed: once this warp's own copies of them have landed,
+                // it transposes its rows in place.  Those are ordinary stores, so the thread also
+                // arrives on the barrier in the ordinary way (A's copies are tracked separately).
+                ptx::cp_async_wait<0>();
+                __syncwarp();
+                transpose_rows<TILE_N, LANES>(sa + A_STAGE_BYTES, gl);
+                ptx::mbar_arrive(fullbar);
             }
             if ((hybridA || hybridB) && !GETT_DBG(g, 4 | 1024)) { // (probe 1024: the gathered atoms are skipped)
                 int64_t xa, xb;
@@ -727,7 +776,7 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
     ptx::cp_async_wait_all();
 }
 
-template <bool A_VEC_K, bool B_VEC_K, int TILE_N, int TILE_M>
+template <bool A_VEC_K, bool B_VEC_K, int TILE_N, int TILE_M, bool B_TRANS = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant__ GettTmaMaps tm)
 {
@@ -754,7 +803,10 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < stages; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&T->full[s]), g.prod_groups == 1 ? PROD_THREADS : GROUP_LANES); // the slab's producers
+            // the slab's producers (twice each with the transposing loader: once for their asynchronous
+            // copies, once for their ordinary stores)
+            ptx::mbar_init(ptx::smem_u32(&T->full[s]),
+                           (g.prod_groups == 1 ? PROD_THREADS : GROUP_LANES) * (B_TRANS ? 2 : 1));
 #ifdef GETT_UMMA_CLUSTER
             ptx::mbar_init(ptx::smem_u32(&T->empty[s]), 2); // both CTAs of the pair are done with the stage
 #else
@@ -790,19 +842,19 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
         const bool hybrid = (tm.a.use && tm.a.hybrid) || (tm.b.use && tm.b.hybrid);
         if (ng == 1) {
             if (hybrid)
-                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, PROD_THREADS, true>(
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, PROD_THREADS, true, B_TRANS>(
                     g, tm, T, stage0, stages, total_work, abort_flag, 0, 1, threadIdx.x - PROD_WARP0 * 32, 3);
             else
-                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, PROD_THREADS, false>(
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, PROD_THREADS, false, B_TRANS>(
                     g, tm, T, stage0, stages, total_work, abort_flag, 0, 1, threadIdx.x - PROD_WARP0 * 32, 3);
         } else {
             const uint32_t pg = (warp - PROD_WARP0) / WARPS_PER_GROUP;
             const uint32_t gl = threadIdx.x - (PROD_WARP0 + pg * WARPS_PER_GROUP) * 32;
             if (hybrid)
-                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, GROUP_LANES, true>(
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, GROUP_LANES, true, B_TRANS>(
                     g, tm, T, stage0, stages, total_work, abort_flag, pg, ng, gl, 3 + pg);
             else
-                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, GROUP_LANES, false>(
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, GROUP_LANES, false, B_TRANS>(
                     g, tm, T, stage0, stages, total_work, abort_flag, pg, ng, gl, 3 + pg);
         }
     } else if (warp == MMA_WARP) {
@@ -1001,7 +1053,7 @@ int gett_umma_block() { return NUM_THREADS; }
 
 int gett_umma_prod_groups(int stages) { return stages >= PROD_GROUPS ? PROD_GROUPS : stages; }
 
-template <bool AK, bool BK>
+template <bool AK, bool BK, bool BT = false>
 static cudaError_t launch_tn(const GettKernelArgs& args, const GettTmaMaps& maps, int grid, int smem,
                              cudaStream_t stream)
 {
@@ -1009,13 +1061,13 @@ static cudaError_t launch_tn(const GettKernelArgs& args, const GettTmaMaps& maps
     if (args.tile_m == 256) {
         if (args.tile_n != 256)
             return cudaErrorInvalidValue;
-        k = gett_umma_kernel<AK, BK, 256, 256>;
+        k = gett_umma_kernel<AK, BK, 256, 256, BT>;
     } else {
         switch (args.tile_n) {
-        case 64: k = gett_umma_kernel<AK, BK, 64, 128>; break;
-        case 128: k = gett_umma_kernel<AK, BK, 128, 128>; break;
-        case 192: k = gett_umma_kernel<AK, BK, 192, 128>; break;
-        case 256: k = gett_umma_kernel<AK, BK, 256, 128>; break;
+        case 64: k = gett_umma_kernel<AK, BK, 64, 128, BT>; break;
+        case 128: k = gett_umma_kernel<AK, BK, 128, 128, BT>; break;
+        case 192: k = gett_umma_kernel<AK, BK, 192, 128, BT>; break;
+        case 256: k = gett_umma_kernel<AK, BK, 256, 128, BT>; break;
         default: return cudaErrorInvalidValue;
         }
     }
@@ -1030,6 +1082,8 @@ cudaError_t gett_launch_umma(const GettKernelArgs& args, const GettTmaMaps& maps
                              cudaStream_t stream)
 {
     const bool ak = args.loader_a == GETT_LOAD_VEC_K, bk = args.loader_b == GETT_LOAD_VEC_K;
+    if (args.loader_b == GETT_LOAD_VEC_KT) // B staged K-major through the transposing loader; A K-major
+        return ak ? launch_tn<true, true, true>(args, maps, grid, smem, stream) : cudaErrorInvalidValue;
     if (ak && bk)
         return launch_tn<true, true>(args, maps, grid, smem, stream);
     if (ak)

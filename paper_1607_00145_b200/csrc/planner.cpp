@@ -654,6 +654,26 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         }
     }
     p->tk = order_with_lead(ik, leadK);
+    // 16-bit operands whose stride-1 modes are two different contracted modes u (A's) and v (B's):
+    // slabs of 8 indices of u times 8 consecutive indices of v (Sec. 3.2.1: a sub-tensor made
+    // of pieces of two modes).  A is then read in 16-byte pieces along u as usual; B is read
+    // in 16-byte pieces along v and its 8 x 8 blocks are transposed on the way (Sec. 3.2.2).
+    bool k_transposed = false;
+    if (dtype != GETT_F32) {
+        const int uA = find_unit(ik, 0), uB = find_unit(ik, 1);
+        if (uA >= 0 && uB >= 0 && uA != uB && ik[uA].ext % 8 == 0 && ik[uB].ext % 8 == 0) {
+            std::vector<GettDigit> t;
+            t.push_back({uA, 8, 1, 0});
+            t.push_back({uB, ik[uB].ext, 1, 0});
+            if (ik[uA].ext > 8)
+                t.push_back({uA, ik[uA].ext / 8, 8, 0});
+            for (int i = 0; i < (int)ik.size(); ++i)
+                if (i != uA && i != uB)
+                    t.push_back({i, ik[i].ext, 1, 0});
+            p->tk = t;
+            k_transposed = true;
+        }
+    }
     p->tm_seg1 = p->tn_seg1 = p->tm_hi = p->tn_hi = -1;
     if ((rc = make_dim(im, p->tm, 0, 2, p->M)) || (rc = make_dim(in, p->tn, 1, 2, p->N)) ||
         (rc = make_dim(ik, p->tk, 0, 1, p->K)))
@@ -691,6 +711,17 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     info.loader_b = vec_ok(p->N, true, p->K, false, vec)   ? GETT_LOAD_VEC_FREE
                     : vec_ok(p->K, false, p->N, true, vec) ? GETT_LOAD_VEC_K
                                                            : GETT_LOAD_SCALAR;
+    if (k_transposed && info.loader_a == GETT_LOAD_VEC_K && info.loader_b == GETT_LOAD_SCALAR && p->K.ndig >= 2 &&
+        p->K.ext[0] == 8 && p->K.sY[1] == 1 && p->K.ext[1] % 8 == 0) {
+        // B in 16-byte pieces along K's second digit: every other stride of B must keep them aligned
+        bool ok = p->K.sY[0] % 8 == 0;
+        for (int d = 2; d < p->K.ndig; ++d)
+            ok = ok && p->K.sY[d] % 8 == 0;
+        for (int d = 0; d < p->N.ndig; ++d)
+            ok = ok && p->N.sX[d] % 8 == 0;
+        if (ok)
+            info.loader_b = GETT_LOAD_VEC_KT;
+    }
 
     // ---- path ----
     int path = o.path;

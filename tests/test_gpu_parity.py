@@ -236,6 +236,27 @@ def test_tensor_times_small_matrix_kernel_a_free_major(spec, sizes, vec_rows):
         assert info.path == g.GETT_PATH_FFMA and info.tile_m == 256 and info.loader_a == g.GETT_LOAD_VEC_FREE
 
 
+@pytest.mark.parametrize("spec,sizes", [
+    ("C[a,b] = A[c,a,d] * B[d,c,b]", dict(a=200, b=136, c=24, d=40)),              # the paper's ab-cad-dcb layout
+    ("C[a,b,c,d] = A[e,a,f,b] * B[f,d,e,c]", dict(a=24, b=9, c=7, d=24, e=16, f=24)),  # abcd-eafb-fdec
+    ("C[a,b] = A[c,a,d,e] * B[d,e,c,b]", dict(a=136, b=72, c=8, d=16, e=5)),       # a third contracted mode, u of extent 8
+])
+def test_transposing_loader_for_two_different_contracted_stride1_modes(spec, sizes):
+    """16-bit operands whose stride-1 modes are two different contracted modes: B is read along its
+    own stride-1 mode and transposed in 8 x 8 blocks on the way to shared memory, so the
+    tensor-core kernel applies (every tile width, split-K, both 16-bit types, ragged tiles)."""
+    con = parse_spec(spec, sizes)
+    for dtype in (BF16_F32, F16_F32):
+        ratio, info = parity_case(con, dtype, "normal", 61, 1.0, 0.5, repeat=2)
+        assert info.path == g.GETT_PATH_UMMA
+        assert (info.loader_a, info.loader_b) == (g.GETT_LOAD_VEC_K, g.GETT_LOAD_VEC_KT)
+    for tile_n in (64, 128, 192, 256):
+        parity_case(con, BF16_F32, "normal", 61, -0.5, 0.0, repeat=2, tile_n=tile_n)
+    parity_case(con, BF16_F32, "normal", 61, 1.0, 1.0, repeat=2, tile_m=256, tile_n=256)
+    parity_case(con, BF16_F32, "normal", 61, 1.0, 0.0, repeat=2, split_k=3)
+    parity_case(con, BF16_F32, "normal", 61, 1.0, 0.0, path=g.GETT_PATH_SIMT)
+
+
 @pytest.mark.parametrize("seed", range(48))
 def test_fuzz_random_contractions(seed):
     rng = np.random.default_rng(5000 + seed)

@@ -336,6 +336,21 @@ def pool(seed: int = 2016, per_family: int = 5) -> List[Workload]:
     return out
 
 
+_DRAW_CACHE: Dict[Tuple[str, int, str, int], np.ndarray] = {}
+
+
+def draw_cached(dist: str, seed: int, tensor: str, n: int, keep: int = 8) -> np.ndarray:
+    """draw() with the last few results kept (an element depends only on seed, tensor and storage
+    offset, so contractions that differ only in the order of their modes share their arrays).
+    The returned array is shared: callers must not write to it."""
+    key = (dist, seed, tensor, n)
+    if key not in _DRAW_CACHE:
+        while len(_DRAW_CACHE) >= keep:
+            _DRAW_CACHE.pop(next(iter(_DRAW_CACHE)))
+        _DRAW_CACHE[key] = draw(dist, seed, tensor, n)
+    return _DRAW_CACHE[key]
+
+
 def draw(dist: str, seed: int, tensor: str, n: int) -> np.ndarray:
     tid = TENSOR_ID[tensor]
     if dist == "uniform":
@@ -347,14 +362,16 @@ def draw(dist: str, seed: int, tensor: str, n: int) -> np.ndarray:
     raise ValueError(dist)
 
 
-def make_inputs(con: Contraction, dtype: int, dist: str, seed: int, beta: float):
+def make_inputs(con: Contraction, dtype: int, dist: str, seed: int, beta: float, cache: bool = False):
     """(A_stored, B_stored, C_old) flat storage arrays of each tensor's span.
 
     A and B are fp32 or uint16 bit patterns depending on dtype; C_old is fp32
     (drawn uniform[-1,1) when beta != 0, zeros otherwise, as the workloads say).
+    cache: reuse the fp32 draws of earlier calls with the same seed and span (read-only arrays).
     """
-    a = encode_operand(draw(dist, seed, "A", con.A.span), dtype)
-    b = encode_operand(draw(dist, seed, "B", con.B.span), dtype)
+    d = draw_cached if cache else draw
+    a = encode_operand(d(dist, seed, "A", con.A.span), dtype)
+    b = encode_operand(d(dist, seed, "B", con.B.span), dtype)
     if beta != 0.0:
         c = uniform_pm1(seed, TENSOR_ID["C"], con.C.span)
     else:
