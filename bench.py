@@ -271,9 +271,15 @@ def _to_dev(x, torch):
     return torch.from_numpy(x).cuda()
 
 
+SEARCH = 0  # --search k: every plan of the pool runs is made with opts.search = k
+
+
 def time_contraction(torch, g, con, dtype, alpha, beta, dev, steps, warmup, opts=None):
     """Device-timed launches of one plan on resident inputs.  Returns seconds/launch."""
-    plan = g.Plan(con, dtype, **(opts or {}))
+    opts = dict(opts or {})
+    if SEARCH:
+        opts["search"] = SEARCH
+    plan = g.Plan(con, dtype, **opts)
     a, b, c = dev
     stream = torch.cuda.current_stream()
     for _ in range(warmup):
@@ -727,6 +733,88 @@ def targets_summary(rows):
     return {"threshold": 0.70, "pairs": out, "met": sum(1 for x in out if x["met"]), "of": len(out)}
 
 
+def ttgt_seconds(torch, g, con, dtype, alpha, beta, dev, steps, flush):
+    """Transpose-Transpose-GEMM-Transpose on the GPU (Sec. 4, Listing 5), the approach GETT is
+    measured against: A and B are unfolded into packed matrices A'[M,K], B'[K,N] by explicit
+    transpositions into auxiliary memory (torch's permuting copy), multiplied by the plain GEMM of
+    this library, and the result C'[M,N] is folded back into C's layout.  Transpositions that are
+    the identity are skipped (as the paper's TTGT candidates do).  Returns (seconds, seconds spent
+    in the transpositions).  Every tensor must be packed."""
+    im, in_, ik = con.index_sets()
+    ext = con.extent_of()
+
+    def view(t, x):       # the flat device array as a torch view with one dim per mode (first mode fastest)
+        return x.view(tuple(reversed(t.extents))).permute(*reversed(range(len(t.extents))))
+
+    def unfold(t, x, rows, cols):   # -> packed matrix [prod rows, prod cols], rows fastest
+        v = view(t, x)
+        order = [t.labels.index(l) for l in rows + cols]
+        identity = order == list(range(len(order)))
+        return v.permute(*order), identity
+
+    a, b, c = dev
+    el = torch.bfloat16 if dtype != F32 else torch.float32
+    a_t, b_t = (a.view(torch.bfloat16), b.view(torch.bfloat16)) if dtype != F32 else (a, b)
+    M, N, K = con.mnk()
+    eg = equal_gemm(con)
+    plan = g.Plan(eg, dtype)
+    a_m = torch.empty(M * K, dtype=el, device="cuda")
+    b_m = torch.empty(K * N, dtype=el, device="cuda")
+    c_m = torch.empty(M * N, dtype=torch.float32, device="cuda")
+    va, ida = unfold(con.A, a_t, im, ik)
+    vb, idb = unfold(con.B, b_t, ik, in_)
+    c_order = [con.C.labels.index(l) for l in im + in_]
+    idc = c_order == list(range(len(c_order)))
+    vc = view(con.C, c)
+    shape_a = tuple(reversed([ext[l] for l in im + ik]))
+    shape_b = tuple(reversed([ext[l] for l in ik + in_]))
+    shape_c = tuple(reversed([ext[l] for l in im + in_]))
+    stream = torch.cuda.current_stream()
+
+    def to_packed(dst, v, shape):   # dst (first-mode-fastest packed) <- v
+        dst.view(shape).copy_(v.permute(*reversed(range(v.dim()))))
+
+    def step(timers=None):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if timers is not None else None
+        if ev:
+            ev[0].record(stream)
+        if not ida:
+            to_packed(a_m, va, shape_a)
+        if not idb:
+            to_packed(b_m, vb, shape_b)
+        if not idc and beta != 0.0:   # C' <- C for the update
+            to_packed(c_m, vc.permute(*c_order), shape_c)
+        if ev:
+            ev[1].record(stream)
+        am = a_m if not ida else a_t
+        bm = b_m if not idb else b_t
+        cm = c_m if not idc else c
+        plan(alpha, am.view(torch.int16) if dtype != F32 else am, bm.view(torch.int16) if dtype != F32 else bm,
+             beta, cm, stream)
+        if ev:
+            ev[2].record(stream)
+        if not idc:   # C <- C'
+            inv = [c_order.index(i) for i in range(len(c_order))]
+            vc.copy_(c_m.view(shape_c).permute(*reversed(range(len(shape_c)))).permute(*inv))
+        if ev:
+            ev[3].record(stream)
+            timers.append(ev)
+
+    for _ in range(2):
+        step()
+    torch.cuda.synchronize()
+    timers = []
+    for _ in range(steps):
+        if flush is not None:
+            flush.zero_()
+        step(timers)
+    torch.cuda.synchronize()
+    plan.close()
+    tot = np.array([e[0].elapsed_time(e[3]) for e in timers]) / 1e3
+    tr = np.array([e[0].elapsed_time(e[1]) + e[2].elapsed_time(e[3]) for e in timers]) / 1e3
+    return float(np.median(tot)), float(np.median(tr))
+
+
 def run_pool(torch, g, peaks, args, items=None, label="pool"):
     """A pool of contractions -- the seeded synthetic pool (workloads.pool) or the paper's own 48
     shapes and its Fig. 11 sweep (workloads.paper_benchmark): per item and dtype the plan,
@@ -749,12 +837,19 @@ def run_pool(torch, g, peaks, args, items=None, label="pool"):
             gdev = (_to_dev(ga, torch), _to_dev(gb, torch), _to_dev(gc, torch))
             t_eq, _ = time_contraction(torch, g, eg, dtype, w.alpha, w.beta, gdev, args.all_steps, 3)
             M, N, K = con.mnk()
-            rows.append({"item": w.key, "spec": con.name, "dtype": DTYPE_NAMES[dtype], "mnk": [M, N, K],
+            extra = {}
+            if args.ttgt:
+                t_ttgt, t_tr = ttgt_seconds(torch, g, con, dtype, w.alpha, w.beta, dev, args.all_steps, None)
+                extra = {"ttgt_ms": t_ttgt * 1e3, "ttgt_transpose_share": t_tr / t_ttgt,
+                         "speedup_vs_ttgt": t_ttgt / t}
+            rows.append({**extra, "item": w.key, "spec": con.name, "dtype": DTYPE_NAMES[dtype], "mnk": [M, N, K],
                          "ms": t * 1e3, "tflops": con.flops() / t / 1e12, "bound": bound,
                          "roofline_frac": t_roof / t, "path": info["path"],
                          "loaders": [info["loader_a"], info["loader_b"]], "epilogue": info["epilogue"],
                          "tile": [info["tile_m"], info["tile_n"], info["tile_k"]],
-                         "split_k": info["split_k"], "speedup_vs_equal_gemm": t_eq / t})
+                         "split_k": info["split_k"], "speedup_vs_equal_gemm": t_eq / t,
+                         "model_us": info["model_us"], "candidates": info["candidates"],
+                         "model_rank": info["model_rank"], "timed": info["timed"]})
             del dev, gdev
     out = {label: rows}
     for name in sorted(DTYPE_BY_NAME):
@@ -764,6 +859,11 @@ def run_pool(torch, g, peaks, args, items=None, label="pool"):
             out[f"{label}_ratio_to_equal_gemm_{name}"] = {
                 "min": float(r.min()), "mean": float(r.mean()), "median": float(np.median(r)),
                 "max": float(r.max()), "n": int(r.size)}
+            tt = np.array([x["speedup_vs_ttgt"] for x in rows if x["dtype"] == name and "speedup_vs_ttgt" in x])
+            if tt.size:
+                out[f"{label}_speedup_vs_ttgt_{name}"] = {"min": float(tt.min()), "mean": float(tt.mean()),
+                                                          "median": float(np.median(tt)), "max": float(tt.max()),
+                                                          "n": int(tt.size)}
             out[f"{label}_roofline_frac_{name}"] = {
                 "min": float(f.min()), "median": float(np.median(f)), "max": float(f.max()),
                 "at_least_0.7": int((f >= 0.7).sum()), "n": int(f.size)}
@@ -785,6 +885,11 @@ def main():
                     help="with --kernel-only: also time the seeded pool of synthetic contractions")
     ap.add_argument("--paper-pool", action="store_true",
                     help="with --kernel-only: the paper's 48 contractions (Table III extents) and its Fig. 11 sweep")
+    ap.add_argument("--ttgt", action="store_true",
+                    help="pool runs: also time Transpose-Transpose-GEMM-Transpose (torch transpositions + this "
+                         "library's plain GEMM) and report GETT's speedup over it")
+    ap.add_argument("--search", type=int, default=0,
+                    help="pool runs: make every plan with opts.search = k (model ranking, k best timed)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end, equal-GEMM and CPU legs (profiling runs)")
     ap.add_argument("--all", action="store_true", help="with --kernel-only: also time every workload")
@@ -797,6 +902,8 @@ def main():
     ap.add_argument("--ref-macs", type=float, default=5.0e8,
                     help="multiply-adds in the oracle's bounded sample")
     args = ap.parse_args()
+    global SEARCH
+    SEARCH = args.search
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

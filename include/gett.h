@@ -126,7 +126,14 @@ typedef struct {
                               the tensor-core kernel when both operands are gathered (its TMA
                               loaders keep the default); meant for tests of the give-up path.   */
     int32_t experiment; /* ignored, except by builds made with -DGETT_EXPERIMENT (timing probes) */
-    int32_t reserved[6];
+    int32_t search;   /* 0 = the planner's rules decide (default).  k >= 1: enumerate the candidate
+                         plans (tile height and width, epilogue, loaders, operand exchange, split-K:
+                         Sec. 3.3), rank them with the performance model (Sec. 3.4, Eq. 12-14,
+                         re-parameterised for this GPU) and take the model's best (k == 1) or time
+                         the k best and the rule-based plan on the device (cold L2, scratch operands
+                         allocated for the purpose) and take the fastest (Sec. 7.3).  The choice is remembered per process
+                         for equal descriptors, dtype, options and device.                      */
+    int32_t reserved[5];
 } gett_plan_opts_t;
 
 /* What the planner decided (Sec. 3.2.1: index sets, fused sizes, blocking). */
@@ -149,7 +156,13 @@ typedef struct {
     int32_t swapped;                  /* 1: the kernel runs with the operands exchanged (its rows
                                          run over I_n, its columns over I_m; tile_m and tile_n are
                                          the kernel's).  Everything else here is the caller's view. */
-    int32_t reserved[6];
+    int32_t candidates;               /* opts.search > 0: candidate plans enumerated (0 when the choice
+                                         was remembered from an earlier search), else 0             */
+    int32_t model_rank;               /* position of this plan in the model's ranking (0 = its best) */
+    int32_t timed;                    /* candidates that were timed on the device                  */
+    float model_us;                   /* the performance model's estimate for this plan            */
+    float timed_us;                   /* measured time of this plan during the search, else 0      */
+    int32_t reserved[1];
 } gett_plan_info_t;
 
 typedef enum {
@@ -167,7 +180,11 @@ typedef enum {
  * choose the order in which each set is fused so that the stride-1 modes of A,
  * B and C stay inside a tile (Sec. 3.2.1), and pick kernel, blocking and split-K.
  *   out    : receives the plan (host pointer to host pointer).  Untouched on error.
- *   A,B,C  : host descriptors; copied.  C's modes must not overlap in memory.
+ *   A,B,C  : host descriptors; copied.  C's modes must not overlap in memory, and the
+ *            library recognises that only for NESTED layouts: sorted by stride, every mode of
+ *            extent > 1 must step over the whole extent of the previous one (stride_j >=
+ *            stride_i * extent_i).  Packed and padded layouts are nested; an interleaved
+ *            layout that is overlap-free without being nested is rejected (INVALID_ARG).
  *   dtype  : gett_dtype_t.
  *   opts   : host pointer or NULL for automatic choices.
  * The plan is bound to the CUDA device current at the call; its split-K
@@ -269,6 +286,14 @@ GETT_API gett_status_t gett_contract_noalloc(const gett_tensor_desc_t* A, const 
                                     int32_t split_k, float alpha, const void* A_data,
                                     const void* B_data, float beta, void* C_data,
                                     void* cuda_stream);
+
+/*
+ * gett_plan_model -- the performance model's estimate for a plan (Sec. 3.4: Time = Time_macro +
+ * Time_A + Time_B + Time_C, Eq. 12-14, with this GPU's rates and with the loads overlapping the
+ * macro-kernel).  terms_us: host array of 4 doubles or NULL; receives the four terms in
+ * microseconds for the whole job.  total_us: host pointer, receives the estimate.
+ */
+GETT_API gett_status_t gett_plan_model(const gett_plan_t* plan, double* total_us, double* terms_us);
 
 /* Human-readable name of a status; never NULL. */
 GETT_API const char* gett_status_string(gett_status_t status);

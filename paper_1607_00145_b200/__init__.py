@@ -3,7 +3,7 @@ over libgett_b200.so.  Every step of the contraction runs in the CUDA library;
 this package only marshals arguments.  There is no CPU fallback: importing
 `binding` raises if the shared library has not been built."""
 from .binding import (GettError, Plan, gett_contract, gett_plan_create, gett_plan_destroy,  # noqa: F401
-                      gett_plan_get_info, gett_plan_get_table, gett_plan_last_device_status,
+                      gett_plan_get_info, gett_plan_get_table, gett_plan_last_device_status, gett_plan_model,
                       gett_status_string, library_path, PlanOpts, PlanInfo,
                       gett_contract_noalloc, GETT_NOALLOC_WORKSPACE_BYTES)
 from .binding import (GETT_F32, GETT_BF16_F32, GETT_F16_F32, GETT_PATH_AUTO, GETT_PATH_SIMT,  # noqa: F401

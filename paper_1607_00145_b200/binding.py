@@ -36,7 +36,7 @@ class PlanOpts(ctypes.Structure):
                 ("tile_k", ctypes.c_int32), ("stages", ctypes.c_int32), ("split_k", ctypes.c_int32),
                 ("epilogue", ctypes.c_int32), ("flags", ctypes.c_int32),
                 ("wait_limit_us", ctypes.c_int32), ("experiment", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 6)]
+                ("search", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -56,7 +56,9 @@ class PlanInfo(ctypes.Structure):
                 ("digits_k", ctypes.c_int32),
                 ("workspace_bytes", ctypes.c_int64), ("tiles", ctypes.c_int64),
                 ("device", ctypes.c_int32), ("swapped", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 6)]
+                ("candidates", ctypes.c_int32), ("model_rank", ctypes.c_int32), ("timed", ctypes.c_int32),
+                ("model_us", ctypes.c_float), ("timed_us", ctypes.c_float),
+                ("reserved", ctypes.c_int32 * 1)]
 
     def as_dict(self) -> Dict[str, object]:
         out = {}
@@ -99,6 +101,8 @@ def _load() -> ctypes.CDLL:
     lib.gett_contract_noalloc.argtypes = [dp2, dp2, dp2, ctypes.c_int, ctypes.c_int32, ctypes.c_float,
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float,
                                           ctypes.c_void_p, ctypes.c_void_p]
+    lib.gett_plan_model.restype = ctypes.c_int
+    lib.gett_plan_model.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     lib.gett_status_string.restype = ctypes.c_char_p
     lib.gett_status_string.argtypes = [ctypes.c_int]
     return lib
@@ -216,6 +220,16 @@ def gett_plan_get_table(plan: int, which: int) -> np.ndarray:
     return dst
 
 
+def gett_plan_model(plan: int):
+    """(total_us, [macro, A, B, C] in us): the performance model's estimate for the plan."""
+    total = ctypes.c_double()
+    terms = (ctypes.c_double * 4)()
+    rc = _lib.gett_plan_model(plan, ctypes.byref(total), terms)
+    if rc:
+        raise GettError(rc, "gett_plan_model")
+    return float(total.value), [float(x) for x in terms]
+
+
 def gett_plan_last_device_status(plan: int) -> int:
     return int(_lib.gett_plan_last_device_status(plan))
 
@@ -242,6 +256,9 @@ class Plan:
 
     def device_status(self) -> int:
         return gett_plan_last_device_status(self.handle)
+
+    def model(self):
+        return gett_plan_model(self.handle)
 
     def close(self) -> None:
         gett_plan_destroy(self.handle)

@@ -5,10 +5,14 @@
 #include <cuda_runtime.h>
 #include <dlfcn.h>
 
+#include <algorithm>
 #include <cstring>
+#include <map>
+#include <mutex>
 #include <new>
 #include <string>
 #include <utility>
+#include <vector>
 
 #include "kernels.h"
 
@@ -125,6 +129,191 @@ int vec_kind(int loader) // the staging layout behind a loader value
     return loader == GETT_LOAD_TMA_FREE ? GETT_LOAD_VEC_FREE : loader == GETT_LOAD_TMA_K ? GETT_LOAD_VEC_K : loader;
 }
 
+// One plan from one set of overrides: host planning, then the device-side status word and workspace.
+gett_status_t create_one(gett_plan_t** out, const gett_tensor_desc_t* A, const gett_tensor_desc_t* B,
+                         const gett_tensor_desc_t* C, gett_dtype_t dtype, const gett_plan_opts_t* opts)
+{
+    gett_plan* p = new (std::nothrow) gett_plan();
+    if (!p)
+        return GETT_ERR_ALLOC;
+    p->ws = nullptr;
+    p->status = nullptr;
+    int device = -1;
+    const int sms = current_device_sm_count(&device);
+    gett_status_t rc = gett_planner_build(p, A, B, C, dtype, opts, sms > 0 ? sms : 148);
+    if (rc != GETT_OK) {
+        delete p;
+        return rc;
+    }
+    p->info.device = device;
+    p->sm_count = sms > 0 ? sms : 148;
+    p->info.model_us = (float)gett_planner_model(p, p->sm_count, nullptr);
+    if (device >= 0) {
+        if (cudaMalloc(&p->status, sizeof(int32_t)) != cudaSuccess ||
+            cudaMemset(p->status, 0, sizeof(int32_t)) != cudaSuccess) {
+            cudaGetLastError();
+            gett_plan_destroy(p);
+            return GETT_ERR_ALLOC;
+        }
+        if (p->info.workspace_bytes > 0 &&
+            cudaMalloc(&p->ws, (size_t)p->info.workspace_bytes) != cudaSuccess) {
+            cudaGetLastError();
+            gett_plan_destroy(p);
+            return GETT_ERR_ALLOC;
+        }
+    }
+    *out = p;
+    return GETT_OK;
+}
+
+// ---- plan search (Sec. 3.3, 3.4, 7.3): candidates, model ranking, timed top-k, cache ----
+std::mutex g_cache_mutex;
+std::map<std::string, gett_plan_opts_t> g_plan_cache; // key: descriptors, dtype, caller's options, device
+
+std::string cache_key(const gett_tensor_desc_t* A, const gett_tensor_desc_t* B, const gett_tensor_desc_t* C, int dtype,
+                      const gett_plan_opts_t& o, int device)
+{
+    std::string k;
+    auto put = [&](const void* p, size_t n) { k.append(static_cast<const char*>(p), n); };
+    for (const gett_tensor_desc_t* t : {A, B, C}) {
+        put(&t->nmodes, sizeof t->nmodes);
+        for (int i = 0; i < t->nmodes; ++i) {
+            put(&t->extent[i], sizeof(int64_t));
+            put(&t->label[i], sizeof(int32_t));
+            const int64_t st = t->stride ? t->stride[i] : -1;
+            put(&st, sizeof st);
+        }
+    }
+    put(&dtype, sizeof dtype);
+    put(&o, sizeof o);
+    put(&device, sizeof device);
+    return k;
+}
+
+size_t span_elems(const gett_tensor_desc_t* t)
+{
+    size_t span = 1, packed = 1;
+    for (int i = 0; i < t->nmodes; ++i) {
+        const size_t st = t->stride ? (size_t)t->stride[i] : packed;
+        span += (size_t)(t->extent[i] - 1) * st;
+        packed *= (size_t)t->extent[i];
+    }
+    return span;
+}
+
+gett_status_t create_by_search(gett_plan_t** out, const gett_tensor_desc_t* A, const gett_tensor_desc_t* B,
+                               const gett_tensor_desc_t* C, gett_dtype_t dtype, const gett_plan_opts_t& asked)
+{
+    int device = -1;
+    const int sms = current_device_sm_count(&device);
+    if (A->nmodes < 0 || B->nmodes < 0 || C->nmodes < 0 || A->nmodes > GETT_MAX_MODES || B->nmodes > GETT_MAX_MODES ||
+        C->nmodes > GETT_MAX_MODES)
+        return GETT_ERR_INVALID_ARG;
+    const std::string key = cache_key(A, B, C, dtype, asked, device);
+    {
+        std::lock_guard<std::mutex> lock(g_cache_mutex);
+        auto it = g_plan_cache.find(key);
+        if (it != g_plan_cache.end()) {
+            gett_plan_opts_t o = it->second;
+            return create_one(out, A, B, C, dtype, &o);
+        }
+    }
+    gett_plan_opts_t base = asked;
+    base.search = 0;
+    const std::vector<gett_plan_opts_t> cand = gett_planner_candidates(A, B, C, dtype, base, sms > 0 ? sms : 148);
+    if (cand.empty()) // not even the rule-based plan exists: report why
+        return create_one(out, A, B, C, dtype, &base);
+    // rank by the model
+    struct Ranked {
+        gett_plan_opts_t o;
+        double model_us;
+        float timed_us;
+        bool rule_based; // the plan the planner's rules give (always timed: the search must not lose to it)
+    };
+    std::vector<Ranked> r;
+    for (size_t i = 0; i < cand.size(); ++i) {
+        gett_plan tmp;
+        tmp.ws = nullptr;
+        tmp.status = nullptr;
+        if (gett_planner_build(&tmp, A, B, C, dtype, &cand[i], sms > 0 ? sms : 148) == GETT_OK)
+            r.push_back({cand[i], gett_planner_model(&tmp, sms > 0 ? sms : 148, nullptr), 0.f, i == 0});
+    }
+    std::stable_sort(r.begin(), r.end(), [](const Ranked& x, const Ranked& y) { return x.model_us < y.model_us; });
+    size_t best = 0;
+    int timed = 0;
+    if (asked.search > 1 && device >= 0) {
+        // time the k best on scratch operands (zeros: finite, and the kernels do not look at values)
+        const size_t es = dtype == GETT_F32 ? 4 : 2;
+        void *dA = nullptr, *dB = nullptr, *dC = nullptr, *dFlush = nullptr;
+        const size_t flush_bytes = 192u << 20; // larger than L2: every timed launch starts cold
+        cudaStream_t st = nullptr;
+        cudaEvent_t e0 = nullptr, e1 = nullptr;
+        const size_t nA = span_elems(A) * es, nB = span_elems(B) * es, nC = span_elems(C) * 4;
+        bool ok = cudaMalloc(&dA, nA) == cudaSuccess && cudaMalloc(&dB, nB) == cudaSuccess &&
+                  cudaMalloc(&dC, nC) == cudaSuccess && cudaMalloc(&dFlush, flush_bytes) == cudaSuccess &&
+                  cudaMemset(dA, 0, nA) == cudaSuccess &&
+                  cudaMemset(dB, 0, nB) == cudaSuccess && cudaMemset(dC, 0, nC) == cudaSuccess &&
+                  cudaStreamCreate(&st) == cudaSuccess && cudaEventCreate(&e0) == cudaSuccess &&
+                  cudaEventCreate(&e1) == cudaSuccess;
+        float best_ms = 0.f;
+        for (size_t i = 0; ok && i < r.size(); ++i) {
+            if (i >= (size_t)asked.search && !r[i].rule_based)
+                continue;
+            gett_plan_t* p = nullptr;
+            if (create_one(&p, A, B, C, dtype, &r[i].o) != GETT_OK)
+                continue;
+            float ms_min = 0.f;
+            bool good = gett_contract(p, 1.f, dA, dB, 0.f, dC, st) == GETT_OK; // warm-up
+            for (int rep = 0; good && rep < 3; ++rep) {
+                cudaMemsetAsync(dFlush, rep, flush_bytes, st);
+                cudaEventRecord(e0, st);
+                good = gett_contract(p, 1.f, dA, dB, 0.f, dC, st) == GETT_OK;
+                cudaEventRecord(e1, st);
+                if (cudaEventSynchronize(e1) != cudaSuccess)
+                    good = false;
+                float ms = 0.f;
+                if (good && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess)
+                    ms_min = rep == 0 ? ms : std::min(ms_min, ms);
+            }
+            good = good && gett_plan_last_device_status(p) == GETT_OK;
+            gett_plan_destroy(p);
+            if (!good)
+                continue;
+            r[i].timed_us = ms_min * 1e3f;
+            ++timed;
+            // (another candidate has to beat the rule-based plan by 3 % to replace it)
+            const float handicap = r[i].rule_based ? 0.97f : 1.f;
+            if (timed == 1 || ms_min * handicap < best_ms) {
+                best_ms = ms_min * handicap;
+                best = i;
+            }
+        }
+        cudaGetLastError();
+        if (e0)
+            cudaEventDestroy(e0);
+        if (e1)
+            cudaEventDestroy(e1);
+        if (st)
+            cudaStreamDestroy(st);
+        cudaFree(dA);
+        cudaFree(dB);
+        cudaFree(dC);
+        cudaFree(dFlush);
+        if (timed == 0)
+            best = 0;
+    }
+    gett_status_t rc = create_one(out, A, B, C, dtype, &r[best].o);
+    if (rc != GETT_OK)
+        return rc;
+    (*out)->info.candidates = (int32_t)r.size();
+    (*out)->info.model_rank = (int32_t)best;
+    (*out)->info.timed = timed;
+    (*out)->info.timed_us = r[best].timed_us;
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    g_plan_cache[key] = r[best].o;
+    return GETT_OK;
+}
+
 } // namespace
 
 extern "C" {
@@ -142,35 +331,18 @@ gett_status_t gett_plan_create(gett_plan_t** out, const gett_tensor_desc_t* A,
 {
     if (!out || !A || !B || !C)
         return GETT_ERR_INVALID_ARG;
-    gett_plan* p = new (std::nothrow) gett_plan();
-    if (!p)
-        return GETT_ERR_ALLOC;
-    p->ws = nullptr;
-    p->status = nullptr;
-    int device = -1;
-    const int sms = current_device_sm_count(&device);
-    gett_status_t rc = gett_planner_build(p, A, B, C, dtype, opts, sms > 0 ? sms : 148);
-    if (rc != GETT_OK) {
-        delete p;
-        return rc;
-    }
-    p->info.device = device;
-    p->sm_count = sms > 0 ? sms : 148;
-    if (device >= 0) {
-        if (cudaMalloc(&p->status, sizeof(int32_t)) != cudaSuccess ||
-            cudaMemset(p->status, 0, sizeof(int32_t)) != cudaSuccess) {
-            cudaGetLastError();
-            gett_plan_destroy(p);
-            return GETT_ERR_ALLOC;
-        }
-        if (p->info.workspace_bytes > 0 &&
-            cudaMalloc(&p->ws, (size_t)p->info.workspace_bytes) != cudaSuccess) {
-            cudaGetLastError();
-            gett_plan_destroy(p);
-            return GETT_ERR_ALLOC;
-        }
-    }
-    *out = p;
+    if (opts && opts->search < 0)
+        return GETT_ERR_INVALID_ARG;
+    if (opts && opts->search > 0)
+        return create_by_search(out, A, B, C, dtype, *opts);
+    return create_one(out, A, B, C, dtype, opts);
+}
+
+gett_status_t gett_plan_model(const gett_plan_t* plan, double* total_us, double* terms_us)
+{
+    if (!plan || !total_us)
+        return GETT_ERR_INVALID_ARG;
+    *total_us = gett_planner_model(plan, plan->sm_count, terms_us);
     return GETT_OK;
 }
 

@@ -134,6 +134,12 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* A,
                                  gett_dtype_t dtype, const gett_plan_opts_t* opts, int sm_count);
 gett_status_t gett_planner_table(const gett_plan* p, int which, int64_t* dst, size_t capacity);
 
+// Candidate enumeration and the performance model (search.cpp).
+double gett_planner_model(const gett_plan* p, int sm_count, double terms[4]);
+std::vector<gett_plan_opts_t> gett_planner_candidates(const gett_tensor_desc_t* A, const gett_tensor_desc_t* B,
+                                                     const gett_tensor_desc_t* C, gett_dtype_t dtype,
+                                                     const gett_plan_opts_t& base, int sm_count);
+
 // Geometry of the tensor-core kernel (kernel_umma.cu), needed by the planner.
 int gett_umma_smem_bytes(int tile_m, int tile_n, int stages, int staged_cv, int lean); // staged_cv: 0, 1 or 8
 int gett_umma_max_stages(int tile_m, int tile_n, int smem_limit, int staged_cv, int lean);
