@@ -107,7 +107,12 @@ typedef enum {
     GETT_OPT_NO_TMA = 1,      /* gather with 16-byte copies even where tensor-map (TMA) boxes apply  */
     GETT_OPT_NO_PAIR = 2,     /* never launch the CTA-pair variant of the tensor-core kernel         */
     GETT_OPT_NO_EXCHANGE = 4, /* never exchange the roles of A and B                                 */
-    GETT_OPT_NO_ATOMS = 8     /* no re-ordering of I_m, I_n, I_k into 64 x 64 atoms that are boxes   */
+    GETT_OPT_NO_ATOMS = 8,    /* no re-ordering of I_m, I_n, I_k into 64 x 64 atoms that are boxes   */
+    GETT_OPT_STREAMK = 16,    /* tensor-core kernel: cut the tiles that are left over after whole rounds
+                                 (one tile per SM) along K wherever that is possible (more tiles than
+                                 SMs, direct epilogue, no K slices), not only when the last round of
+                                 tiles would be mostly empty                                          */
+    GETT_OPT_NO_STREAMK = 32  /* ... never                                                           */
 } gett_opt_flags_t;
 
 /* Planner overrides; zero-initialise for "auto".  Unsupported combinations make
@@ -162,7 +167,8 @@ typedef struct {
     int32_t timed;                    /* candidates that were timed on the device                  */
     float model_us;                   /* the performance model's estimate for this plan            */
     float timed_us;                   /* measured time of this plan during the search, else 0      */
-    int32_t reserved[1];
+    int32_t stream_k;                 /* 1: the tiles left over after whole rounds are cut along K and shared
+                                         by all SMs (stream-K); workspace_bytes holds their pieces    */
 } gett_plan_info_t;
 
 typedef enum {

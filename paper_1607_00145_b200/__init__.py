@@ -11,4 +11,5 @@ from .binding import (GETT_F32, GETT_BF16_F32, GETT_F16_F32, GETT_PATH_AUTO, GET
                       GETT_EPI_STAGED, GETT_LOAD_SCALAR, GETT_LOAD_VEC_FREE, GETT_LOAD_VEC_K,
                       GETT_LOAD_TMA_FREE, GETT_LOAD_TMA_K, GETT_LOAD_VEC_KT,
                       GETT_OPT_NO_TMA, GETT_OPT_NO_PAIR, GETT_OPT_NO_EXCHANGE, GETT_OPT_NO_ATOMS,
+                      GETT_OPT_STREAMK, GETT_OPT_NO_STREAMK,
                       TABLE_NAMES)

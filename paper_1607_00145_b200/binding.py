@@ -14,6 +14,7 @@ GETT_LOAD_SCALAR, GETT_LOAD_VEC_FREE, GETT_LOAD_VEC_K = 0, 1, 2
 GETT_LOAD_TMA_FREE, GETT_LOAD_TMA_K, GETT_LOAD_VEC_KT = 3, 4, 5
 GETT_EPI_AUTO, GETT_EPI_DIRECT, GETT_EPI_STAGED = 0, 1, 2
 GETT_OPT_NO_TMA, GETT_OPT_NO_PAIR, GETT_OPT_NO_EXCHANGE, GETT_OPT_NO_ATOMS = 1, 2, 4, 8
+GETT_OPT_STREAMK, GETT_OPT_NO_STREAMK = 16, 32
 TABLE_NAMES = ("A_M", "A_K", "B_N", "B_K", "C_M", "C_N")
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -58,7 +59,7 @@ class PlanInfo(ctypes.Structure):
                 ("device", ctypes.c_int32), ("swapped", ctypes.c_int32),
                 ("candidates", ctypes.c_int32), ("model_rank", ctypes.c_int32), ("timed", ctypes.c_int32),
                 ("model_us", ctypes.c_float), ("timed_us", ctypes.c_float),
-                ("reserved", ctypes.c_int32 * 1)]
+                ("stream_k", ctypes.c_int32)]
 
     def as_dict(self) -> Dict[str, object]:
         out = {}

@@ -415,6 +415,11 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     args.c_vec = plan->c_vec;
     args.prod_groups = plan->info.path == GETT_PATH_UMMA ? gett_umma_prod_groups(plan->info.stages) : 0;
     args.epi_lean = plan->epi_lean;
+    args.stream_k = plan->stream_k;
+    args.sk_full = plan->sk_full;
+    args.sk_units = plan->sk_units;
+    args.sk_slabs = plan->sk_slabs;
+    args.sk_pmax = plan->sk_pmax;
 #ifdef GETT_EXPERIMENT
     if (plan->debug & 2048) // probe: all producer warps as one wide group
         args.prod_groups = 1;
@@ -428,6 +433,7 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     cudaError_t err = cudaSuccess;
     switch (path) {
     case GETT_PATH_SIMT: {
+        args.stream_k = 0; // (only reached as the fall-back for unaligned bases: the plan's slices are kept)
         args.tiles_m = (plan->M.size + 63) / 64;
         args.tiles_n = (plan->N.size + 63) / 64;
         const uint64_t grid = (uint64_t)args.tiles_m * args.tiles_n * args.split_k;
@@ -465,6 +471,8 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
     }
     if (err == cudaSuccess && args.split_k > 1)
         err = gett_launch_splitk_reduce(args, plan->sm_count, stream);
+    if (err == cudaSuccess && path == GETT_PATH_UMMA && args.stream_k)
+        err = gett_launch_streamk_fixup(args, plan->info.grid, stream);
     return err == cudaSuccess ? GETT_OK : GETT_ERR_CUDA;
 }
 

@@ -63,6 +63,11 @@ struct GettKernelArgs {
     uint32_t wait_limit_us; // bound of every device-side wait on a barrier
     int32_t prod_groups;  // producer groups the tensor-core kernel uses (divides stages)
     int32_t epi_lean;     // staged epilogue of the tensor-core kernel with one narrow staging buffer per warp
+    uint32_t stream_k;    // tensor-core kernel: the tiles left over after whole rounds are cut along K (see item_count())
+    uint32_t sk_full;     // ... whole rounds of tiles (one tile per CTA and round)
+    uint32_t sk_units;    // ... slab units of the left-over tiles per CTA
+    uint32_t sk_slabs;    // ... slabs per tile
+    uint32_t sk_pmax;     // ... pieces per left-over tile, at most (workspace: [tile][piece][tile_n][tile_m])
 };
 
 // How the coordinates of a TMA box follow from fused indices: digit d of the operand's free
@@ -116,6 +121,7 @@ struct gett_plan {
     int32_t skinny; // fp32: B resident in shared memory, A streamed (small N and K)
     int32_t epi_lean; // see GettKernelArgs
     int32_t pair_ok;  // the CTA-pair variant of the tensor-core kernel applies (used if its library is there)
+    uint32_t stream_k, sk_full, sk_units, sk_slabs, sk_pmax; // see GettKernelArgs
     int32_t swapped;  // the kernels get the caller's B as their A and vice versa (im / in / ik, tm / tn / tk,
                       // M / N / K and the loaders below are the kernels' view; info is the caller's)
     GettTmaRecipe tma_a, tma_b;

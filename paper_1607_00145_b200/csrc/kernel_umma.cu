@@ -25,6 +25,7 @@
 // memory and returns.
 #include "kernels.h"
 #include "ptx_sm100.cuh"
+#include "umma_raster.h"
 
 // The file is compiled a second time, with GETT_UMMA_CLUSTER defined, by the source that adds
 // the CTA-pair variant (two CTAs of a cluster work on two neighbouring tile columns of one
@@ -64,7 +65,6 @@ constexpr int MAX_STAGES = 8;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t ATOM_BYTES = 1024;      // 8 rows x 128 B
 constexpr uint32_t MN_BLOCK_BYTES = 8192;  // one 64-wide block of an MN-major operand: 64 k rows
-constexpr int RASTER_M = 16;               // tile rows per rasterisation panel
 constexpr int EPI_PITCH = 68;              // floats per staged row: 64 + 4 keeps 128-bit accesses conflict-free
 constexpr int EPI_GROUPS = 256 / 4;          // 16-byte groups per tile row, at most
 constexpr int EPI_DEPTH = 2;                 // staging buffers per warp: old C is fetched EPI_DEPTH-1 chunks ahead
@@ -105,37 +105,84 @@ __host__ __device__ constexpr uint32_t stage_bytes(uint32_t tile_m, uint32_t til
 
 struct WorkItem {
     uint32_t m0, n0, z, kbeg, kend, nslab;
+    uint32_t r;   // stream-K: number of the left-over tile the item is a piece of
+    bool partial; // the item's sums go to the workspace (a K slice, or a piece of a tile), not to C
 };
+
+// Origin of output tile (or, in the CTA-pair build, tile pair) number t.
+__device__ __forceinline__ void tile_origin(const GettKernelArgs& g, uint32_t t, uint32_t tile_m, uint32_t& m0,
+                                            uint32_t& n0)
+{
+    uint32_t tm, tn;
+#ifdef GETT_UMMA_CLUSTER
+    gett_raster_tile(t, g.tiles_m, g.tiles_n >> 1, tm, tn); // columns of tile pairs
+    n0 = (2 * tn + GETT_WRANK) * (uint32_t)g.tile_n;
+#else
+    gett_raster_tile(t, g.tiles_m, g.tiles_n, tm, tn);
+    n0 = tn * (uint32_t)g.tile_n;
+#endif
+    m0 = tm * tile_m;
+}
 
 __device__ __forceinline__ WorkItem decode_work(const GettKernelArgs& g, uint32_t w, uint32_t tile_m)
 {
 #ifdef GETT_UMMA_CLUSTER
-    const uint32_t tiles_n = g.tiles_n >> 1; // columns of tile pairs
+    const uint32_t tiles = g.tiles_m * (g.tiles_n >> 1);
 #else
-    const uint32_t tiles_n = g.tiles_n;
+    const uint32_t tiles = g.tiles_m * g.tiles_n;
 #endif
-    const uint32_t tiles = g.tiles_m * tiles_n;
     WorkItem it;
     it.z = w / tiles;
-    const uint32_t t = w - it.z * tiles;
-    // Tiles are numbered panel by panel: a panel is RASTER_M tile rows high and spans all
-    // tile columns, and inside it the row index runs fastest.  The ~148 tiles in flight at
-    // any time then share few distinct rows of A and columns of B, which keeps them in L2.
-    const uint32_t per_panel = RASTER_M * tiles_n;
-    const uint32_t panel = t / per_panel;
-    const uint32_t first_m = panel * RASTER_M;
-    const uint32_t rows = min((uint32_t)RASTER_M, g.tiles_m - first_m);
-    const uint32_t in_panel = t - panel * per_panel;
-    const uint32_t tn = in_panel / rows;
-    it.m0 = (first_m + (in_panel - tn * rows)) * tile_m;
-#ifdef GETT_UMMA_CLUSTER
-    it.n0 = (2 * tn + GETT_WRANK) * (uint32_t)g.tile_n;
-#else
-    it.n0 = tn * (uint32_t)g.tile_n;
-#endif
+    tile_origin(g, w - it.z * tiles, tile_m, it.m0, it.n0);
     it.kbeg = it.z * g.k_per_split;
     it.kend = min(g.K.size, it.kbeg + g.k_per_split);
     it.nslab = (it.kend - it.kbeg + TILE_K - 1) / TILE_K;
+    it.partial = g.split_k > 1;
+    return it;
+}
+
+// The CTA's work list.  Ordinarily the (tile, K slice) pairs number WB, WB + WG, ... of
+// `total_work`.  With stream-K (Sec. 2.1 / Sec. 3.3: choosing how the three loops are cut; here
+// the cut that leaves no SM idle in a last partial wave) the first sk_full rounds of tiles are
+// dealt out the same way, and the tiles that are left (fewer than there are CTAs) are cut along
+// K: their tiles x slabs space is one sequence of slab units of which every CTA takes
+// sk_units consecutive ones.  Such an item is a piece of one tile; its sums go to the
+// workspace as piece number z of that tile, and a second kernel adds the pieces.
+__device__ __forceinline__ uint32_t item_count(const GettKernelArgs& g, uint32_t total_work)
+{
+    if (g.stream_k) {
+        const uint32_t tiles = g.tiles_m * g.tiles_n;
+        const uint32_t total = (tiles - g.sk_full * GETT_WG) * g.sk_slabs; // slab units of the left-over tiles
+        const uint32_t beg = GETT_WB * g.sk_units;
+        if (beg >= total)
+            return g.sk_full;
+        const uint32_t end = min(total, beg + g.sk_units);
+        return g.sk_full + (end - 1) / g.sk_slabs - beg / g.sk_slabs + 1;
+    }
+    return total_work > GETT_WB ? (total_work - GETT_WB + GETT_WG - 1) / GETT_WG : 0;
+}
+
+__device__ __forceinline__ WorkItem decode_item(const GettKernelArgs& g, uint32_t i, uint32_t tile_m)
+{
+    if (!g.stream_k || i < g.sk_full) {
+        WorkItem it = decode_work(g, GETT_WB + i * GETT_WG, tile_m);
+        it.r = 0;
+        return it;
+    }
+    const uint32_t S = g.sk_slabs, W = g.sk_units;
+    const uint32_t tiles = g.tiles_m * g.tiles_n, done = g.sk_full * GETT_WG;
+    const uint32_t total = (tiles - done) * S;
+    const uint32_t beg = GETT_WB * W, end = min(total, beg + W);
+    const uint32_t r = beg / S + (i - g.sk_full); // which of the left-over tiles
+    const uint32_t ub = max(beg, r * S), ue = min(end, (r + 1) * S);
+    WorkItem it;
+    tile_origin(g, done + r, tile_m, it.m0, it.n0);
+    it.r = r;
+    it.z = GETT_WB - (r * S) / W; // pieces of a tile are numbered from the first CTA that touches it
+    it.kbeg = (ub - r * S) * TILE_K;
+    it.kend = min(g.K.size, (ue - r * S) * TILE_K);
+    it.nslab = ue - ub;
+    it.partial = true; // (even a whole left-over tile goes through the workspace: the fix-up treats all alike)
     return it;
 }
 
@@ -609,8 +656,9 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
     };
     uint32_t first = 0; // slab number of the current work item's first slab
     bool alive = true;
-    for (uint32_t w = GETT_WB; w < total_work && pg < ng; w += GETT_WG) {
-        const WorkItem wi = decode_work(g, w, TILE_M);
+    const uint32_t nitems = item_count(g, total_work);
+    for (uint32_t wn = 0; wn < nitems && pg < ng; ++wn) {
+        const WorkItem wi = decode_item(g, wn, TILE_M);
         // my group's first slab in this item: smallest j with (first + j) % ng == pg
         uint32_t j = (pg + ng - first % ng) % ng;
         if (j < wi.nslab) {
@@ -868,8 +916,9 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
             const uint32_t lbo = MN_BLOCK_BYTES, sbo = ATOM_BYTES;
             uint32_t it = 0, local = 0;
             bool alive = true;
-            for (uint32_t w = GETT_WB; w < total_work && alive; w += GETT_WG, ++local) {
-                const WorkItem wi = decode_work(g, w, TILE_M);
+            const uint32_t nitems = item_count(g, total_work);
+            for (; local < nitems && alive; ++local) {
+                const WorkItem wi = decode_item(g, local, TILE_M);
                 // 128-row tiles alternate between the two accumulator buffers; a 256-row tile
                 // uses both (rows 0-127 in buffer 0, rows 128-255 in buffer 1)
                 const uint32_t buf = TWO_HALVES ? 0u : (local & 1);
@@ -950,10 +999,9 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
         uint32_t j = 0; // counts this set's tiles
         // 128-row tiles: set es takes every other tile.  256-row tiles: both sets work on
         // every tile, set es on its rows 128 es .. 128 es + 127.
-        const uint32_t w_first = GETT_WB + (TWO_HALVES ? 0u : es * GETT_WG);
-        const uint32_t w_step = (TWO_HALVES ? 1u : 2u) * GETT_WG;
-        for (uint32_t w = w_first; w < total_work && !staged; w += w_step, ++j) {
-            WorkItem wi = decode_work(g, w, TILE_M);
+        const uint32_t nitems = item_count(g, total_work);
+        for (uint32_t wn = TWO_HALVES ? 0u : es; wn < nitems && !staged; wn += TWO_HALVES ? 1u : 2u, ++j) {
+            WorkItem wi = decode_item(g, wn, TILE_M);
             if (TWO_HALVES)
                 wi.m0 += es * MMA_M;
             const uint32_t buf = es;
@@ -983,7 +1031,14 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                 ptx::tmem_wait_ld();
                 if (!row_ok || GETT_DBG(g, 2)) // (debug & 2: experiment switch, no stores)
                     continue;
-                if (g.split_k > 1) {
+                if (wi.partial && g.stream_k) {
+                    // piece z of left-over tile r: a whole tile_m x TILE_N buffer [column][row]
+                    float* dst = g.ws + (((size_t)wi.r * g.sk_pmax + wi.z) * TILE_N + c0) * (size_t)g.tile_m +
+                                 (TWO_HALVES ? es * MMA_M : 0u) + et;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        dst[(size_t)i * g.tile_m] = __uint_as_float(v[i]);
+                } else if (wi.partial) {
                     float* dst = g.ws + ((size_t)wi.z * g.N.size + wi.n0 + c0) * g.M.size + wi.m0 + et;
 #pragma unroll
                     for (int i = 0; i < 16; ++i)

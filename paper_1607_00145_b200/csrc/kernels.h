@@ -11,6 +11,10 @@ cudaError_t gett_launch_simt(const GettKernelArgs& args, int grid, cudaStream_t 
 cudaError_t gett_launch_splitk_reduce(const GettKernelArgs& args, int sm_count,
                                       cudaStream_t stream);
 
+// Stream-K: add the pieces of the left-over tiles (workspace [tile][piece][tile_n][tile_m]) and apply
+// C <- alpha * sum + beta * C.  grid: CTAs of the contraction kernel's launch.
+cudaError_t gett_launch_streamk_fixup(const GettKernelArgs& args, int grid, cudaStream_t stream);
+
 // Tensor-core kernel (16-bit inputs, tcgen05 + tensor memory), persistent grid.
 cudaError_t gett_launch_umma(const GettKernelArgs& args, const GettTmaMaps& maps, int grid, int smem,
                              cudaStream_t stream);

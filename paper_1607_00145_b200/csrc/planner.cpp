@@ -1021,13 +1021,44 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     info.grid = (int32_t)(tiles * split);
     if (path == GETT_PATH_UMMA) // persistent: one CTA per SM walks the work list
         info.grid = (int32_t)std::min<uint64_t>(tiles * split, (uint64_t)sms);
+    // ---- stream-K: no idle SMs in a last partial wave of tiles ----
+    // With more tiles than SMs but a tile count that leaves much of the last wave empty, the
+    // tiles of the whole rounds are dealt out as usual and the left-over tiles are cut along K
+    // (one more way of cutting the three loops, Sec. 2.1 / Sec. 3.3): their tiles x slabs space
+    // is dealt out in equal shares, the pieces go through the workspace and a second kernel adds
+    // them.  Only with the direct epilogue, without K slices.
+    p->stream_k = p->sk_full = p->sk_units = p->sk_slabs = p->sk_pmax = 0;
+    if (path == GETT_PATH_UMMA && split == 1 && info.epilogue == GETT_EPI_DIRECT && !(p->flags & GETT_OPT_NO_STREAMK) &&
+        tiles > (uint64_t)sms && tiles % sms != 0 && kslabs >= 2 && tiles * kslabs < (1ull << 31)) {
+        const uint64_t full = tiles / sms, left = tiles - full * sms;
+        const uint64_t units = (left * kslabs + sms - 1) / sms; // slab units per CTA
+        uint64_t pmax = 1;
+        for (uint64_t r = 0; r < left; ++r)
+            pmax = std::max<uint64_t>(pmax, ((r + 1) * kslabs - 1) / units - (r * kslabs) / units + 1);
+        const int64_t ws_bytes = (int64_t)(left * pmax) * info.tile_m * info.tile_n * 4;
+        // worth it when the time of the SMs that would idle through the last round exceeds what the
+        // pieces cost (their trip through memory and the second launch), with a margin
+        const double slab_us = 2.0 * info.tile_m * info.tile_n * 64 / (1.67e15 / sms) * 1e6 / 0.8; // one SM
+        const double saved_us = (1.0 - (double)left / sms) * kslabs * slab_us;
+        const double cost_us = 2.0 * (double)ws_bytes / 6.5e6 + 10.0;
+        if (((saved_us > 1.5 * cost_us && units >= 4) || (p->flags & GETT_OPT_STREAMK)) && ws_bytes <= (1ll << 30)) {
+            p->stream_k = 1;
+            p->sk_full = (uint32_t)full;
+            p->sk_slabs = kslabs;
+            p->sk_units = (uint32_t)units;
+            p->sk_pmax = (uint32_t)pmax;
+            info.workspace_bytes = ws_bytes;
+            info.grid = sms;
+        }
+    }
+    info.stream_k = (int32_t)p->stream_k;
     if (p->skinny) // persistent: two CTAs per SM stream the row tiles
         info.grid = (int32_t)std::min<uint64_t>(p->tiles_m, 2ull * sms);
     // two neighbouring 256 x 256 tiles per CTA pair, A shared between the two CTAs
     p->pair_ok = path == GETT_PATH_UMMA && p->tma_a.enabled && p->tma_b.enabled && !p->tma_a.hybrid &&
                  !p->tma_b.hybrid && info.tile_m == 256 &&
                  info.tile_n == 256 && info.epilogue == GETT_EPI_DIRECT && split == 1 && p->tiles_n % 2 == 0 &&
-                 !(p->flags & GETT_OPT_NO_PAIR);
+                 !p->stream_k && !(p->flags & GETT_OPT_NO_PAIR);
     info.swapped = p->swapped;
     if (p->swapped) { // report the caller's view
         std::swap(info.M, info.N);

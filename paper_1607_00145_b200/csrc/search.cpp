@@ -69,7 +69,8 @@ double gett_planner_model(const gett_plan* p, int sm_count, double terms[4])
     else if (in.path == GETT_PATH_SIMT)
         ctas_per_sm = 4.0;
     const double slots = sms * ctas_per_sm;
-    const double waves = std::ceil(items / slots);
+    // (stream-K: every SM gets the same share of the tiles x slabs space, no partial last wave)
+    const double waves = p->stream_k ? items / slots : std::ceil(items / slots);
     // per slab of one work item, in clocks of the SM it shares with ctas_per_sm - 1 others
     const double rate = in.path == GETT_PATH_UMMA ? TENSOR_FLOP_PER_CLK
                         : in.path == GETT_PATH_FFMA ? FMA_FLOP_PER_CLK * 0.75 // (fragment loads share the issue slots)
@@ -82,7 +83,9 @@ double gett_planner_model(const gett_plan* p, int sm_count, double terms[4])
     double c_bytes = M * N * 4.0 * 2.0; // written, and read when beta != 0 (the model does not know beta)
     double c_derate = 1.0;
     const bool rows_along_c = p->M.ndig >= 1 && p->M.sY[0] == 1;
-    if (in.split_k > 1) {
+    if (p->stream_k) {
+        c_bytes += 2.0 * 4.0 * (double)p->sk_pmax * std::fmod(items, slots) * tm * tn; // the left-over tiles' pieces, out and back in
+    } else if (in.split_k > 1) {
         c_bytes = M * N * 4.0 * (2.0 * in.split_k + 2.0); // partial sums out and back in, then C
     } else if (in.epilogue == GETT_EPI_STAGED) {
         c_derate = 0.8; // whole runs of C, through shared memory
@@ -120,7 +123,7 @@ std::vector<gett_plan_opts_t> gett_planner_candidates(const gett_tensor_desc_t* 
     auto same = [](const gett_plan_info_t& x, const gett_plan_info_t& y) {
         return x.path == y.path && x.loader_a == y.loader_a && x.loader_b == y.loader_b && x.epilogue == y.epilogue &&
                x.tile_m == y.tile_m && x.tile_n == y.tile_n && x.stages == y.stages && x.split_k == y.split_k &&
-               x.swapped == y.swapped && x.digits_m == y.digits_m && x.digits_n == y.digits_n && x.digits_k == y.digits_k;
+               x.swapped == y.swapped && x.stream_k == y.stream_k && x.digits_m == y.digits_m && x.digits_n == y.digits_n && x.digits_k == y.digits_k;
     };
     auto consider = [&](gett_plan_opts_t o) {
         gett_plan tmp;
@@ -139,7 +142,8 @@ std::vector<gett_plan_opts_t> gett_planner_candidates(const gett_tensor_desc_t* 
     const int tile_ms[] = {0, 64, 128, 256};
     const int tile_ns[] = {0, 32, 64, 128, 192, 256};
     const int epis[] = {GETT_EPI_AUTO, GETT_EPI_DIRECT};
-    const int flagsets[] = {0, GETT_OPT_NO_ATOMS, GETT_OPT_NO_TMA, GETT_OPT_NO_EXCHANGE};
+    const int flagsets[] = {0, GETT_OPT_NO_ATOMS, GETT_OPT_NO_TMA, GETT_OPT_NO_EXCHANGE, GETT_OPT_STREAMK,
+                            GETT_OPT_NO_STREAMK};
     const int splits[] = {0, 1, 2, 4, 8, 16, 32};
     for (int tmv : tile_ms)
         for (int tnv : tile_ns)

@@ -257,6 +257,28 @@ def test_transposing_loader_for_two_different_contracted_stride1_modes(spec, siz
     parity_case(con, BF16_F32, "normal", 61, 1.0, 0.0, path=g.GETT_PATH_SIMT)
 
 
+@pytest.mark.parametrize("spec,sizes,opts", [
+    # 15 x 11 = 165 tiles of 128 x 64 on 148 SMs, 5 slabs (the last one ragged): TMA boxes
+    ("C[m,n] = A[m,k] * B[k,n]", dict(m=1904, n=696, k=296), dict(tile_m=128, tile_n=64)),
+    # gathered operands, 4-D, several modes per dimension
+    ("C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]", dict(m0=24, m1=80, n0=30, n1=24, k0=8, k1=20),
+     dict(tile_m=128, tile_n=64)),
+    # 256-row tiles (both accumulator buffers per tile): 3 x 53 = 159 tiles
+    ("C[m,n] = A[k,m] * B[n,k]", dict(m=600, n=13504, k=200), dict(tile_m=256, tile_n=256)),
+])
+def test_stream_k_shares_of_the_tile_slab_space(spec, sizes, opts):
+    """Stream-K, forced: every CTA takes an equal share of the tiles x slabs space, tiles shared by
+    two CTAs go through the workspace and the fix-up kernel; against the oracle, twice (fixed
+    order of the pieces: bit-reproducible), with and without the old C."""
+    con = parse_spec(spec, sizes)
+    for dtype in (BF16_F32, F16_F32):
+        for alpha, beta in [(1.0, 0.5), (-0.5, 0.0)]:
+            ratio, info = parity_case(con, dtype, "normal", 71, alpha, beta, repeat=2, flags=g.GETT_OPT_STREAMK, **opts)
+            assert info.stream_k == 1 and info.split_k == 1 and info.workspace_bytes > 0
+    ratio, info = parity_case(con, BF16_F32, "normal", 71, 1.0, 0.5, flags=g.GETT_OPT_NO_STREAMK, **opts)
+    assert info.stream_k == 0
+
+
 @pytest.mark.parametrize("seed", range(48))
 def test_fuzz_random_contractions(seed):
     rng = np.random.default_rng(5000 + seed)

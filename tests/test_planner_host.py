@@ -261,3 +261,18 @@ def test_pair_variant_guard_rule():
     assert f(DEVICE, 1, 0) == 0          # a peer GPU's memory
     assert f(HOST, 0, 0) == 0 and f(MANAGED, 0, 0) == 0 and f(UNREGISTERED, 0, 0) == 0
     assert f(DEVICE, -1, -1) == 0        # a plan without a device
+
+
+def test_stream_k_is_chosen_when_the_last_round_of_tiles_would_be_mostly_empty():
+    """896 tiles on 148 SMs = six whole rounds + 8 tiles: the 8 are cut along K and shared by all SMs.
+    512 tiles = three rounds + 68: the idle time saved would not pay for the pieces' trip through memory."""
+    big = parse_spec("C[a,b,c,d] = A[a,e,b,f] * B[f,d,e,c]", dict(a=96, b=84, c=84, d=84, e=84, f=96))
+    i = g.Plan(big, g.GETT_BF16_F32).info
+    if i.grid == 148:   # (the rule depends on the SM count; without a device 148 is assumed)
+        assert i.stream_k == 1 and i.split_k == 1 and i.tiles == 896 and i.workspace_bytes > 0
+    assert g.Plan(big, g.GETT_BF16_F32, flags=g.GETT_OPT_NO_STREAMK).info.stream_k == 0
+    mid = parse_spec("C[m,n] = A[m,k] * B[k,n]", dict(m=4096, n=4096, k=2048))
+    assert g.Plan(mid, g.GETT_BF16_F32).info.stream_k == 0
+    assert g.Plan(mid, g.GETT_BF16_F32, flags=g.GETT_OPT_STREAMK).info.stream_k == 1
+    # never with K slices, never with fewer tiles than SMs
+    assert g.Plan(workload("splitk_vec").contraction, g.GETT_BF16_F32, flags=g.GETT_OPT_STREAMK).info.stream_k == 0
