@@ -33,7 +33,9 @@ from workloads import (BF16_F32, DTYPE_NAMES, F32, Contraction, TensorSpec, make
 
 METRIC = "TFLOP/s per contraction"
 UNIT = "TFLOP/s"
-DTYPE_BY_NAME = {"f32": F32, "bf16": BF16_F32}
+from workloads import F64  # noqa: E402
+
+DTYPE_BY_NAME = {"f32": F32, "bf16": BF16_F32, "f64": F64}
 
 
 def _peaks():
@@ -64,17 +66,17 @@ def measure_ffma_peak(torch, index: int):
     fn = lib.gett_bench_ffma_peak
     fn.restype = ctypes.c_longlong
     fn.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
-    out = torch.zeros(4, dtype=torch.float32, device="cuda")
+    out = torch.zeros(8, dtype=torch.float32, device="cuda")
     stream = torch.cuda.current_stream()
     sms = torch.cuda.get_device_properties(index).multi_processor_count
     res = {}
     with clock_sampler(index) as clk:
-        for name, packed in (("plain", 0), ("packed", 1)):
+        for name, packed in (("plain", 0), ("packed", 1), ("fp64", 2)):
             best = 0.0
             for rep in range(6):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
-                fmas = fn(packed, 4096, 2 * sms, out.data_ptr(), stream.cuda_stream)
+                fmas = fn(packed, 4096 if packed < 2 else 512, 2 * sms, out.data_ptr(), stream.cuda_stream)
                 e1.record(stream)
                 torch.cuda.synchronize()
                 if fmas < 0:
@@ -87,7 +89,7 @@ def measure_ffma_peak(torch, index: int):
             fn(1, 4096, 2 * sms, out.data_ptr(), stream.cuda_stream)
             torch.cuda.synchronize()
     c = clk.summary()
-    res["tflops"] = max(res["plain"], res["packed"])
+    res["tflops"] = max(res["plain"], res["packed"])  # fp32; res["fp64"] is the double-precision rate
     res["sm_mhz"] = c["sm_mhz"]
     res["reasons"] = c["reasons"]
     res["derived_at_sampled_clock"] = _fp32_peak_tflops(c["sm_mhz"]) if c["sm_mhz"] else None
@@ -203,10 +205,10 @@ def equal_gemm(con: Contraction) -> Contraction:
 
 def roofline_time_s(con, dtype, beta, peaks, fp32_peak):
     flops = con.flops()
-    peak = peaks["bf16_burst"] if dtype != F32 else fp32_peak
+    peak = peaks["bf16_burst"] if dtype not in (F32, F64) else fp32_peak  # (f64 rows pass their own FMA peak)
     t_c = flops / (peak * 1e12)
     t_m = con.compulsory_bytes(dtype, beta) / (peaks["hbm_gbs"] * 1e9)
-    return max(t_c, t_m), ("hbm" if t_m >= t_c else ("tensor" if dtype != F32 else "alu"))
+    return max(t_c, t_m), ("hbm" if t_m >= t_c else ("tensor" if dtype not in (F32, F64) else "alu"))
 
 
 # --------------------------------------------------------------------------- #
@@ -352,7 +354,11 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = _peaks()
     scale = {kv.split("=")[0]: int(kv.split("=")[1]) for kv in args.scale.split(",") if kv}
-    w = workload(args.workload, scale or None)
+    if args.workload.startswith("paper:"):  # one of the paper's 48 contractions (Table III extents), by its string
+        from workloads.paper_benchmark import paper_pool
+        w = [x for x in paper_pool("sp") if x.key == args.workload[6:]][0]
+    else:
+        w = workload(args.workload, scale or None)
     dtype = DTYPE_BY_NAME[args.dtype]
     con = w.contraction
     M, N, K = con.mnk()
@@ -413,6 +419,8 @@ def run_ours(args):
     sm_mhz = clocks["sm_mhz"] or 1965.0
     ffma = measure_ffma_peak(torch, local) if rank == 0 else None
     fp32_peak = ffma["tflops"] if ffma else _fp32_peak_tflops(sm_mhz)
+    if dtype == F64:  # the double-precision FMA rate measured the same way
+        fp32_peak = ffma["fp64"] if ffma else fp32_peak / 2
 
     # ---- roofline of the contraction kernel ----
     avg = float(per.mean())
@@ -464,6 +472,9 @@ def run_ours(args):
             out.update(run_pool(torch, g, peaks, args, paper_pool("sp"), "paper_pool"))
             out.update(run_pool(torch, g, peaks, args, fig11_sweep(), "fig11"))
             # the paper's own figures for the same statistic (one Haswell core, MKL GEMM): context only
+            if args.paper_pool_dp and ffma:  # Table IV: the same contractions with their double-precision extents
+                out.update(run_pool(torch, g, peaks, args, paper_pool("dp"), "paper_pool_dp", dtypes=(F64,),
+                                    fp_peak=ffma["fp64"]))
             out["paper_pool_context"] = {"gett_vs_equal_gemm_percent_sp": {"min": 72.4, "mean": 98.1, "max": 141.4},
                                          "source": "Sec. 7.2, Fig. 9"}
     elif rank == 0:
@@ -815,7 +826,7 @@ def ttgt_seconds(torch, g, con, dtype, alpha, beta, dev, steps, flush):
     return float(np.median(tot)), float(np.median(tr))
 
 
-def run_pool(torch, g, peaks, args, items=None, label="pool"):
+def run_pool(torch, g, peaks, args, items=None, label="pool", dtypes=None, fp_peak=None):
     """A pool of contractions -- the seeded synthetic pool (workloads.pool) or the paper's own 48
     shapes and its Fig. 11 sweep (workloads.paper_benchmark): per item and dtype the plan,
     TFLOP/s, roofline fraction and the ratio to the equal-sized GEMM through the same library
@@ -825,20 +836,20 @@ def run_pool(torch, g, peaks, args, items=None, label="pool"):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     for w in (items if items is not None else pool()):
         con = w.contraction
-        for dtype in w.dtypes:
+        for dtype in (dtypes or w.dtypes):
             a, b, c = make_inputs(con, dtype, w.dist, w.seed, w.beta, cache=True)
             dev = (_to_dev(a, torch), _to_dev(b, torch), _to_dev(c, torch))
             t, info = time_contraction(torch, g, con, dtype, w.alpha, w.beta, dev, args.all_steps, 3)
             flush.zero_()
             mhz = info["clocks"]["sm_mhz"] or 1965.0
-            t_roof, bound = roofline_time_s(con, dtype, w.beta, peaks, _fp32_peak_tflops(mhz))
+            t_roof, bound = roofline_time_s(con, dtype, w.beta, peaks, fp_peak or _fp32_peak_tflops(mhz))
             eg = equal_gemm(con)
             ga, gb, gc = make_inputs(eg, dtype, w.dist, w.seed, w.beta)
             gdev = (_to_dev(ga, torch), _to_dev(gb, torch), _to_dev(gc, torch))
             t_eq, _ = time_contraction(torch, g, eg, dtype, w.alpha, w.beta, gdev, args.all_steps, 3)
             M, N, K = con.mnk()
             extra = {}
-            if args.ttgt:
+            if args.ttgt and dtype != F64:
                 t_ttgt, t_tr = ttgt_seconds(torch, g, con, dtype, w.alpha, w.beta, dev, args.all_steps, None)
                 extra = {"ttgt_ms": t_ttgt * 1e3, "ttgt_transpose_share": t_tr / t_ttgt,
                          "speedup_vs_ttgt": t_ttgt / t}
@@ -885,6 +896,8 @@ def main():
                     help="with --kernel-only: also time the seeded pool of synthetic contractions")
     ap.add_argument("--paper-pool", action="store_true",
                     help="with --kernel-only: the paper's 48 contractions (Table III extents) and its Fig. 11 sweep")
+    ap.add_argument("--paper-pool-dp", action="store_true",
+                    help="with --paper-pool: also the 48 contractions with their Table IV extents in double precision")
     ap.add_argument("--ttgt", action="store_true",
                     help="pool runs: also time Transpose-Transpose-GEMM-Transpose (torch transpositions + this "
                          "library's plain GEMM) and report GETT's speedup over it")
@@ -904,6 +917,8 @@ def main():
     args = ap.parse_args()
     global SEARCH
     SEARCH = args.search
+    if args.dtype == "f64":
+        args.kernel_only = True  # (the end-to-end and equal-GEMM legs are set up for fp32 outputs)
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

@@ -53,7 +53,9 @@ typedef enum {
 typedef enum {
     GETT_F32 = 0,      /* A, B, C fp32; strict fp32 FMA accumulation          */
     GETT_BF16_F32 = 1, /* A, B bf16; fp32 accumulation; C fp32                */
-    GETT_F16_F32 = 2   /* A, B fp16; fp32 accumulation; C fp32                */
+    GETT_F16_F32 = 2,  /* A, B fp16; fp32 accumulation; C fp32                */
+    GETT_F64 = 3       /* A, B, C fp64; fp64 FMA accumulation (the precision of the paper's
+                          Table IV); scalar-gather kernel only, no K slices       */
 } gett_dtype_t;
 
 /*
@@ -208,7 +210,7 @@ GETT_API gett_status_t gett_plan_create(gett_plan_t** out, const gett_tensor_des
  * gett_contract -- run C <- alpha * A*B + beta * C (Eq. 2) on `cuda_stream`
  * (a cudaStream_t passed as void*; NULL = the default stream).
  *   A, B, C : DEVICE pointers, caller-owned, covering 1 + sum (extent-1)*stride
- *             elements each; A/B of the plan's input type, C fp32.  Bases must be
+ *             elements each; A/B of the plan's input type, C fp32 (fp64 for GETT_F64).  Bases must be
  *             aligned to the element size; 16-byte aligned bases enable the
  *             vectorised kernels, otherwise the scalar path is used.
  *   alpha, beta : host scalars.  beta == 0 means C is not read (NaN/Inf in the

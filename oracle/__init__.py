@@ -75,7 +75,7 @@ def _mk(spec):
 
 
 def _operand(x: np.ndarray, dtype: int) -> np.ndarray:
-    want = np.float32 if dtype == 0 else np.uint16
+    want = np.float32 if dtype == 0 else np.float64 if dtype == 3 else np.uint16
     x = np.ascontiguousarray(x)
     if x.dtype != want:
         raise TypeError(f"operand dtype {x.dtype}, expected {want}")
@@ -103,7 +103,7 @@ def contract(con, dtype: int, alpha: float, A: np.ndarray, B: np.ndarray, beta: 
     cabs = np.zeros(con.C.span, dtype=np.float64) if want_abs else None
     cold = None
     if beta != 0.0:
-        cold = np.ascontiguousarray(C_old, dtype=np.float32)
+        cold = np.ascontiguousarray(C_old, dtype=np.float64 if dtype == 3 else np.float32)
         if cold.size < con.C.span:
             raise ValueError("C_old smaller than its span")
     rc = lib.gett_oracle_contract(ctypes.byref(ta), ctypes.byref(tb), ctypes.byref(tc), dtype,
@@ -133,7 +133,7 @@ def points(con, dtype: int, alpha: float, A: np.ndarray, B: np.ndarray, beta: fl
     ab = np.zeros(n, dtype=np.float64)
     cold = None
     if beta != 0.0:
-        cold = np.ascontiguousarray(C_old, dtype=np.float32)
+        cold = np.ascontiguousarray(C_old, dtype=np.float64 if dtype == 3 else np.float32)
     rc = lib.gett_oracle_points(ctypes.byref(ta), ctypes.byref(tb), ctypes.byref(tc), dtype,
                                 float(alpha), A.ctypes.data, B.ctypes.data, float(beta),
                                 cold.ctypes.data if cold is not None else None, n,

@@ -35,7 +35,7 @@
 
 #define ORACLE_MAX_MODES 32
 
-enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_F16 = 2 };
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_F16 = 2, ORACLE_F64 = 3 /* A, B and the old C stored as double */ };
 
 enum {
     ORACLE_OK = 0,
@@ -51,11 +51,19 @@ typedef struct {
     const int32_t *label;
 } oracle_tensor_t;
 
+/* the old value of C: stored as float, except for ORACLE_F64 */
+static double load_c_old(const void *base, int64_t off, int dtype)
+{
+    return dtype == ORACLE_F64 ? ((const double *)base)[off] : (double)((const float *)base)[off];
+}
+
 /* exact widening of one stored operand element */
 static double load_operand(const void *base, int64_t off, int dtype)
 {
     if (dtype == ORACLE_F32)
         return (double)((const float *)base)[off];
+    if (dtype == ORACLE_F64)
+        return ((const double *)base)[off];
     uint16_t h = ((const uint16_t *)base)[off];
     if (dtype == ORACLE_BF16) {
         uint32_t u = (uint32_t)h << 16;
@@ -186,7 +194,7 @@ static void one_output(const loops_t *L, const void *A, const void *B, int dtype
 typedef struct {
     const loops_t *L;
     const void *A, *B;
-    const float *C_old;
+    const void *C_old;
     int dtype;
     double alpha, beta;
     double *C_ref, *absacc;
@@ -215,7 +223,7 @@ static void *run_job(void *arg)
         one_output(L, J->A, J->B, J->dtype, oa, ob, &acc, &aacc);
         double r = J->alpha * acc;
         if (J->beta != 0.0)
-            r += J->beta * (double)J->C_old[oc];
+            r += J->beta * load_c_old(J->C_old, oc, J->dtype);
         J->C_ref[oc] = r;
         if (J->absacc)
             J->absacc[oc] = aacc;
@@ -239,7 +247,7 @@ static void *run_job(void *arg)
  */
 int gett_oracle_contract(const oracle_tensor_t *A, const oracle_tensor_t *B,
                          const oracle_tensor_t *C, int dtype, double alpha, const void *A_data,
-                         const void *B_data, double beta, const float *C_old, double *C_ref,
+                         const void *B_data, double beta, const void *C_old, double *C_ref,
                          double *absacc, int nthreads)
 {
     loops_t L;
@@ -248,7 +256,7 @@ int gett_oracle_contract(const oracle_tensor_t *A, const oracle_tensor_t *B,
         return rc;
     if (!A_data || !B_data || !C_ref || (beta != 0.0 && !C_old))
         return ORACLE_ERR_ARG;
-    if (dtype < ORACLE_F32 || dtype > ORACLE_F16)
+    if (dtype < ORACLE_F32 || dtype > ORACLE_F64)
         return ORACLE_ERR_ARG;
     int64_t outer = L.nfree ? L.free_ext[L.nfree - 1] : 1;
     if (nthreads < 1)
@@ -278,7 +286,7 @@ int gett_oracle_contract(const oracle_tensor_t *A, const oracle_tensor_t *B,
 typedef struct {
     const loops_t *L;
     const void *A, *B;
-    const float *C_old;
+    const void *C_old;
     int dtype;
     double alpha, beta;
     const int64_t *points;
@@ -302,7 +310,7 @@ static void *run_points(void *arg)
         one_output(L, J->A, J->B, J->dtype, oa, ob, &acc, &aacc);
         double r = J->alpha * acc;
         if (J->beta != 0.0)
-            r += J->beta * (double)J->C_old[oc];
+            r += J->beta * load_c_old(J->C_old, oc, J->dtype);
         J->out[p] = r;
         if (J->absacc)
             J->absacc[p] = aacc;
@@ -316,7 +324,7 @@ static void *run_points(void *arg)
  */
 int gett_oracle_points(const oracle_tensor_t *A, const oracle_tensor_t *B,
                        const oracle_tensor_t *C, int dtype, double alpha, const void *A_data,
-                       const void *B_data, double beta, const float *C_old, int64_t npoints,
+                       const void *B_data, double beta, const void *C_old, int64_t npoints,
                        const int64_t *points, double *out, double *absacc, int nthreads)
 {
     loops_t L;
@@ -326,7 +334,7 @@ int gett_oracle_points(const oracle_tensor_t *A, const oracle_tensor_t *B,
     if (!A_data || !B_data || !out || (npoints > 0 && L.nfree > 0 && !points) ||
         (beta != 0.0 && !C_old))
         return ORACLE_ERR_ARG;
-    if (dtype < ORACLE_F32 || dtype > ORACLE_F16)
+    if (dtype < ORACLE_F32 || dtype > ORACLE_F64)
         return ORACLE_ERR_ARG;
     for (int64_t p = 0; p < npoints; ++p)
         for (int f = 0; f < L.nfree; ++f)

@@ -8,7 +8,7 @@ from typing import Dict, Optional, Sequence
 import numpy as np
 
 GETT_MAX_MODES = 12
-GETT_F32, GETT_BF16_F32, GETT_F16_F32 = 0, 1, 2
+GETT_F32, GETT_BF16_F32, GETT_F16_F32, GETT_F64 = 0, 1, 2, 3
 GETT_PATH_AUTO, GETT_PATH_SIMT, GETT_PATH_FFMA, GETT_PATH_UMMA = 0, 1, 2, 3
 GETT_LOAD_SCALAR, GETT_LOAD_VEC_FREE, GETT_LOAD_VEC_K = 0, 1, 2
 GETT_LOAD_TMA_FREE, GETT_LOAD_TMA_K, GETT_LOAD_VEC_KT = 3, 4, 5

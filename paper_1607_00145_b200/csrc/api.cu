@@ -243,12 +243,12 @@ gett_status_t create_by_search(gett_plan_t** out, const gett_tensor_desc_t* A, c
     int timed = 0;
     if (asked.search > 1 && device >= 0) {
         // time the k best on scratch operands (zeros: finite, and the kernels do not look at values)
-        const size_t es = dtype == GETT_F32 ? 4 : 2;
+        const size_t es = dtype == GETT_F32 ? 4 : dtype == GETT_F64 ? 8 : 2;
         void *dA = nullptr, *dB = nullptr, *dC = nullptr, *dFlush = nullptr;
         const size_t flush_bytes = 192u << 20; // larger than L2: every timed launch starts cold
         cudaStream_t st = nullptr;
         cudaEvent_t e0 = nullptr, e1 = nullptr;
-        const size_t nA = span_elems(A) * es, nB = span_elems(B) * es, nC = span_elems(C) * 4;
+        const size_t nA = span_elems(A) * es, nB = span_elems(B) * es, nC = span_elems(C) * (dtype == GETT_F64 ? 8 : 4);
         bool ok = cudaMalloc(&dA, nA) == cudaSuccess && cudaMalloc(&dB, nB) == cudaSuccess &&
                   cudaMalloc(&dC, nC) == cudaSuccess && cudaMalloc(&dFlush, flush_bytes) == cudaSuccess &&
                   cudaMemset(dA, 0, nA) == cudaSuccess &&
@@ -377,8 +377,8 @@ gett_status_t gett_contract(const gett_plan_t* plan, float alpha, const void* A,
         if (dev != plan->info.device)
             return GETT_ERR_INVALID_ARG;
     }
-    const uintptr_t es = plan->dtype == GETT_F32 ? 4 : 2;
-    if (((uintptr_t)A % es) || ((uintptr_t)B % es) || ((uintptr_t)C % 4))
+    const uintptr_t es = plan->dtype == GETT_F32 ? 4 : plan->dtype == GETT_F64 ? 8 : 2;
+    if (((uintptr_t)A % es) || ((uintptr_t)B % es) || ((uintptr_t)C % (plan->dtype == GETT_F64 ? 8 : 4)))
         return GETT_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 

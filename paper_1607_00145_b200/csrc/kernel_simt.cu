@@ -15,9 +15,21 @@ namespace {
 
 constexpr int TM = 64, TN = 64, TK = 16, NT = 256;
 
+// The type the sums are kept in (and C is stored as): double for GETT_F64, else float.
 template <int DT>
-__device__ __forceinline__ float load_elem(const void* base, int64_t off)
+struct Acc {
+    typedef float type;
+};
+template <>
+struct Acc<GETT_F64> {
+    typedef double type;
+};
+
+template <int DT>
+__device__ __forceinline__ typename Acc<DT>::type load_elem(const void* base, int64_t off)
 {
+    if (DT == GETT_F64)
+        return __ldg(reinterpret_cast<const double*>(base) + off);
     if (DT == GETT_F32)
         return __ldg(reinterpret_cast<const float*>(base) + off);
     unsigned short h = __ldg(reinterpret_cast<const unsigned short*>(base) + off);
@@ -30,7 +42,8 @@ template <int DT>
 __global__ void __launch_bounds__(NT) gett_simt_kernel(const __grid_constant__ GettKernelArgs g)
 {
     __shared__ int64_t offAM[TM], offCM[TM], offBN[TN], offCN[TN], offAK[TK], offBK[TK];
-    __shared__ float As[TK][TM + 1], Bs[TK][TN + 1];
+    typedef typename Acc<DT>::type T; // fp32, or fp64 for GETT_F64 (round-to-nearest FMAs either way)
+    __shared__ T As[TK][TM + 1], Bs[TK][TN + 1];
 
     const uint32_t tiles = g.tiles_m * g.tiles_n;
     const uint32_t z = blockIdx.x / tiles;
@@ -57,12 +70,12 @@ __global__ void __launch_bounds__(NT) gett_simt_kernel(const __grid_constant__ G
         offCN[c] = y;
     }
 
-    float acc[4][4];
+    T acc[4][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            acc[i][j] = 0.f;
+            acc[i][j] = 0;
     const int tx = tid & 15, ty = tid >> 4;
 
     for (uint32_t k0 = kbeg; k0 < kend; k0 += TK) {
@@ -86,7 +99,7 @@ __global__ void __launch_bounds__(NT) gett_simt_kernel(const __grid_constant__ G
                 r = e % TM;
                 k = e / TM;
             }
-            float v = 0.f;
+            T v = 0;
             if (m0 + r < Msz && k0 + k < kend)
                 v = load_elem<DT>(g.A, offAM[r] + offAK[k]);
             As[k][r] = v;
@@ -102,7 +115,7 @@ __global__ void __launch_bounds__(NT) gett_simt_kernel(const __grid_constant__ G
                 c = e % TN;
                 k = e / TN;
             }
-            float v = 0.f;
+            T v = 0;
             if (n0 + c < Nsz && k0 + k < kend)
                 v = load_elem<DT>(g.B, offBN[c] + offBK[k]);
             Bs[k][c] = v;
@@ -110,7 +123,7 @@ __global__ void __launch_bounds__(NT) gett_simt_kernel(const __grid_constant__ G
         __syncthreads();
 #pragma unroll
         for (int k = 0; k < TK; ++k) {
-            float a[4], b[4];
+            T a[4], b[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
                 a[i] = As[k][tx + 16 * i];
@@ -121,7 +134,7 @@ __global__ void __launch_bounds__(NT) gett_simt_kernel(const __grid_constant__ G
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+                    acc[i][j] = fma(a[i], b[j], acc[i][j]);
         }
     }
     __syncthreads(); // offset tables visible even when the K range was empty
@@ -137,12 +150,12 @@ __global__ void __launch_bounds__(NT) gett_simt_kernel(const __grid_constant__ G
             if (m0 + r >= Msz)
                 continue;
             if (g.split_k > 1) {
-                g.ws[((size_t)z * Nsz + (n0 + c)) * Msz + (m0 + r)] = acc[i][j];
+                g.ws[((size_t)z * Nsz + (n0 + c)) * Msz + (m0 + r)] = (float)acc[i][j]; // (never GETT_F64)
             } else {
-                float* dst = g.C + offCM[r] + offCN[c];
-                float v = g.alpha * acc[i][j];
+                T* dst = reinterpret_cast<T*>(g.C) + offCM[r] + offCN[c];
+                T v = (T)g.alpha * acc[i][j];
                 if (g.beta != 0.f)
-                    v = fmaf(g.beta, *dst, v);
+                    v = fma((T)g.beta, *dst, v);
                 *dst = v;
             }
         }
@@ -156,6 +169,7 @@ cudaError_t gett_launch_simt(const GettKernelArgs& args, int grid, cudaStream_t 
     switch (args.dtype) {
     case GETT_F32: gett_simt_kernel<GETT_F32><<<grid, NT, 0, stream>>>(args); break;
     case GETT_BF16_F32: gett_simt_kernel<GETT_BF16_F32><<<grid, NT, 0, stream>>>(args); break;
+    case GETT_F64: gett_simt_kernel<GETT_F64><<<grid, NT, 0, stream>>>(args); break;
     default: gett_simt_kernel<GETT_F16_F32><<<grid, NT, 0, stream>>>(args); break;
     }
     return cudaGetLastError();

@@ -60,6 +60,8 @@ extern "C" gett_status_t gett_contract_noalloc(const gett_tensor_desc_t* A, cons
 {
     if (!A || !B || !C || !A_data || !B_data || !C_data || split_k < 0)
         return GETT_ERR_INVALID_ARG;
+    if (dtype == GETT_F64)
+        return GETT_ERR_UNSUPPORTED; // (its partial sums are fp32)
     float* scratch = nullptr;
     int sms = 0;
     gett_status_t rc = scratch_for_current_device(&scratch, &sms);

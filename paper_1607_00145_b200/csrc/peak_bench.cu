@@ -40,6 +40,26 @@ __global__ void __launch_bounds__(1024, 1) ffma_peak_kernel(float* out, float a,
         out[0] = s;
 }
 
+// The same loop in double precision (the denominator for GETT_F64 rows).
+__global__ void __launch_bounds__(1024, 1) dfma_peak_kernel(double* out, double a, double b, int iters)
+{
+    double acc[CHAINS / 2];
+#pragma unroll
+    for (int i = 0; i < CHAINS / 2; ++i)
+        acc[i] = (double)threadIdx.x * 1e-6 + (double)i;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < CHAINS / 2; ++i)
+            acc[i] = fma(acc[i], a, b);
+    }
+    double s = 0.0;
+#pragma unroll
+    for (int i = 0; i < CHAINS / 2; ++i)
+        s += acc[i];
+    if (s == 12345.678)
+        out[0] = s;
+}
+
 } // namespace
 
 // Launches the loop on `stream`; returns the FMA count (one FMA = 2 flop) or -1 on a launch
@@ -51,6 +71,12 @@ extern "C" __attribute__((visibility("default"))) long long gett_bench_ffma_peak
     if (iters < 1 || blocks < 1 || !out)
         return -1;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (packed == 2) { // double precision; out must then hold at least one double
+        dfma_peak_kernel<<<blocks, 1024, 0, s>>>(reinterpret_cast<double*>(out), 1.0000001, 1e-9, iters);
+        if (cudaGetLastError() != cudaSuccess)
+            return -1;
+        return (long long)blocks * 1024 * (CHAINS / 2) * (long long)iters;
+    }
     if (packed)
         ffma_peak_kernel<1><<<blocks, 1024, 0, s>>>(out, 1.0000001f, 1e-9f, iters);
     else

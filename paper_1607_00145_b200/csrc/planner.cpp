@@ -480,7 +480,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     gett_status_t rc;
     if ((rc = read_desc(dA, A)) || (rc = read_desc(dB, B)) || (rc = read_desc(dC, C)))
         return rc;
-    if (dtype != GETT_F32 && dtype != GETT_BF16_F32 && dtype != GETT_F16_F32)
+    if (dtype != GETT_F32 && dtype != GETT_BF16_F32 && dtype != GETT_F16_F32 && dtype != GETT_F64)
         return GETT_ERR_UNSUPPORTED;
     gett_plan_opts_t o;
     memset(&o, 0, sizeof o);
@@ -544,7 +544,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         for (const GettMode& m : ik)
             ksz *= m.ext;
         const bool small_nk = dtype == GETT_F32 && nsz <= 64 && ksz <= gett_ffma_skinny_max_k();
-        bool want = !small_nk && unitCm >= 0 && unitAm >= 0 && unitCm != unitAm && im[unitAm].ext % vec == 0 &&
+        bool want = dtype != GETT_F64 && !small_nk && unitCm >= 0 && unitAm >= 0 && unitCm != unitAm && im[unitAm].ext % vec == 0 &&
                     im[unitAm].ext > vec && im[unitCm].ext % 4 == 0 && o.epilogue != GETT_EPI_DIRECT &&
                     !(o.flags & GETT_OPT_NO_EXCHANGE);
         if (want && dtype == GETT_F32) { // the same alignment the fp32 split asks for
@@ -575,7 +575,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     // modes of I_n, and B's can be split into pieces of one 16-byte vector (vecB elements).
     auto n_split_ok = [&](int64_t vecB) {
         const int unitCn = find_unit(in, 2);
-        if (!(leadN >= 0 && unitCn >= 0 && unitCn != leadN && in[leadN].ext % vecB == 0 &&
+        if (!(dtype != GETT_F64 && leadN >= 0 && unitCn >= 0 && unitCn != leadN && in[leadN].ext % vecB == 0 &&
               in[leadN].ext > vecB && o.epilogue != GETT_EPI_DIRECT))
             return false;
         if (dtype != GETT_F32)
@@ -659,7 +659,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     // of pieces of two modes).  A is then read in 16-byte pieces along u as usual; B is read
     // in 16-byte pieces along v and its 8 x 8 blocks are transposed on the way (Sec. 3.2.2).
     bool k_transposed = false;
-    if (dtype != GETT_F32) {
+    if (dtype == GETT_BF16_F32 || dtype == GETT_F16_F32) {
         const int uA = find_unit(ik, 0), uB = find_unit(ik, 1);
         if (uA >= 0 && uB >= 0 && uA != uB && ik[uA].ext % 8 == 0 && ik[uB].ext % 8 == 0) {
             std::vector<GettDigit> t;
@@ -745,7 +745,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         const int64_t worst = std::max(maxA, maxB);
         offsets_fit = dtype == GETT_F32 ? worst < (int64_t)0xFFFFFFF0ll : (worst >> 3) < (int64_t)0xFFFFFFF0ll;
     }
-    const bool umma_ok = dtype != GETT_F32 && both_vec && offsets_fit;
+    const bool umma_ok = dtype != GETT_F32 && dtype != GETT_F64 && both_vec && offsets_fit;
     // fp32 with small N and K and a K-major A: B is read once element by element, so
     // only A has to be gatherable in 16-byte vectors
     const bool skinny_ok = dtype == GETT_F32 &&
@@ -790,6 +790,8 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     if (o.tile_m < 0 || o.tile_n < 0 || o.tile_k < 0 || o.stages < 0 || o.split_k < 0)
         return GETT_ERR_INVALID_ARG;
     const int sms = sm_count > 0 ? sm_count : 148;
+    if (dtype == GETT_F64 && o.split_k > 1)
+        return GETT_ERR_UNSUPPORTED; // (the workspace of the K slices holds fp32 sums)
     if (path == GETT_PATH_SIMT) {
         if ((o.tile_m && o.tile_m != 64) || (o.tile_n && o.tile_n != 64) ||
             (o.tile_k && o.tile_k != 16) || (o.stages && o.stages != 1) ||
@@ -997,7 +999,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     uint32_t split = 1;
     if (o.split_k > 1) {
         split = std::min<uint32_t>((uint32_t)o.split_k, kslabs);
-    } else if (o.split_k == 0 && sm_count > 0 && tiles * 2 <= (uint64_t)sm_count && kslabs >= 8) {
+    } else if (o.split_k == 0 && dtype != GETT_F64 && sm_count > 0 && tiles * 2 <= (uint64_t)sm_count && kslabs >= 8) {
         // choose the slice count whose (waves of work items) x (slabs per item + a fixed
         // per-item cost for the epilogue and the reduction) is smallest
         const uint64_t slots = (uint64_t)sm_count * (path == GETT_PATH_UMMA ? 1 : path == GETT_PATH_FFMA ? 2 : 4);

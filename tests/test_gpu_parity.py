@@ -6,7 +6,7 @@ import pytest
 import paper_1607_00145_b200 as g
 from gpu_util import TOL, parity_case
 from helpers import random_contraction
-from workloads import BF16_F32, F16_F32, F32, parse_spec, workload
+from workloads import BF16_F32, F16_F32, F32, F64, parse_spec, workload
 
 pytestmark = pytest.mark.gpu
 
@@ -277,6 +277,30 @@ def test_stream_k_shares_of_the_tile_slab_space(spec, sizes, opts):
             assert info.stream_k == 1 and info.split_k == 1 and info.workspace_bytes > 0
     ratio, info = parity_case(con, BF16_F32, "normal", 71, 1.0, 0.5, flags=g.GETT_OPT_NO_STREAMK, **opts)
     assert info.stream_k == 0
+
+
+@pytest.mark.parametrize("key", sorted(SMALL))
+def test_double_precision_path(key):
+    """GETT_F64 (the precision of the paper's Table IV): fp64 operands, fp64 FMAs, fp64 C, through the
+    scalar-gather kernel; against the oracle to 1e-13 of the scale, twice, and with beta = 0 on NaN."""
+    w = workload(key, SMALL[key])
+    ratio, info = parity_case(w.contraction, F64, w.dist, w.seed, w.alpha, w.beta, repeat=2)
+    assert info.path == g.GETT_PATH_SIMT and info.split_k == 1
+    parity_case(w.contraction, F64, w.dist, w.seed, -0.5, 0.0)
+    with pytest.raises(g.GettError) as e:   # no K slices, no vector kernels in double precision
+        g.Plan(w.contraction, F64, split_k=2)
+    assert e.value.status == 4
+    with pytest.raises(g.GettError) as e:
+        g.Plan(w.contraction, F64, path=g.GETT_PATH_FFMA)
+    assert e.value.status == 4
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_double_precision_fuzz(seed):
+    rng = np.random.default_rng(9000 + seed)
+    con = random_contraction(rng, max_rank=6, max_extent=9, min_each=0 if seed % 6 == 0 else 1)
+    alpha, beta = [(1.0, 0.0), (1.0, 1.0), (-0.5, 2.0)][seed % 3]
+    parity_case(con, F64, "uniform", seed, alpha, beta)
 
 
 @pytest.mark.parametrize("seed", range(48))

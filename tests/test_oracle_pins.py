@@ -290,3 +290,28 @@ def test_repeated_label_and_extent_mismatch_are_rejected():
     with pytest.raises(oracle.OracleError) as e:
         oracle.contract(con, F32, 1.0, np.zeros(6, np.float32), np.zeros(8, np.float32), 0.0, None)
     assert e.value.code == 3
+
+
+# ---- fp64 operands (the precision of the paper's Table IV): same loop nest, double storage ----
+@pytest.mark.parametrize("seed", range(12))
+def test_fp64_operands_match_brute_force_exactly_and_einsum(seed):
+    from workloads import F64, uniform_pm1_f64
+    rng = np.random.default_rng(300 + seed)
+    con = random_contraction(rng, max_rank=5, max_extent=5)
+    # small integers stored as double: the flatten-to-matrix brute force is exact
+    a, b, c = (x.astype(np.float64) for x in _ints(con, seed))
+    alpha, beta = [(1.0, 0.0), (2.0, -1.0), (-3.0, 2.0)][seed % 3]
+    got, _ = oracle.contract(con, F64, alpha, a, b, beta, c, threads=1 + seed % 3)
+    assert np.array_equal(got, brute_force(con, a, b, alpha, beta, c))
+    # 53-bit draws: the old C really is read as double (a float read would lose the low bits)
+    a, b, c = (uniform_pm1_f64(seed, t, n) for t, n in ((1, con.A.span), (2, con.B.span), (3, con.C.span)))
+    got, absacc = oracle.contract(con, F64, 1.0, a, b, 1.0, c)
+    ref = scatter_nd(einsum_ref(con, a, b), con.C)
+    off = oracle.c_offsets(con)
+    np.testing.assert_allclose(got[off], ref[off] + c[off], rtol=0, atol=4e-15 * max(1.0, absacc.max()))
+    only_c, _ = oracle.contract(con, F64, 0.0, a, b, 1.0, c)
+    assert np.array_equal(only_c[off], c[off])          # bit-exact doubles, not floats
+    pts = np.stack([rng.integers(0, e, 20) for e in con.C.extents], axis=1) if con.C.extents else np.zeros((1, 0), int)
+    pv, _ = oracle.points(con, F64, 1.0, a, b, 1.0, c, pts)
+    poff = (pts * np.array(con.C.strides, dtype=np.int64)).sum(axis=1) if con.C.extents else np.zeros(1, int)
+    assert np.array_equal(pv, got[poff])

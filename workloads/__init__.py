@@ -25,8 +25,8 @@ from typing import Dict, List, Optional, Sequence, Tuple
 
 import numpy as np
 
-F32, BF16_F32, F16_F32 = 0, 1, 2
-DTYPE_NAMES = {F32: "f32", BF16_F32: "bf16", F16_F32: "f16"}
+F32, BF16_F32, F16_F32, F64 = 0, 1, 2, 3
+DTYPE_NAMES = {F32: "f32", BF16_F32: "bf16", F16_F32: "f16", F64: "f64"}
 
 _GOLDEN = np.uint64(0x9E3779B97F4A7C15)
 _MIX = np.uint64(0xBF58476D1CE4E5B9)
@@ -58,6 +58,17 @@ def uniform_pm1(seed: int, tensor_id: int, n: int, chunk: int = 1 << 24) -> np.n
         h = _hash(seed, tensor_id, np.arange(s, e, dtype=np.uint64))
         v = (h >> np.uint64(40)).astype(np.int64) - (1 << 23)
         out[s:e] = (v.astype(np.float64) / float(1 << 23)).astype(np.float32)
+    return out
+
+
+def uniform_pm1_f64(seed: int, tensor_id: int, n: int, chunk: int = 1 << 24) -> np.ndarray:
+    """n fp64 values in [-1, 1) with 53 random bits each: ((h >> 11) - 2^52) / 2^52."""
+    out = np.empty(n, dtype=np.float64)
+    for s in range(0, n, chunk):
+        e = min(n, s + chunk)
+        h = _hash(seed, tensor_id, np.arange(s, e, dtype=np.uint64))
+        v = (h >> np.uint64(11)).astype(np.int64) - (1 << 52)
+        out[s:e] = v.astype(np.float64) / float(1 << 52)
     return out
 
 
@@ -198,8 +209,8 @@ class Contraction:
 
     def compulsory_bytes(self, dtype: int, beta: float) -> int:
         """|A| + |B| + |C| * (1 + [beta != 0]) with fp32 C."""
-        ab = 4 if dtype == F32 else 2
-        c = self.C.numel * 4
+        ab = 4 if dtype == F32 else 8 if dtype == F64 else 2
+        c = self.C.numel * (8 if dtype == F64 else 4)
         return self.A.numel * ab + self.B.numel * ab + c * (2 if beta != 0.0 else 1)
 
 
@@ -369,6 +380,11 @@ def make_inputs(con: Contraction, dtype: int, dist: str, seed: int, beta: float,
     (drawn uniform[-1,1) when beta != 0, zeros otherwise, as the workloads say).
     cache: reuse the fp32 draws of earlier calls with the same seed and span (read-only arrays).
     """
+    if dtype == F64:  # double precision throughout: A, B and C are fp64 with 53-bit draws
+        a = uniform_pm1_f64(seed, TENSOR_ID["A"], con.A.span)
+        b = uniform_pm1_f64(seed, TENSOR_ID["B"], con.B.span)
+        c = uniform_pm1_f64(seed, TENSOR_ID["C"], con.C.span) if beta != 0.0 else np.zeros(con.C.span, dtype=np.float64)
+        return a, b, c
     d = draw_cached if cache else draw
     a = encode_operand(d(dist, seed, "A", con.A.span), dtype)
     b = encode_operand(d(dist, seed, "B", con.B.span), dtype)
