@@ -97,6 +97,31 @@ def measure_ffma_peak(torch, index: int):
     return res
 
 
+def run_copy_probe():
+    """One launch per access pattern of the 16-byte asynchronous copy (see csrc/copy_probe_bench.cu);
+    prints the time of each; meant to be run under a profiler that counts the L2 -> SM bytes."""
+    import ctypes
+    import torch
+    lib = ctypes.CDLL(os.path.join(ROOT, "paper_1607_00145_b200", "libgett_b200_bench.so"))
+    fn = lib.gett_bench_copy_probe
+    fn.restype = ctypes.c_longlong
+    fn.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+    span = 384 << 20  # more than one launch touches, so that no region is read twice
+    buf = torch.ones(span + 4096, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    rows = []
+    for rep in range(2):
+        for pattern in range(11):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            asked = fn(pattern, 64, 148 * 4, buf.data_ptr(), span, stream.cuda_stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if rep:
+                rows.append({"pattern": pattern, "ms": e0.elapsed_time(e1), "bytes_asked": int(asked)})
+    print(json.dumps({"copy_probe": rows}))
+
+
 class NvmlSampler:
     """SM clock and throttle reasons read through NVML (read-only) every few ms."""
     BITS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
@@ -898,6 +923,8 @@ def main():
                     help="with --kernel-only: the paper's 48 contractions (Table III extents) and its Fig. 11 sweep")
     ap.add_argument("--paper-pool-dp", action="store_true",
                     help="with --paper-pool: also the 48 contractions with their Table IV extents in double precision")
+    ap.add_argument("--copy-probe", action="store_true",
+                    help="run the access-pattern probe of the 16-byte asynchronous copy and exit")
     ap.add_argument("--ttgt", action="store_true",
                     help="pool runs: also time Transpose-Transpose-GEMM-Transpose (torch transpositions + this "
                          "library's plain GEMM) and report GETT's speedup over it")
@@ -917,6 +944,9 @@ def main():
     args = ap.parse_args()
     global SEARCH
     SEARCH = args.search
+    if args.copy_probe:
+        run_copy_probe()
+        return
     if args.dtype == "f64":
         args.kernel_only = True  # (the end-to-end and equal-GEMM legs are set up for fp32 outputs)
     if args.warmup < 3 and args.impl == "ours":
