@@ -41,7 +41,7 @@ __global__ void copy_probe_kernel(const char* __restrict__ g, int pattern, int i
         case 10: off = lane * 32; break;
         default: off = lane * 16; break;
         }
-        copy16(s0 + warp * 1024 + lane * 16, g + base + off);
+        copy16(s0 + warp * 1024 + (it & 1) * 512 + lane * 16, g + base + off);
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
 }

@@ -98,6 +98,27 @@ struct alignas(16) SmemTables { // the staging rows that follow it hold 128-bit 
 
 static_assert(sizeof(SmemTables) % 16 == 0, "staging area must stay 16-byte aligned");
 
+// Time stamps of CTA 0's roles (experiment builds only, opts.experiment & 4096): role = producer
+// group 0 / 1, 2 = MMA issuer, 4 / 5 = first warp of epilogue set 0 / 1; one thread per role writes.
+#ifdef GETT_EXPERIMENT
+__device__ unsigned long long gett_trace_buf[8][4096];
+__device__ unsigned int gett_trace_n[8];
+#define GETT_TRACE(role, tag)                                                                          \
+    do {                                                                                               \
+        if (blockIdx.x == 0 && (g.debug & 4096)) {                                                     \
+            const unsigned n_ = gett_trace_n[role];                                                    \
+            if (n_ < 4096) {                                                                           \
+                gett_trace_buf[role][n_] = ((unsigned long long)(tag) << 56) | (clock64() & 0xFFFFFFFFFFFFFFull); \
+                gett_trace_n[role] = n_ + 1;                                                           \
+            }                                                                                          \
+        }                                                                                              \
+    } while (0)
+#else
+#define GETT_TRACE(role, tag)                                                                          \
+    do {                                                                                               \
+    } while (0)
+#endif
+
 __host__ __device__ constexpr uint32_t stage_bytes(uint32_t tile_m, uint32_t tile_n)
 {
     return (tile_m + tile_n) * TILE_K * 2;
@@ -408,9 +429,12 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
     using Sh = StagedShape<TILE_N, CV, LEAN>;
     const uint64_t wait_ns = (uint64_t)g.wait_limit_us * 1000ull;
     constexpr uint32_t NCH = Sh::NCH, PITCH = Sh::PITCH, GPR = Sh::GPR, NP = Sh::NP, DEPTH = Sh::DEPTH;
-    constexpr uint32_t FULL = 0xFFFFFFFFu;
     float* S = reinterpret_cast<float*>(epi_smem + warp * epi_warp_bytes(TILE_N, CV, LEAN));
-    int64_t* grp = reinterpret_cast<int64_t*>(S + DEPTH * 32 * PITCH);
+    // C offsets, in units of 16 bytes (every group of four slots is one aligned vector of C; the
+    // planner keeps C's largest offset below 2^36 bytes for this epilogue), for tiles j even / odd:
+    uint32_t* grp16 = reinterpret_cast<uint32_t*>(S + DEPTH * 32 * PITCH); // ... of the tile's 16-byte column groups
+    uint32_t* row16 = grp16 + 2 * EPI_GROUPS;                              // ... of this warp's 32 rows
+    static_assert(2 * EPI_GROUPS * 4 + 2 * 32 * 4 <= EPI_DEPTH * EPI_GROUPS * 8, "offset tables fit their space");
     const uint32_t s_u32 = ptx::smem_u32(S);
     const float alpha = g.alpha, beta = g.beta;
     const bool rmw = beta != 0.f && !GETT_DBG(g, 128); // (debug & 128: experiment, old C not read)
@@ -419,50 +443,55 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
     const uint32_t ncta = total_work > GETT_WB ? (total_work - GETT_WB + GETT_WG - 1) / GETT_WG : 0;
     const uint32_t ntile = ncta > es ? (ncta - es + 1) / 2 : 0;
     const uint32_t nchunk = ntile * NCH;
-    static_assert(EPI_DEPTH == 2, "row offsets are kept in two scalars");
-    long long rowC_0 = -1, rowC_1 = -1; // C offset of my row, for j even / odd
-    auto my_row = [&](uint32_t j) { return (j & 1) ? rowC_1 : rowC_0; };
+    // Moving a chunk (32 rows x GPR groups of 16 bytes) between C and the staging buffer, lanes
+    // running along C: copy number t of a lane is item lane + 32 t, item q = group q % GPR of row
+    // q / GPR.  32 t % GPR has period GCYC in t, so a lane meets only GCYC different groups --
+    // whose C offsets it reads once per chunk -- and its rows advance by RSTEP per period:
+    // what is left per copy is one table read (the row's offset), one add and the copy.
+    constexpr uint32_t GCYC = 32 % GPR == 0 ? 1 : 3;
+    static_assert((32 * GCYC) % GPR == 0 && GPR % GCYC == 0, "GPR is 4, 8, 12 or 16");
+    constexpr uint32_t RSTEP = 32 * GCYC / GPR, NU = GPR / GCYC;
+    uint32_t it_row[GCYC], it_grp[GCYC];
+#pragma unroll
+    for (uint32_t v = 0; v < GCYC; ++v) {
+        it_row[v] = (lane + 32 * v) / GPR;
+        it_grp[v] = (lane + 32 * v) % GPR;
+    }
 
+    // C offsets of the warp's rows and of the 16-byte groups of tile j's columns
+    auto tile_offsets = [&](uint32_t j) {
+        const WorkItem wi = decode_work(g, GETT_WB + (es + 2 * j) * GETT_WG, MMA_M);
+        const uint32_t m = wi.m0 + eq * 32 + lane;
+        row16[(j & 1) * 32 + lane] = m < g.M.size ? (uint32_t)(gett_offset_y(g.M, m) >> 2) : INVALID16;
+        for (uint32_t e = lane; e < TILE_N / 4; e += 32) {
+            const uint32_t col = Sh::col_of_group(e);
+            grp16[(j & 1) * EPI_GROUPS + e] =
+                wi.n0 + col < g.N.size ? (uint32_t)(gett_offset_y(g.N, wi.n0 + col) >> 2) : INVALID16;
+        }
+        __syncwarp();
+    };
+
+    // (elements outside C are not fetched: what the staging slots then hold is combined but never stored)
     auto prepare = [&](uint32_t cj) {
         if (cj < nchunk) {
             const uint32_t j = cj / NCH, ch = cj - j * NCH;
-            if (ch == 0) {
-                const WorkItem wi = decode_work(g, GETT_WB + (es + 2 * j) * GETT_WG, MMA_M);
-                int64_t rc = -1;
-                const uint32_t m = wi.m0 + eq * 32 + lane;
-                if (m < g.M.size)
-                    rc = gett_offset_y(g.M, m);
-                rowC_0 = (j & 1) ? rowC_0 : rc;
-                rowC_1 = (j & 1) ? rc : rowC_1;
-                for (uint32_t e = lane; e < TILE_N / 4; e += 32) {
-                    const uint32_t col = Sh::col_of_group(e);
-                    int64_t y = -1;
-                    if (wi.n0 + col < g.N.size)
-                        y = gett_offset_y(g.N, wi.n0 + col);
-                    grp[(j & 1) * EPI_GROUPS + e] = y;
-                }
-                __syncwarp();
-            }
+            if (ch == 0)
+                tile_offsets(j);
             if (rmw) {
-                const long long myrow = my_row(j);
                 const uint32_t dst = s_u32 + (cj & (DEPTH - 1)) * (32 * PITCH * 4);
-                const int64_t* gch = grp + (j & 1) * EPI_GROUPS + ch * GPR;
-                // four copies at a time: offsets first, then the copies back to back
+                const uint32_t* gt = grp16 + (j & 1) * EPI_GROUPS + ch * GPR;
+                const uint32_t* rt = row16 + (j & 1) * 32;
 #pragma unroll
-                for (uint32_t t0 = 0; t0 < GPR; t0 += 4) {
-                    const float* src[4];
-                    uint32_t d[4];
+                for (uint32_t v = 0; v < GCYC; ++v) {
+                    const uint32_t g16 = gt[it_grp[v]];
+                    const uint32_t d0 = dst + (it_row[v] * PITCH + 4 * it_grp[v]) * 4;
 #pragma unroll
-                    for (uint32_t k = 0; k < 4; ++k) {
-                        const uint32_t q = lane + 32 * (t0 + k), row = q / GPR, gi = q - row * GPR;
-                        const long long rc = __shfl_sync(FULL, myrow, row);
-                        const int64_t cn = gch[gi];
-                        src[k] = (rc >= 0 && cn >= 0) ? g.C + rc + cn : nullptr;
-                        d[k] = dst + (row * PITCH + 4 * gi) * 4;
+                    for (uint32_t u = 0; u < NU; ++u) {
+                        const uint32_t r16 = rt[it_row[v] + u * RSTEP];
+                        if (g16 != INVALID16 && r16 != INVALID16)
+                            ptx::cp_async_16(d0 + u * (RSTEP * PITCH * 4),
+                                             reinterpret_cast<const float4*>(g.C) + ((uint64_t)r16 + g16), 16u);
                     }
-#pragma unroll
-                    for (uint32_t k = 0; k < 4; ++k)
-                        ptx::cp_async_16(d[k], src[k] ? src[k] : g.C, src[k] ? 16u : 0u);
                 }
             }
         }
@@ -498,21 +527,30 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
 
     if (DEPTH == 2)
         prepare(0);
+    const bool tracer = eq == 0 && lane == 0;
     for (uint32_t ci = 0; ci < nchunk; ++ci) {
+        if (tracer)
+            GETT_TRACE(4 + es, 0);
         if (DEPTH == 2) {
             prepare(ci + 1);
+            if (tracer)
+                GETT_TRACE(4 + es, 5);
             ptx::cp_async_wait<1>(); // chunk ci's old C has landed (my copies) ...
         } else {
             prepare(ci);
             ptx::cp_async_wait<0>();
         }
         __syncwarp(); // ... and everybody else's
+        if (tracer)
+            GETT_TRACE(4 + es, 1);
         const uint32_t j = ci / NCH, ch = ci - j * NCH, buf = es; // tile es + 2j uses accumulator es
         if (ch == 0) {
             if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag, wait_ns))
                 break;
             ptx::tc_fence_after();
         }
+        if (tracer)
+            GETT_TRACE(4 + es, 2);
         float* Sb = S + (ci & (DEPTH - 1)) * (32 * PITCH);
         float* Srow = Sb + lane * PITCH;
         const uint32_t tacc = tmem_base + ((eq * 32u) << 16) + buf * 256;
@@ -571,27 +609,35 @@ __device__ __forceinline__ void epilogue_staged(const GettKernelArgs& g, SmemTab
             ptx::mbar_arrive(ptx::smem_u32(&T->acc_empty[buf]));
         }
         __syncwarp();
-        const long long myrow = my_row(j);
-        const int64_t* gch = grp + (j & 1) * EPI_GROUPS + ch * GPR;
-        // four groups at a time: staging reads first, then the global stores
+        if (tracer)
+            GETT_TRACE(4 + es, 3);
+        if (!GETT_DBG(g, 256)) { // (debug & 256: experiment, no store phase)
+            const uint32_t* gt = grp16 + (j & 1) * EPI_GROUPS + ch * GPR;
+            const uint32_t* rt = row16 + (j & 1) * 32;
 #pragma unroll
-        for (uint32_t t0 = 0; t0 < GPR && !GETT_DBG(g, 256); t0 += 4) { // (debug & 256: experiment, no store phase)
-            float4 val[4];
-            float* dstp[4];
+            for (uint32_t v = 0; v < GCYC; ++v) {
+                const uint32_t g16 = gt[it_grp[v]];
+                const float* src = Sb + it_row[v] * PITCH + 4 * it_grp[v];
+                // four groups at a time: staging reads first, then the global stores
 #pragma unroll
-            for (uint32_t k = 0; k < 4; ++k) {
-                const uint32_t q = lane + 32 * (t0 + k), row = q / GPR, gi = q - row * GPR;
-                const long long rc = __shfl_sync(FULL, myrow, row);
-                const int64_t cn = gch[gi];
-                dstp[k] = (rc >= 0 && cn >= 0 && !GETT_DBG(g, 2)) ? g.C + rc + cn : nullptr; // (debug & 2: no stores)
-                val[k] = *reinterpret_cast<const float4*>(Sb + row * PITCH + 4 * gi);
+                for (uint32_t u0 = 0; u0 < NU; u0 += 4) {
+                    float4 val[4];
+                    uint32_t r16[4];
+#pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k) {
+                        r16[k] = rt[it_row[v] + (u0 + k) * RSTEP];
+                        val[k] = *reinterpret_cast<const float4*>(src + (u0 + k) * (RSTEP * PITCH));
+                    }
+#pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k)
+                        if (g16 != INVALID16 && r16[k] != INVALID16 && !GETT_DBG(g, 2)) // (debug & 2: no stores)
+                            reinterpret_cast<float4*>(g.C)[(uint64_t)r16[k] + g16] = val[k];
+                }
             }
-#pragma unroll
-            for (uint32_t k = 0; k < 4; ++k)
-                if (dstp[k])
-                    *reinterpret_cast<float4*>(dstp[k]) = val[k];
         }
         __syncwarp(); // this staging buffer is free for the next prefetch into it
+        if (tracer)
+            GETT_TRACE(4 + es, 4);
     }
     ptx::cp_async_wait_all();
 }
@@ -686,6 +732,8 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
         for (; j < wi.nslab; j += ng) {
             const uint32_t it = first + j;
             const uint32_t k0 = wi.kbeg + j * TILE_K;
+            if (gl == 0)
+                GETT_TRACE(pg, 0);
             if (!all_tma) {
                 ptx::named_barrier(gbar, LANES); // previous slab's k table no longer read
                 if (gl < TILE_K) {
@@ -702,6 +750,8 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
                 }
                 ptx::named_barrier(gbar, LANES); // tables (rows and k) complete
             }
+            if (gl == 0)
+                GETT_TRACE(pg, 1);
             const uint32_t s = it % stages;
             // the slab's part of the TMA coordinates, before the wait for the stage
             int32_t* ckA = T->slabc[pg][0]; // (written and read by thread 0 of the group only)
@@ -721,6 +771,8 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
                 alive = false;
             if (!alive)
                 continue;
+            if (gl == 0)
+                GETT_TRACE(pg, 2);
             const uint32_t sa = stage0 + s * sbytes;
             const uint32_t fullbar = ptx::smem_u32(&T->full[s]);
             if (gl == 0 && tma_bytes && !GETT_DBG(g, 4)) {
@@ -818,6 +870,8 @@ __device__ __forceinline__ void producer_role(const GettKernelArgs& g, const Get
             }
             // full[s] hears from this thread when its copies for the slab have landed
             ptx::cp_async_mbar_arrive_noinc(fullbar);
+            if (gl == 0)
+                GETT_TRACE(pg, 3);
         }
         first += wi.nslab;
     }
@@ -923,8 +977,10 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                 // uses both (rows 0-127 in buffer 0, rows 128-255 in buffer 1)
                 const uint32_t buf = TWO_HALVES ? 0u : (local & 1);
                 const uint32_t par = TWO_HALVES ? (local & 1) : ((local >> 1) & 1);
+                GETT_TRACE(2, 0);
                 if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[buf]), par ^ 1, abort_flag, wait_ns))
                     break;
+                GETT_TRACE(2, 1);
                 if (TWO_HALVES && !ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[1]), par ^ 1, abort_flag, wait_ns))
                     break;
                 ptx::tc_fence_after();
@@ -935,6 +991,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                         alive = false;
                         break;
                     }
+                    GETT_TRACE(2, 2);
                     // the copies were generic-proxy writes; the tensor core reads through the
                     // async proxy, so order the two before issuing
                     ptx::fence_proxy_async_smem();
@@ -960,6 +1017,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                     ptx::umma_commit(ptx::smem_u32(&T->empty[s])); // stage reusable once these MMAs retire
 #endif
                 }
+                GETT_TRACE(2, 3);
                 if (alive) {
                     ptx::umma_commit(ptx::smem_u32(&T->acc_full[buf]));
                     if (TWO_HALVES)
@@ -1017,50 +1075,84 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                 colC[c] = y;
             }
             ptx::named_barrier(1 + es, EPI_SET_THREADS);
+            const bool row_ok = rowC >= 0;
+            const float alpha = g.alpha, beta = g.beta;
+            // beta != 0: the old values of C do not depend on the accumulator, so those of the
+            // first 16 columns are asked for before the wait for it, and those of every later
+            // group of 16 one group ahead of their use (two register buffers, A and B)
+            // (the same for every lane of the warp: the tensor-memory loads below are warp-wide
+            //  instructions and must not sit in branches that lanes take differently; a lane
+            //  whose row lies outside C fetches and stores nothing)
+            const bool rmw = beta != 0.f && !wi.partial && !GETT_DBG(g, 2);
+            float oldA[16], oldB[16];
+            auto fetch = [&](uint32_t c0, float (&old)[16]) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int64_t co = colC[c0 + i];
+                    old[i] = (row_ok && co >= 0) ? __ldcg(g.C + rowC + co) : 0.f;
+                }
+            };
+            if (rmw)
+                fetch(0, oldA);
             if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag, wait_ns))
                 alive = false;
             if (!alive)
                 continue; // keep the named barriers above matched, do nothing else
             ptx::tc_fence_after();
             const uint32_t taddr = tmem_base + ((eq * 32u) << 16) + buf * 256;
-            const bool row_ok = rowC >= 0;
-            const float alpha = g.alpha, beta = g.beta;
-            for (uint32_t c0 = 0; c0 < TILE_N; c0 += 16) {
-                uint32_t v[16];
-                ptx::tmem_ld_32x16(taddr + c0, v);
-                ptx::tmem_wait_ld();
-                if (!row_ok || GETT_DBG(g, 2)) // (debug & 2: experiment switch, no stores)
-                    continue;
-                if (wi.partial && g.stream_k) {
-                    // piece z of left-over tile r: a whole tile_m x TILE_N buffer [column][row]
-                    float* dst = g.ws + (((size_t)wi.r * g.sk_pmax + wi.z) * TILE_N + c0) * (size_t)g.tile_m +
-                                 (TWO_HALVES ? es * MMA_M : 0u) + et;
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        dst[(size_t)i * g.tile_m] = __uint_as_float(v[i]);
-                } else if (wi.partial) {
-                    float* dst = g.ws + ((size_t)wi.z * g.N.size + wi.n0 + c0) * g.M.size + wi.m0 + et;
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (wi.n0 + c0 + i < g.N.size)
-                            dst[(size_t)i * g.M.size] = __uint_as_float(v[i]);
-                } else {
+            if (rmw) {
+                auto step = [&](uint32_t c0, float (&old)[16], float (&nxt)[16]) {
+                    if (c0 + 16 < (uint32_t)TILE_N)
+                        fetch(c0 + 16, nxt);
+                    uint32_t v[16];
+                    ptx::tmem_ld_32x16(taddr + c0, v);
+                    ptx::tmem_wait_ld();
+                    if (!row_ok)
+                        return;
                     float* crow = g.C + rowC;
-                    int64_t co[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        co[i] = colC[c0 + i];
-                    if (beta != 0.f) {
-                        // all reads of the old C first, so their latencies overlap
-                        float old[16];
+                    for (int h = 0; h < 2; ++h) { // eight columns at a time: their offsets, then the stores
+                        int64_t co[8];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            old[i] = co[i] >= 0 ? __ldcg(crow + co[i]) : 0.f;
+                        for (int i = 0; i < 8; ++i)
+                            co[i] = colC[c0 + 8 * h + i];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
+                        for (int i = 0; i < 8; ++i)
                             if (co[i] >= 0)
-                                crow[co[i]] = fmaf(beta, old[i], alpha * __uint_as_float(v[i]));
+                                crow[co[i]] = fmaf(beta, old[8 * h + i], alpha * __uint_as_float(v[8 * h + i]));
+                    }
+                };
+                static_assert(TILE_N % 32 == 0, "two groups of 16 columns per turn");
+                for (uint32_t c0 = 0; c0 < TILE_N; c0 += 32) {
+                    step(c0, oldA, oldB);
+                    step(c0 + 16, oldB, oldA);
+                }
+            } else {
+                for (uint32_t c0 = 0; c0 < TILE_N; c0 += 16) {
+                    uint32_t v[16];
+                    ptx::tmem_ld_32x16(taddr + c0, v);
+                    ptx::tmem_wait_ld();
+                    if (!row_ok || GETT_DBG(g, 2)) // (debug & 2: experiment switch, no stores)
+                        continue;
+                    if (wi.partial && g.stream_k) {
+                        // piece z of left-over tile r: a whole tile_m x TILE_N buffer [column][row]
+                        float* dst = g.ws + (((size_t)wi.r * g.sk_pmax + wi.z) * TILE_N + c0) * (size_t)g.tile_m +
+                                     (TWO_HALVES ? es * MMA_M : 0u) + et;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            dst[(size_t)i * g.tile_m] = __uint_as_float(v[i]);
+                    } else if (wi.partial) {
+                        float* dst = g.ws + ((size_t)wi.z * g.N.size + wi.n0 + c0) * g.M.size + wi.m0 + et;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (wi.n0 + c0 + i < g.N.size)
+                                dst[(size_t)i * g.M.size] = __uint_as_float(v[i]);
                     } else {
+                        float* crow = g.C + rowC;
+                        int64_t co[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            co[i] = colC[c0 + i];
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
                             if (co[i] >= 0)
@@ -1148,3 +1240,17 @@ cudaError_t gett_launch_umma(const GettKernelArgs& args, const GettTmaMaps& maps
     return launch_tn<false, false>(args, maps, grid, smem, stream);
 }
 #endif // !GETT_UMMA_CLUSTER
+
+#if defined(GETT_EXPERIMENT) && !defined(GETT_UMMA_CLUSTER)
+// experiment builds: fetch (and reset) the time stamps; out holds 8 x 4096 values, n 8 counts
+extern "C" __attribute__((visibility("default"))) int gett_debug_trace(unsigned long long* out, unsigned int* n)
+{
+    if (cudaDeviceSynchronize() != cudaSuccess)
+        return -1;
+    if (cudaMemcpyFromSymbol(out, gett_trace_buf, sizeof(gett_trace_buf)) != cudaSuccess ||
+        cudaMemcpyFromSymbol(n, gett_trace_n, sizeof(gett_trace_n)) != cudaSuccess)
+        return -1;
+    const unsigned int zero[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    return cudaMemcpyToSymbol(gett_trace_n, zero, sizeof(zero)) == cudaSuccess ? 0 : -1;
+}
+#endif

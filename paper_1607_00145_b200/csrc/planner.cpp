@@ -15,6 +15,13 @@
 
 #include "gett_plan.h"
 
+// Longest contraction (fused K) for which a C that runs along A's stride-1 mode is moved to the
+// column side by exchanging the operands: beyond it the element-wise update of C hides behind the
+// next tile's main loop and the direct stores keep the whole operand ring.
+#ifndef GETT_EXCHANGE_MAX_K
+#define GETT_EXCHANGE_MAX_K 256
+#endif
+
 namespace {
 
 struct RawTensor {
@@ -553,6 +560,20 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
             for (int i = 0; i < (int)im.size(); ++i)
                 want = want && (i == unitCm || im[i].sC % 4 == 0);
         }
+        // 16-bit types, short contraction, C's stride-1 mode is A's own: the kernel's rows would
+        // run along C and each thread would update its row of C element by element, with
+        // nothing to hide that behind.  With the roles exchanged the mode leads the columns
+        // and C goes through the staged unpacking (whole 16-byte vectors, old values fetched
+        // ahead of the accumulator).
+        if (!want && (dtype == GETT_BF16_F32 || dtype == GETT_F16_F32) && unitCm >= 0 && unitAm == unitCm &&
+            ksz <= GETT_EXCHANGE_MAX_K && im[unitCm].ext % 8 == 0 && o.epilogue != GETT_EPI_DIRECT &&
+            o.tile_m != 256 && !(o.flags & GETT_OPT_NO_EXCHANGE)) { // (256-row tiles store directly)
+            want = true;
+            for (const GettMode& m : in)
+                want = want && m.sC % 4 == 0;
+            for (int i = 0; i < (int)im.size(); ++i)
+                want = want && (i == unitCm || im[i].sC % 4 == 0);
+        }
         if (want) {
             std::swap(im, in);
             for (std::vector<GettMode>* v : {&im, &in, &ik})
@@ -655,18 +676,28 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
     }
     p->tk = order_with_lead(ik, leadK);
     // 16-bit operands whose stride-1 modes are two different contracted modes u (A's) and v (B's):
-    // slabs of 8 indices of u times 8 consecutive indices of v (Sec. 3.2.1: a sub-tensor made
-    // of pieces of two modes).  A is then read in 16-byte pieces along u as usual; B is read
+    // slabs of 8 consecutive indices of u times 8 consecutive indices of v (Sec. 3.2.1: a
+    // sub-tensor made of pieces of two modes).  A is then read in 16-byte pieces along u as usual; B is read
     // in 16-byte pieces along v and its 8 x 8 blocks are transposed on the way (Sec. 3.2.2).
     bool k_transposed = false;
     if (dtype == GETT_BF16_F32 || dtype == GETT_F16_F32) {
         const int uA = find_unit(ik, 0), uB = find_unit(ik, 1);
         if (uA >= 0 && uB >= 0 && uA != uB && ik[uA].ext % 8 == 0 && ik[uB].ext % 8 == 0) {
+            // Consecutive slabs first walk f blocks of u under the same block of v, then the
+            // blocks of v: the 16-byte pieces that share a 32-byte sector (a 128-byte line) of
+            // A are asked for by neighbouring slabs, those of B at most f slabs apart, while
+            // the line is still in L2.
+            const int64_t eu = ik[uA].ext, ev = ik[uB].ext;
+            const int64_t f = eu % 64 == 0 ? 8 : eu % 32 == 0 ? 4 : eu % 16 == 0 ? 2 : 1;
             std::vector<GettDigit> t;
             t.push_back({uA, 8, 1, 0});
-            t.push_back({uB, ik[uB].ext, 1, 0});
-            if (ik[uA].ext > 8)
-                t.push_back({uA, ik[uA].ext / 8, 8, 0});
+            t.push_back({uB, 8, 1, 0});
+            if (f > 1)
+                t.push_back({uA, f, 8, 0});
+            if (ev > 8)
+                t.push_back({uB, ev / 8, 8, 0});
+            if (eu > 8 * f)
+                t.push_back({uA, eu / (8 * f), 8 * f, 0});
             for (int i = 0; i < (int)ik.size(); ++i)
                 if (i != uA && i != uB)
                     t.push_back({i, ik[i].ext, 1, 0});
@@ -865,6 +896,16 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
             else if (p->N.ndig >= 1 && p->N.sY[0] == 1 && p->N.ext[0] % 4 == 0 && others_mult4(0))
                 staged_cv = 1;
         }
+        {
+            // the staged epilogue keeps C offsets in 32 bits, in units of 16 bytes
+            int64_t maxC = 0;
+            for (const GettMode& m : im)
+                maxC += (m.ext - 1) * m.sC;
+            for (const GettMode& m : in)
+                maxC += (m.ext - 1) * m.sC;
+            if ((maxC >> 2) >= (int64_t)0xFFFFFFF0ll)
+                staged_cv = 0;
+        }
         if (o.epilogue == GETT_EPI_DIRECT)
             staged_cv = 0;
         if (o.epilogue == GETT_EPI_STAGED && !staged_cv)
@@ -898,6 +939,31 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
                 }
             }
         }
+        // A small output with a long contraction is cut along K until every SM has a piece
+        // (below), so the tile count no longer matters; what the tile shape then decides is
+        // how often the operands are delivered: A once per column of tiles, B once per row
+        // of tiles, padding included.  Take the shape that moves the fewest bytes.
+        int tm_few = 0;
+        if (o.tile_n == 0 && staged_cv != 8 && o.split_k != 1 && p->K.size >= 8 * 64 &&
+            (uint64_t)ceil_div(p->M.size, 128) * ceil_div(p->N.size, (uint32_t)tn) * 2 <= (uint64_t)sms) {
+            uint64_t best = UINT64_MAX;
+            for (int cm : {128, 256})
+                for (int cn : {64, 128, 192, 256}) {
+                    if (cm == 256 && (cn != 256 || staged_cv || (o.tile_m && o.tile_m != 256)))
+                        continue;
+                    if (cm == 128 && o.tile_m == 256)
+                        continue;
+                    const uint64_t rows = ceil_div(p->M.size, (uint32_t)cm), cols = ceil_div(p->N.size, (uint32_t)cn);
+                    if (rows * cols * 2 > (uint64_t)sms)
+                        continue;
+                    const uint64_t moved = cols * rows * cm + rows * cols * cn; // x K elements
+                    if (moved < best) {
+                        best = moved;
+                        tn = cn;
+                        tm_few = cm;
+                    }
+                }
+        }
         if (tn != 64 && tn != 128 && tn != 192 && tn != 256)
             return GETT_ERR_UNSUPPORTED;
         const int smem_limit = 227 * 1024;
@@ -920,7 +986,7 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         int tmh = o.tile_m;
         if (tmh == 0) {
             const uint64_t t256 = (uint64_t)ceil_div(p->M.size, 256) * ceil_div(p->N.size, 256);
-            tmh = (tn == 256 && !staged && p->K.size >= 2048 && t256 >= 2ull * sms) ? 256 : 128;
+            tmh = tm_few ? tm_few : (tn == 256 && !staged && p->K.size >= 2048 && t256 >= 2ull * sms) ? 256 : 128;
         }
         if (tmh == 256 && (tn != 256 || staged))
             return GETT_ERR_UNSUPPORTED;

@@ -120,6 +120,24 @@ def test_256_row_tiles(spec, sizes):
 
 
 @pytest.mark.parametrize("spec,sizes", [
+    ("C[m,n] = A[m,k] * B[k,n]", dict(m=264, n=200, k=88)),
+    ("C[m,n] = A[m,k] * B[n,k]", dict(m=136, n=328, k=200)),
+    ("C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]", dict(m0=24, m1=9, n0=7, n1=24, k0=8, k1=11)),
+])
+def test_short_contractions_unpack_through_the_column_side(spec, sizes):
+    """C runs along A's own stride-1 mode and K is short: the operands change places so that C goes
+    through the staged unpacking; with the sides kept (direct stores, old values of C fetched one
+    group of columns ahead) the result must pass as well."""
+    con = parse_spec(spec, sizes)
+    for dtype in (BF16_F32, F16_F32):
+        for alpha, beta in [(1.0, 0.0), (0.5, -2.0)]:
+            ratio, info = parity_case(con, dtype, "normal", 23, alpha, beta, repeat=2)
+            assert info.swapped == 1 and info.epilogue == g.GETT_EPI_STAGED and info.path == g.GETT_PATH_UMMA
+            ratio, info = parity_case(con, dtype, "normal", 23, alpha, beta, repeat=2, flags=g.GETT_OPT_NO_EXCHANGE)
+            assert info.swapped == 0 and info.epilogue == g.GETT_EPI_DIRECT
+
+
+@pytest.mark.parametrize("spec,sizes", [
     ("C[m,n] = A[m,k] * B[k,n]", dict(m=200, n=136, k=88)),                        # A free-major, B K-major
     ("C[m,n] = A[k,m] * B[n,k]", dict(m=136, n=264, k=72)),                        # A K-major, B free-major
     ("C[n0,m2,m1,n2,m0,n1] = A[m1,k,m0,m2] * B[n2,n0,k,n1]",
@@ -159,9 +177,12 @@ def test_atom_tma_loader_against_gather_loader_and_oracle(spec, sizes):
     tiles, and with a ragged last tile in both directions."""
     con = parse_spec(spec, sizes)
     for dtype in (BF16_F32, F16_F32):
-        ratio, info = parity_case(con, dtype, "normal", 51, 1.0, 0.5, repeat=2)
+        # (a short contraction whose C runs along A's stride-1 mode would exchange its operands for
+        #  the staged unpacking, which keeps the gather: the atoms are tested with the sides kept)
+        ratio, info = parity_case(con, dtype, "normal", 51, 1.0, 0.5, repeat=2, flags=g.GETT_OPT_NO_EXCHANGE)
         assert info.path == g.GETT_PATH_UMMA
         assert g.GETT_LOAD_TMA_FREE in (info.loader_a, info.loader_b)
+        parity_case(con, dtype, "normal", 51, 1.0, 0.5)
         ratio2, info2 = parity_case(con, dtype, "normal", 51, 1.0, 0.5, flags=g.GETT_OPT_NO_TMA)
         assert info2.loader_a == g.GETT_LOAD_VEC_FREE and info2.loader_b == g.GETT_LOAD_VEC_FREE
     parity_case(con, BF16_F32, "normal", 51, -0.5, 0.0, repeat=2, split_k=2)
@@ -273,9 +294,12 @@ def test_stream_k_shares_of_the_tile_slab_space(spec, sizes, opts):
     con = parse_spec(spec, sizes)
     for dtype in (BF16_F32, F16_F32):
         for alpha, beta in [(1.0, 0.5), (-0.5, 0.0)]:
-            ratio, info = parity_case(con, dtype, "normal", 71, alpha, beta, repeat=2, flags=g.GETT_OPT_STREAMK, **opts)
+            # (sides kept: these short contractions would otherwise take the staged unpacking, which has no pieces)
+            ratio, info = parity_case(con, dtype, "normal", 71, alpha, beta, repeat=2,
+                                      flags=g.GETT_OPT_STREAMK | g.GETT_OPT_NO_EXCHANGE, **opts)
             assert info.stream_k == 1 and info.split_k == 1 and info.workspace_bytes > 0
-    ratio, info = parity_case(con, BF16_F32, "normal", 71, 1.0, 0.5, flags=g.GETT_OPT_NO_STREAMK, **opts)
+    ratio, info = parity_case(con, BF16_F32, "normal", 71, 1.0, 0.5,
+                              flags=g.GETT_OPT_NO_STREAMK | g.GETT_OPT_NO_EXCHANGE, **opts)
     assert info.stream_k == 0
 
 

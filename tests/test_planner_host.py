@@ -152,6 +152,27 @@ def test_operands_are_exchanged_when_c_runs_along_a_mode_of_a_that_is_not_a_s_ow
     assert g.Plan(workload("cfg3").contraction, g.GETT_F32).info.swapped == 0
 
 
+def test_short_16_bit_contractions_move_c_s_mode_to_the_column_side():
+    """C runs along A's own stride-1 mode and the contraction is short: each thread of the tensor-core
+    kernel would update its row of C element by element with no main loop to hide that behind, so the
+    operands change places and C goes through the staged unpacking.  Long contractions, fp32 and
+    plans with the flag keep their sides."""
+    spec = "C[m0,n0,m1,n1] = A[m0,k0,m1,k1] * B[n1,k1,n0,k0]"
+    short = parse_spec(spec, dict(m0=96, m1=16, n0=16, n1=96, k0=8, k1=32))      # K = 256
+    i = _tables_match(short, g.GETT_BF16_F32).info
+    assert i.swapped == 1 and i.epilogue == g.GETT_EPI_STAGED and (i.M, i.N, i.K) == short.mnk()
+    assert g.Plan(short, g.GETT_BF16_F32, flags=g.GETT_OPT_NO_EXCHANGE).info.swapped == 0
+    assert g.Plan(short, g.GETT_BF16_F32, epilogue=g.GETT_EPI_DIRECT).info.swapped == 0
+    assert g.Plan(short, g.GETT_F32).info.swapped == 0
+    long_ = parse_spec(spec, dict(m0=96, m1=16, n0=16, n1=96, k0=8, k1=128))     # K = 1024
+    assert g.Plan(long_, g.GETT_BF16_F32).info.swapped == 0
+    # a mode of C whose stride is not a multiple of four elements rules the 16-byte vectors out
+    gemm = parse_spec("C[m,n] = A[m,k] * B[k,n]", dict(m=96, n=64, k=64))
+    assert g.Plan(gemm, g.GETT_BF16_F32).info.swapped == 1
+    padded = parse_spec("C[m,n] = A[m,k] * B[k,n]", dict(m=96, n=64, k=64), strides={"C": [1, 98]})
+    assert g.Plan(padded, g.GETT_BF16_F32).info.swapped == 0
+
+
 def test_split_k_planning():
     con = workload("splitk").contraction
     auto = g.Plan(con, g.GETT_F32)
@@ -165,6 +186,23 @@ def test_split_k_planning():
     assert g.Plan(workload("cfg3").contraction, g.GETT_F32, path=g.GETT_PATH_SIMT,
                   split_k=2).info.split_k == 2
     assert g.Plan(workload("cfg3").contraction, g.GETT_F32).info.split_k == 1
+
+
+def test_sliced_contractions_take_the_tile_that_moves_the_fewest_operand_bytes():
+    """384 x 376 x 147456 is cut along K until every SM has a piece, so the tile shape only decides how
+    often A and B are delivered: 128 x 192 tiles deliver (2 + 3) x 384 rows of K, 128 x 64 tiles
+    (6 + 3) x 384, 256 x 256 tiles (2 + 2) x 512."""
+    for key in ("splitk", "splitk_vec"):
+        i = g.Plan(workload(key).contraction, g.GETT_BF16_F32).info
+        assert (i.tile_m, i.tile_n) == (128, 192) and i.tiles == 6 and i.split_k == 24 and i.grid == 144
+        # an explicit width is kept
+        assert g.Plan(workload(key).contraction, g.GETT_BF16_F32, tile_n=64).info.tile_n == 64
+    # square 512 x 512: 256 x 256 tiles deliver (2 + 2) x 512 rows, 128 x 256 (2 + 4) x 512
+    con = parse_spec("C[m,n] = A[k,m] * B[k,n]", dict(m=512, n=512, k=65536))
+    i = g.Plan(con, g.GETT_BF16_F32).info
+    assert (i.tile_m, i.tile_n, i.tiles) == (256, 256, 4) and i.split_k > 1
+    # with enough tiles for the machine the rule stays out of it
+    assert g.Plan(workload("cfg4").contraction, g.GETT_BF16_F32).info.split_k == 1
 
 
 def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
