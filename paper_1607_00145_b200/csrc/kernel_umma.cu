@@ -99,7 +99,7 @@ struct alignas(16) SmemTables { // the staging rows that follow it hold 128-bit 
 static_assert(sizeof(SmemTables) % 16 == 0, "staging area must stay 16-byte aligned");
 
 // Time stamps of CTA 0's roles (experiment builds only, opts.experiment & 4096): role = producer
-// group 0 / 1, 2 = MMA issuer, 4 / 5 = first warp of epilogue set 0 / 1; one thread per role writes.
+// group 0 .. 3, 6 = MMA issuer, 4 / 5 = first warp of epilogue set 0 / 1; one thread per role writes.
 #ifdef GETT_EXPERIMENT
 __device__ unsigned long long gett_trace_buf[8][4096];
 __device__ unsigned int gett_trace_n[8];
@@ -908,7 +908,10 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
             // the slab's producers (twice each with the transposing loader: once for their asynchronous
             // copies, once for their ordinary stores)
             ptx::mbar_init(ptx::smem_u32(&T->full[s]),
-                           (g.prod_groups == 1 ? PROD_THREADS : GROUP_LANES) * (B_TRANS ? 2 : 1));
+                           (g.prod_groups == 1                        ? PROD_THREADS
+                            : g.prod_groups == 2 && PROD_GROUPS == 4 ? 2 * GROUP_LANES
+                                                                     : GROUP_LANES) *
+                               (B_TRANS ? 2 : 1));
 #ifdef GETT_UMMA_CLUSTER
             ptx::mbar_init(ptx::smem_u32(&T->empty[s]), 2); // both CTAs of the pair are done with the stage
 #else
@@ -949,6 +952,17 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
             else
                 producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, PROD_THREADS, false, B_TRANS>(
                     g, tm, T, stage0, stages, total_work, abort_flag, 0, 1, threadIdx.x - PROD_WARP0 * 32, 3);
+        } else if (ng == 2 && PROD_GROUPS == 4) {
+            // a ring of two stages: two groups of twice the width, so that no producer warp idles
+            constexpr uint32_t WPG = 2 * WARPS_PER_GROUP;
+            const uint32_t pg = (warp - PROD_WARP0) / WPG;
+            const uint32_t gl = threadIdx.x - (PROD_WARP0 + pg * WPG) * 32;
+            if (hybrid)
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, 2 * GROUP_LANES, true, B_TRANS>(
+                    g, tm, T, stage0, stages, total_work, abort_flag, pg, ng, gl, 3 + pg);
+            else
+                producer_role<A_VEC_K, B_VEC_K, TILE_N, TILE_M, 2 * GROUP_LANES, false, B_TRANS>(
+                    g, tm, T, stage0, stages, total_work, abort_flag, pg, ng, gl, 3 + pg);
         } else {
             const uint32_t pg = (warp - PROD_WARP0) / WARPS_PER_GROUP;
             const uint32_t gl = threadIdx.x - (PROD_WARP0 + pg * WARPS_PER_GROUP) * 32;
@@ -977,10 +991,10 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                 // uses both (rows 0-127 in buffer 0, rows 128-255 in buffer 1)
                 const uint32_t buf = TWO_HALVES ? 0u : (local & 1);
                 const uint32_t par = TWO_HALVES ? (local & 1) : ((local >> 1) & 1);
-                GETT_TRACE(2, 0);
+                GETT_TRACE(6, 0);
                 if (!ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[buf]), par ^ 1, abort_flag, wait_ns))
                     break;
-                GETT_TRACE(2, 1);
+                GETT_TRACE(6, 1);
                 if (TWO_HALVES && !ptx::mbar_wait(ptx::smem_u32(&T->acc_empty[1]), par ^ 1, abort_flag, wait_ns))
                     break;
                 ptx::tc_fence_after();
@@ -991,7 +1005,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                         alive = false;
                         break;
                     }
-                    GETT_TRACE(2, 2);
+                    GETT_TRACE(6, 2);
                     // the copies were generic-proxy writes; the tensor core reads through the
                     // async proxy, so order the two before issuing
                     ptx::fence_proxy_async_smem();
@@ -1017,7 +1031,7 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
                     ptx::umma_commit(ptx::smem_u32(&T->empty[s])); // stage reusable once these MMAs retire
 #endif
                 }
-                GETT_TRACE(2, 3);
+                GETT_TRACE(6, 3);
                 if (alive) {
                     ptx::umma_commit(ptx::smem_u32(&T->acc_full[buf]));
                     if (TWO_HALVES)
@@ -1094,11 +1108,15 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
             };
             if (rmw)
                 fetch(0, oldA);
+            if (et == 0)
+                GETT_TRACE(4 + es, 0);
             if (alive && !ptx::mbar_wait(ptx::smem_u32(&T->acc_full[buf]), j & 1, abort_flag, wait_ns))
                 alive = false;
             if (!alive)
                 continue; // keep the named barriers above matched, do nothing else
             ptx::tc_fence_after();
+            if (et == 0)
+                GETT_TRACE(4 + es, 1);
             const uint32_t taddr = tmem_base + ((eq * 32u) << 16) + buf * 256;
             if (rmw) {
                 auto step = [&](uint32_t c0, float (&old)[16], float (&nxt)[16]) {
@@ -1162,6 +1180,8 @@ gett_umma_kernel(const __grid_constant__ GettKernelArgs g, const __grid_constant
             }
             ptx::tc_fence_before();
             ptx::mbar_arrive(ptx::smem_u32(&T->acc_empty[buf]));
+            if (et == 0)
+                GETT_TRACE(4 + es, 2);
         }
     }
 
