@@ -59,9 +59,13 @@ __device__ __forceinline__ void load_operand(const char* __restrict__ base, uint
     }
     constexpr int PIECES = R * TK / 4;
     constexpr int NP = (PIECES + NT - 1) / NT;
-    if (L == GETT_LOAD_VEC_K) {
+    if (L == GETT_LOAD_VEC_K || L == GETT_LOAD_VEC_KT) {
         const uint32_t kc = tid & 7;
-        const uint32_t k1 = kTab[kc * 4];
+        // VEC_KT: the 16-byte pieces run along K's SECOND digit (the slab is 4 indices of the
+        // first digit x 8 of the second, first fastest): piece kc = 4 j + c starts at k = c + 16 j
+        // and holds second-digit indices 4 j .. 4 j + 3 of first-digit index c, i.e. the
+        // transpose of what slots 4 j .. 4 j + 3 must hold; transpose_kt() puts that right.
+        const uint32_t k1 = kTab[L == GETT_LOAD_VEC_KT ? (kc & 3) + 16 * (kc >> 2) : kc * 4];
 #pragma unroll
         for (int p = 0; p < NP; ++p) {
             const uint32_t m = (tid >> 3) + (NT / 8) * p;
@@ -88,6 +92,26 @@ __device__ __forceinline__ void load_operand(const char* __restrict__ base, uint
     }
 }
 
+// In-place transposition of the 4 x 4 blocks of a [row][k] tile loaded with VEC_KT (packing
+// as a transposition, Sec. 3.2.2, at the granularity of one 16-byte vector): block j of a row
+// occupies slots 4 j .. 4 j + 3; before, slot 4 j + c holds (c; d = 4 j .. 4 j + 3), after,
+// slot 4 j + dd holds (c = 0 .. 3; d = 4 j + dd) = k 4 (4 j + dd) .. + 3.
+template <int R, int NT>
+__device__ __forceinline__ void transpose_kt(char* tile, int tid)
+{
+    for (int b = tid; b < 2 * R; b += NT) {
+        const uint32_t row = (uint32_t)b >> 1, j = (uint32_t)b & 1, sw = (row >> 2) & 7;
+        float4 v[4];
+#pragma unroll
+        for (uint32_t c = 0; c < 4; ++c)
+            v[c] = *reinterpret_cast<const float4*>(tile + row * 128 + (((4 * j + c) ^ sw) << 4));
+        *reinterpret_cast<float4*>(tile + row * 128 + (((4 * j + 0) ^ sw) << 4)) = make_float4(v[0].x, v[1].x, v[2].x, v[3].x);
+        *reinterpret_cast<float4*>(tile + row * 128 + (((4 * j + 1) ^ sw) << 4)) = make_float4(v[0].y, v[1].y, v[2].y, v[3].y);
+        *reinterpret_cast<float4*>(tile + row * 128 + (((4 * j + 2) ^ sw) << 4)) = make_float4(v[0].z, v[1].z, v[2].z, v[3].z);
+        *reinterpret_cast<float4*>(tile + row * 128 + (((4 * j + 3) ^ sw) << 4)) = make_float4(v[0].w, v[1].w, v[2].w, v[3].w);
+    }
+}
+
 // Fragment of F (4 or 8, or 2) rows for 4 consecutive k from a [row][k] swizzled tile.
 template <int F>
 __device__ __forceinline__ void frag_kmajor(const char* tile, const uint32_t (&rows)[F], uint32_t sw,
@@ -107,7 +131,8 @@ template <int LA, int LB, int TN, int TM>
 __global__ void __launch_bounds__(2 * TM, 256 / TM) gett_ffma_kernel(const __grid_constant__ GettKernelArgs g)
 {
     constexpr int NT = 2 * TM;
-    constexpr bool A_K = LA == GETT_LOAD_VEC_K, B_K = LB == GETT_LOAD_VEC_K; // staged [row][k]
+    constexpr bool B_KT = LB == GETT_LOAD_VEC_KT;
+    constexpr bool A_K = LA == GETT_LOAD_VEC_K, B_K = LB == GETT_LOAD_VEC_K || B_KT; // staged [row][k]
     constexpr int FN = TN / 16;                 // columns per thread (8 or 2)
     constexpr int STAGE = ffma_stage_bytes<TM, TN>();
     extern __shared__ __align__(128) uint8_t smem[];
@@ -246,6 +271,10 @@ __global__ void __launch_bounds__(2 * TM, 256 / TM) gett_ffma_kernel(const __gri
         fill_ktab(slab + stages); // for the issue of the next iteration
         const char* As = reinterpret_cast<const char*>(smem) + (slab % stages) * STAGE;
         const char* Bs = As + TM * TK * 4;
+        if (B_KT) { // B's rows have landed transposed block by block
+            transpose_kt<TN, NT>(reinterpret_cast<char*>(smem) + (slab % stages) * STAGE + TM * TK * 4, tid);
+            __syncthreads();
+        }
 #pragma unroll
         for (int k4 = 0; k4 < TK / 4 && !GETT_DBG(g, 64); ++k4) { // (debug & 64: experiment, no math)
             float a[8][4], b[FN][4];
@@ -453,6 +482,12 @@ cudaError_t launch_tn(const GettKernelArgs& args, int grid, int smem, cudaStream
 template <int LA>
 cudaError_t launch_b(const GettKernelArgs& args, int grid, int smem, cudaStream_t stream)
 {
+    if (args.loader_b == GETT_LOAD_VEC_KT) { // (planned only together with a K-major A)
+        if constexpr (LA == GETT_LOAD_VEC_K)
+            return launch_tn<LA, GETT_LOAD_VEC_KT>(args, grid, smem, stream);
+        else
+            return cudaErrorInvalidValue;
+    }
     switch (args.loader_b) {
     case GETT_LOAD_VEC_K: return launch_tn<LA, GETT_LOAD_VEC_K>(args, grid, smem, stream);
     case GETT_LOAD_VEC_FREE: return launch_tn<LA, GETT_LOAD_VEC_FREE>(args, grid, smem, stream);

@@ -675,29 +675,31 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         }
     }
     p->tk = order_with_lead(ik, leadK);
-    // 16-bit operands whose stride-1 modes are two different contracted modes u (A's) and v (B's):
-    // slabs of 8 consecutive indices of u times 8 consecutive indices of v (Sec. 3.2.1: a
-    // sub-tensor made of pieces of two modes).  A is then read in 16-byte pieces along u as usual; B is read
-    // in 16-byte pieces along v and its 8 x 8 blocks are transposed on the way (Sec. 3.2.2).
+    // Operands whose stride-1 modes are two different contracted modes u (A's) and v (B's):
+    // slabs of W consecutive indices of u times 8 consecutive indices of v (Sec. 3.2.1: a
+    // sub-tensor made of pieces of two modes), W = one 16-byte vector (8 elements of 16 bits,
+    // 4 of 32).  A is then read in 16-byte pieces along u as usual; B is read in 16-byte
+    // pieces along v and its W x W blocks are transposed on the way (Sec. 3.2.2).
     bool k_transposed = false;
-    if (dtype == GETT_BF16_F32 || dtype == GETT_F16_F32) {
+    if (dtype == GETT_BF16_F32 || dtype == GETT_F16_F32 || dtype == GETT_F32) {
+        const int64_t W = dtype == GETT_F32 ? 4 : 8;
         const int uA = find_unit(ik, 0), uB = find_unit(ik, 1);
-        if (uA >= 0 && uB >= 0 && uA != uB && ik[uA].ext % 8 == 0 && ik[uB].ext % 8 == 0) {
+        if (uA >= 0 && uB >= 0 && uA != uB && ik[uA].ext % W == 0 && ik[uB].ext % 8 == 0) {
             // Consecutive slabs first walk f blocks of u under the same block of v, then the
             // blocks of v: the 16-byte pieces that share a 32-byte sector (a 128-byte line) of
             // A are asked for by neighbouring slabs, those of B at most f slabs apart, while
             // the line is still in L2.
             const int64_t eu = ik[uA].ext, ev = ik[uB].ext;
-            const int64_t f = eu % 64 == 0 ? 8 : eu % 32 == 0 ? 4 : eu % 16 == 0 ? 2 : 1;
+            const int64_t f = eu % (8 * W) == 0 ? 8 : eu % (4 * W) == 0 ? 4 : eu % (2 * W) == 0 ? 2 : 1;
             std::vector<GettDigit> t;
-            t.push_back({uA, 8, 1, 0});
+            t.push_back({uA, W, 1, 0});
             t.push_back({uB, 8, 1, 0});
             if (f > 1)
-                t.push_back({uA, f, 8, 0});
+                t.push_back({uA, f, W, 0});
             if (ev > 8)
                 t.push_back({uB, ev / 8, 8, 0});
-            if (eu > 8 * f)
-                t.push_back({uA, eu / (8 * f), 8 * f, 0});
+            if (eu > W * f)
+                t.push_back({uA, eu / (W * f), W * f, 0});
             for (int i = 0; i < (int)ik.size(); ++i)
                 if (i != uA && i != uB)
                     t.push_back({i, ik[i].ext, 1, 0});
@@ -743,13 +745,13 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
                     : vec_ok(p->K, false, p->N, true, vec) ? GETT_LOAD_VEC_K
                                                            : GETT_LOAD_SCALAR;
     if (k_transposed && info.loader_a == GETT_LOAD_VEC_K && info.loader_b == GETT_LOAD_SCALAR && p->K.ndig >= 2 &&
-        p->K.ext[0] == 8 && p->K.sY[1] == 1 && p->K.ext[1] % 8 == 0) {
+        p->K.ext[0] == vec && p->K.sY[1] == 1 && p->K.ext[1] % 8 == 0) {
         // B in 16-byte pieces along K's second digit: every other stride of B must keep them aligned
-        bool ok = p->K.sY[0] % 8 == 0;
+        bool ok = p->K.sY[0] % vec == 0;
         for (int d = 2; d < p->K.ndig; ++d)
-            ok = ok && p->K.sY[d] % 8 == 0;
+            ok = ok && p->K.sY[d] % vec == 0;
         for (int d = 0; d < p->N.ndig; ++d)
-            ok = ok && p->N.sX[d] % 8 == 0;
+            ok = ok && p->N.sX[d] % vec == 0;
         if (ok)
             info.loader_b = GETT_LOAD_VEC_KT;
     }

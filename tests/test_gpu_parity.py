@@ -278,6 +278,28 @@ def test_transposing_loader_for_two_different_contracted_stride1_modes(spec, siz
     parity_case(con, BF16_F32, "normal", 61, 1.0, 0.0, path=g.GETT_PATH_SIMT)
 
 
+@pytest.mark.parametrize("spec,sizes", [
+    ("C[a,b] = A[c,a,d] * B[d,c,b]", dict(a=136, b=72, c=24, d=40)),               # ab-cad-dcb
+    ("C[a,b,c,d] = A[e,a,f,b] * B[f,d,e,c]", dict(a=24, b=9, c=7, d=24, e=12, f=24)),  # abcd-eafb-fdec, u = 3 blocks of 4
+    ("C[a,b] = A[c,a,d,e] * B[d,e,c,b]", dict(a=136, b=72, c=4, d=16, e=5)),       # a third contracted mode, u of extent 4
+    ("C[a,b] = A[c,a,d] * B[d,c,b]", dict(a=40, b=136, c=64, d=8)),                # eight blocks of u per block of v
+])
+def test_fp32_transposing_loader(spec, sizes):
+    """fp32 operands whose stride-1 modes are two different contracted modes: slabs of 4 x 8 indices
+    of the two modes, B read in 16-byte pieces along its own mode and transposed in 4 x 4 blocks in
+    shared memory (both tile heights, narrow tiles, split-K, ragged tiles), against the oracle and
+    against the element-wise gather."""
+    con = parse_spec(spec, sizes)
+    for alpha, beta in [(1.0, 0.5), (-0.5, 0.0)]:
+        ratio, info = parity_case(con, F32, "normal", 67, alpha, beta, repeat=2)
+        assert info.path == g.GETT_PATH_FFMA
+        assert (info.loader_a, info.loader_b) == (g.GETT_LOAD_VEC_K, g.GETT_LOAD_VEC_KT)
+    parity_case(con, F32, "normal", 67, 1.0, 0.0, repeat=2, tile_m=64)
+    parity_case(con, F32, "normal", 67, 1.0, 0.0, repeat=2, tile_n=32)
+    parity_case(con, F32, "normal", 67, 1.0, 1.0, repeat=2, split_k=3)
+    parity_case(con, F32, "normal", 67, 1.0, 0.0, path=g.GETT_PATH_SIMT)
+
+
 @pytest.mark.parametrize("spec,sizes,opts", [
     # 15 x 11 = 165 tiles of 128 x 64 on 148 SMs, 5 slabs (the last one ragged): TMA boxes
     ("C[m,n] = A[m,k] * B[k,n]", dict(m=1904, n=696, k=296), dict(tile_m=128, tile_n=64)),
