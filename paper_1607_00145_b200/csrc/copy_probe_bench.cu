@@ -42,6 +42,11 @@ __global__ void copy_probe_kernel(const char* __restrict__ g, int pattern, int i
         default: off = lane * 16; break;
         }
         copy16(s0 + warp * 1024 + (it & 1) * 512 + lane * 16, g + base + off);
+        // two copies per thread in flight, each to a destination of its own: a copy whose
+        // destination is overwritten by a later one while it is still in flight need not be
+        // carried out, which would make the byte counts depend on timing
+        if (it & 1)
+            asm volatile("cp.async.wait_all;" ::: "memory");
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
 }
