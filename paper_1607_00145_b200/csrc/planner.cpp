@@ -565,7 +565,9 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         // nothing to hide that behind.  With the roles exchanged the mode leads the columns
         // and C goes through the staged unpacking (whole 16-byte vectors, old values fetched
         // ahead of the accumulator).
-        if (!want && (dtype == GETT_BF16_F32 || dtype == GETT_F16_F32) && unitCm >= 0 && unitAm == unitCm &&
+        // (the same when A's stride-1 mode is a contracted one: I_m is then ordered for C anyway)
+        if (!want && (dtype == GETT_BF16_F32 || dtype == GETT_F16_F32) && unitCm >= 0 &&
+            (unitAm == unitCm || unitAm < 0) &&
             ksz <= GETT_EXCHANGE_MAX_K && im[unitCm].ext % 8 == 0 && o.epilogue != GETT_EPI_DIRECT &&
             o.tile_m != 256 && !(o.flags & GETT_OPT_NO_EXCHANGE)) { // (256-row tiles store directly)
             want = true;

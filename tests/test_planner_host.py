@@ -167,6 +167,11 @@ def test_short_16_bit_contractions_move_c_s_mode_to_the_column_side():
     long_ = parse_spec(spec, dict(m0=96, m1=16, n0=16, n1=96, k0=8, k1=128))     # K = 1024
     assert g.Plan(long_, g.GETT_BF16_F32).info.swapped == 0
     # a mode of C whose stride is not a multiple of four elements rules the 16-byte vectors out
+    # A's own stride-1 mode is a contracted one: I_m is ordered for C anyway, the same applies
+    kmaj = parse_spec("C[a,b,c,d,e,f] = A[g,d,a,b] * B[e,f,g,c]", dict(a=24, b=16, c=16, d=24, e=24, f=16, g=24))
+    i = _tables_match(kmaj, g.GETT_BF16_F32).info
+    assert i.swapped == 1 and i.epilogue == g.GETT_EPI_STAGED
+    assert g.Plan(kmaj, g.GETT_BF16_F32, flags=g.GETT_OPT_NO_EXCHANGE).info.epilogue == g.GETT_EPI_DIRECT
     gemm = parse_spec("C[m,n] = A[m,k] * B[k,n]", dict(m=96, n=64, k=64))
     assert g.Plan(gemm, g.GETT_BF16_F32).info.swapped == 1
     padded = parse_spec("C[m,n] = A[m,k] * B[k,n]", dict(m=96, n=64, k=64), strides={"C": [1, 98]})
