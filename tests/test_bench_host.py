@@ -50,3 +50,22 @@ def test_replica_aggregation_on_two_gloo_ranks(tmp_path):
         out, err = p.communicate(timeout=180)
         assert p.returncode == 0, err
         assert "ok" in out
+
+
+def test_alu_denominator_is_the_larger_of_the_measured_loop_and_the_unit_counts():
+    """A register-only FMA loop measured under a power cap must not flatter the ALU-bound fractions:
+    the denominator is never below 148 SMs x 128 (64) lanes x 2 x the sampled clock."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from workloads import F32, F64
+    derived32 = 148 * 128 * 2 * 1965e6 / 1e12
+    assert abs(bench.fma_peak(None, F32, 1965.0) - derived32) < 1e-9
+    assert abs(bench.fma_peak(None, F64, 1965.0) - derived32 / 2) < 1e-9
+    throttled = {"tflops": 53.8, "fp64": 25.8}
+    assert bench.fma_peak(throttled, F32, 1965.0) == bench.fma_peak(None, F32, 1965.0)
+    assert bench.fma_peak(throttled, F64, 1965.0) == bench.fma_peak(None, F64, 1965.0)
+    high = {"tflops": 80.0, "fp64": 40.0}
+    assert bench.fma_peak(high, F32, 1965.0) == 80.0 and bench.fma_peak(high, F64, 1965.0) == 40.0
+    # a row sampled at a lower clock gets the measured loop if that is larger
+    cool = {"tflops": 73.6, "fp64": 34.5}
+    assert bench.fma_peak(cool, F32, 1500.0) == 73.6
