@@ -869,8 +869,9 @@ gett_status_t gett_planner_build(gett_plan* p, const gett_tensor_desc_t* dA,
         // of two.  Long contractions keep the 128-row tile's higher flops per byte.
         int tmh = o.tile_m;
         if (tmh == 0)
-            tmh = (tn == 128 && p->K.size <= 128 &&
-                   (uint64_t)ceil_div(p->M.size, 64) * ceil_div(p->N.size, 128) >= 8ull * sms)
+            tmh = (tn == 128 && ((p->K.size <= 128 && p->M.size > 128 &&
+                                  (uint64_t)ceil_div(p->M.size, 64) * ceil_div(p->N.size, 128) >= 8ull * sms) ||
+                                 p->M.size <= 64)) // (all rows fit the lower tile: half the padding)
                       ? 64
                       : 128;
         if (tmh == 64 && tn != 128)

@@ -210,6 +210,17 @@ def test_sliced_contractions_take_the_tile_that_moves_the_fewest_operand_bytes()
     assert g.Plan(workload("cfg4").contraction, g.GETT_BF16_F32).info.split_k == 1
 
 
+def test_fp32_tile_height_follows_the_rows_there_are():
+    """Strict fp32: 64-row tiles when all rows fit them (a 24-row output in a 128-row tile is 81 %
+    padding, in a 64-row tile 62 %), 128-row tiles when 64-row tiles would not pad less."""
+    ttm = parse_spec("C[a,b,c] = A[b,d,a] * B[d,c]", dict(a=384, b=384, c=24, d=384))      # abc-bda-dc
+    i = g.Plan(ttm, g.GETT_F32).info
+    assert i.swapped == 1 and (i.tile_m, i.tile_n) == (64, 128)
+    wide = parse_spec("C[a,b,c,d] = A[e,a] * B[e,b,c,d]", dict(a=96, b=84, c=84, d=84, e=96))  # abcd-ea-ebcd
+    assert g.Plan(wide, g.GETT_F32).info.tile_m == 128
+    assert g.Plan(workload("cfg5").contraction, g.GETT_F32).info.tile_m == 64
+
+
 def test_paths_loaders_and_epilogues_chosen_for_the_workloads():
     want = {  # key, dtype -> (path, loader_a, loader_b, epilogue)
         # cfg1: N = 40, K = 48 -> the small-N kernel (A staged MN-major, B read once element by element)
