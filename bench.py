@@ -124,7 +124,7 @@ def run_copy_probe():
     stream = torch.cuda.current_stream()
     rows = []
     for rep in range(2):
-        for pattern in range(11):
+        for pattern in range(12):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
             asked = fn(pattern, 64, 148 * 4, buf.data_ptr(), span, stream.cuda_stream)

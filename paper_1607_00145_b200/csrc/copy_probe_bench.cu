@@ -19,6 +19,9 @@ __device__ __forceinline__ void copy16(uint32_t dst, const void* src)
 //         6: shifted by 16, lanes rotated by one (lane pairs cover whole 32-byte sectors again)
 //         7: four 128-byte runs 256 bytes apart          8: those runs shifted by 16
 //         9: those runs shifted by 64                   10: every lane in a sector of its own
+//        11: pattern 0 with the DESTINATIONS rotated by one lane: every aligned pair of lanes
+//            reads the two halves of one sector but writes to two different 32-byte units
+//            of shared memory
 __global__ void copy_probe_kernel(const char* __restrict__ g, int pattern, int iters, size_t span)
 {
     extern __shared__ __align__(1024) uint8_t sm[];
@@ -41,7 +44,8 @@ __global__ void copy_probe_kernel(const char* __restrict__ g, int pattern, int i
         case 10: off = lane * 32; break;
         default: off = lane * 16; break;
         }
-        copy16(s0 + warp * 1024 + (it & 1) * 512 + lane * 16, g + base + off);
+        const int dlane = pattern == 11 ? ((lane + 1) & 31) : lane;
+        copy16(s0 + warp * 1024 + (it & 1) * 512 + dlane * 16, g + base + off);
         // two copies per thread in flight, each to a destination of its own: a copy whose
         // destination is overwritten by a later one while it is still in flight need not be
         // carried out, which would make the byte counts depend on timing
@@ -58,7 +62,7 @@ extern "C" __attribute__((visibility("default"))) long long gett_bench_copy_prob
                                                                                   const void* src, size_t span,
                                                                                   void* stream)
 {
-    if (pattern < 0 || pattern > 10 || iters < 1 || blocks < 1 || !src || span < 1024 || span % 1024)
+    if (pattern < 0 || pattern > 11 || iters < 1 || blocks < 1 || !src || span < 1024 || span % 1024)
         return -1;
     copy_probe_kernel<<<blocks, 256, 8 * 1024, static_cast<cudaStream_t>(stream)>>>(static_cast<const char*>(src),
                                                                                    pattern, iters, span);
